@@ -1,0 +1,400 @@
+"""CPU oracle for the FreeBalance per-layer hot path.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain restatement of what the paper's method computes,
+written from the paper's equations and Algorithm 1.  It exists so the CUDA
+library can be checked against something that is not itself.  Nothing in the
+product may import it: only the tests, the smoke check and the benchmark's
+CPU-baseline leg do.  It shares no code with the CUDA path.
+
+Precision: router logits are accumulated in float64 from the same bf16 bit
+patterns the GPU reads.  Everything after top-k is exact integer / rational
+arithmetic (``int`` and ``fractions.Fraction``).
+
+Pinning status (the tests that hold each function to something other than
+itself live in ``tests/test_oracle_*.py``):
+
+* ``router_logits``      pinned: exact rational dot products on tiny inputs, and
+                          integer-valued inputs whose product is exact.
+* ``select_topk``        pinned: brute-force subset search, monotonicity of
+                          softmax, the all-equal tie case, a hand-worked
+                          group-limited example.
+* ``expert_histogram``   pinned: brute-force counting, sum = T*k.
+* ``rank_loads``         pinned: brute force, sum invariant.
+* ``swap_cost_ns``       pinned: hand-computed value for the DeepSeek-V3-shaped
+                          budget (99 858 ns) and exact rational ceiling.
+* ``plan_swaps``         pinned: two hand-worked plans, exhaustive enumeration of
+                          every iteration's choice, the paper's invariants
+                          (budget, no max-load increase, permutation, once per
+                          expert), degenerate cases with known empty plans.
+* ``dispatch_index``     pinned: brute-force ``sorted`` on tiny inputs, a
+                          hand-worked example, permutation/offset invariants.
+* ``budget_ns``          pinned: Eq. 10 special cases.
+"""
+from __future__ import annotations
+
+import dataclasses
+from fractions import Fraction
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+GATE_SOFTMAX_TOPK = 0
+GATE_SIGMOID_GROUP_TOPK = 1
+U64_OFF = 2**64 - 1          # a residual budget with this initial value is not enforced
+GROUP_SCORE_TOP = 2          # a group's score is the sum of its 2 largest selection keys
+
+
+# ----------------------------------------------------------------------------
+# Eq. 4: the linear router
+# ----------------------------------------------------------------------------
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16) to float64 exactly."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def router_logits(x_bits: np.ndarray, W_bits: np.ndarray,
+                  logit_bias: Optional[np.ndarray] = None) -> np.ndarray:
+    """g(X) = X W + 1 b^T (Eq. 4), in float64.
+
+    ``x_bits`` is [T, d] and ``W_bits`` is [E, d] (one row per expert, i.e. the
+    paper's W transposed), both bf16 bit patterns.  Used for the early pass on
+    h_{l-1} (Eq. 2) and for the normal pass on H_l (Eq. 3) alike.
+    """
+    X = bf16_bits_to_f64(x_bits)
+    W = bf16_bits_to_f64(W_bits)
+    z = X @ W.T
+    if logit_bias is not None:
+        z = z + np.asarray(logit_bias, dtype=np.float64)[None, :]
+    return z
+
+
+# ----------------------------------------------------------------------------
+# "the original top-k rule" (text after Eq. 4; the rule itself is the model's)
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass(frozen=True)
+class Gate:
+    E: int
+    k: int
+    gate: int = GATE_SOFTMAX_TOPK
+    n_group: int = 1
+    topk_group: int = 1
+    renorm: int = 1
+    route_scale: float = 1.0
+
+
+def _topk_desc(key: np.ndarray, k: int) -> np.ndarray:
+    """Indices of the k largest entries per row, descending; equal keys -> lower index first."""
+    order = np.argsort(-key, axis=1, kind="stable")
+    return order[:, :k]
+
+
+def selection_keys(z: np.ndarray, g: Gate, select_bias: Optional[np.ndarray] = None
+                   ) -> Tuple[np.ndarray, np.ndarray, Optional[np.ndarray]]:
+    """Return (q, eligible, group_score).
+
+    softmax gate: q = z (softmax is strictly increasing in z for a fixed row, so
+    the top-k of the probabilities is the top-k of the logits); all experts eligible.
+    sigmoid gate: s = 1/(1+exp(-z)); q = s + select_bias; experts form n_group
+    contiguous groups; a group's score is the sum of its two largest q; only the
+    topk_group best groups (ties -> lower group) stay eligible.
+    """
+    T, E = z.shape
+    if g.gate == GATE_SOFTMAX_TOPK:
+        return z, np.ones((T, E), dtype=bool), None
+    s = 1.0 / (1.0 + np.exp(-z))
+    q = s if select_bias is None else s + np.asarray(select_bias, dtype=np.float64)[None, :]
+    gs = E // g.n_group
+    qg = q.reshape(T, g.n_group, gs)
+    n_top = min(GROUP_SCORE_TOP, gs)
+    part = -np.sort(-qg, axis=2)[:, :, :n_top]
+    group_score = part.sum(axis=2)
+    kept = _topk_desc(group_score, g.topk_group)
+    elig_g = np.zeros((T, g.n_group), dtype=bool)
+    np.put_along_axis(elig_g, kept, True, axis=1)
+    eligible = np.repeat(elig_g, gs, axis=1)
+    return q, eligible, group_score
+
+
+def select_topk(z: np.ndarray, g: Gate, select_bias: Optional[np.ndarray] = None
+                ) -> Tuple[np.ndarray, np.ndarray]:
+    """Top-k expert ids (descending key, ties -> lower id) and routing weights.
+
+    Weights: softmax gate -> softmax probabilities of the chosen experts,
+    renormalised over the k chosen when ``renorm``; sigmoid gate -> the unbiased
+    sigmoid scores of the chosen experts, divided by their sum when ``renorm``,
+    times ``route_scale``.
+    """
+    T, E = z.shape
+    q, eligible, _ = selection_keys(z, g, select_bias)
+    masked = np.where(eligible, q, -np.inf)
+    ids = _topk_desc(masked, g.k).astype(np.int32)
+    if g.gate == GATE_SOFTMAX_TOPK:
+        zmax = z.max(axis=1, keepdims=True) if E else z
+        p = np.exp(z - zmax)
+        p = p / p.sum(axis=1, keepdims=True)
+        w = np.take_along_axis(p, ids, axis=1)
+        if g.renorm:
+            w = w / w.sum(axis=1, keepdims=True)
+    else:
+        s = 1.0 / (1.0 + np.exp(-z))
+        w = np.take_along_axis(s, ids, axis=1)
+        if g.renorm:
+            w = w / w.sum(axis=1, keepdims=True)
+        w = w * g.route_scale
+    return ids, w
+
+
+def near_tie_margins(z: np.ndarray, g: Gate, select_bias: Optional[np.ndarray] = None
+                     ) -> Tuple[np.ndarray, np.ndarray]:
+    """Per token: (key gap between the k-th and (k+1)-th eligible expert,
+    score gap between the last kept and first dropped group).  +inf where there
+    is no (k+1)-th candidate / no dropped group.  A token whose gaps are below a
+    threshold may legitimately route differently under fp32 arithmetic."""
+    T, E = z.shape
+    q, eligible, group_score = selection_keys(z, g, select_bias)
+    masked = np.where(eligible, q, -np.inf)
+    srt = -np.sort(-masked, axis=1)
+    if g.k < E:
+        nxt = srt[:, g.k]
+        key_gap = np.where(np.isfinite(nxt), srt[:, g.k - 1] - nxt, np.inf)
+    else:
+        key_gap = np.full(T, np.inf)
+    if group_score is not None and g.topk_group < g.n_group:
+        gs = -np.sort(-group_score, axis=1)
+        group_gap = gs[:, g.topk_group - 1] - gs[:, g.topk_group]
+    else:
+        group_gap = np.full(T, np.inf)
+    return key_gap, group_gap
+
+
+# ----------------------------------------------------------------------------
+# Eq. 5: predicted expert workload; Algorithm 1 line 2: rank loads
+# ----------------------------------------------------------------------------
+def expert_histogram(ids: np.ndarray, E: int) -> np.ndarray:
+    """n_e = number of tokens whose assignment set contains e (Eq. 5)."""
+    counts = np.zeros(E, dtype=np.int64)
+    for e in np.asarray(ids).reshape(-1):
+        counts[int(e)] += 1
+    return counts
+
+
+def rank_of_slot(slot: int, m: int) -> int:
+    return slot // m
+
+
+def rank_loads(counts: Sequence[int], expert_to_slot: Sequence[int], R: int) -> List[int]:
+    """L_r = sum of n_e over the experts placed on rank r (Algorithm 1, line 2).
+    Slot p belongs to rank p // m with m = E / R expert slots per rank."""
+    E = len(counts)
+    m = E // R
+    L = [0] * R
+    for e in range(E):
+        L[rank_of_slot(int(expert_to_slot[e]), m)] += int(counts[e])
+    return L
+
+
+# ----------------------------------------------------------------------------
+# Eqs. 9, 10: cost model and budget
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass(frozen=True)
+class Budget:
+    max_swaps: int = 0
+    global_ns: int = U64_OFF
+    rank_ns: int = U64_OFF
+    link_ns: int = U64_OFF
+    tau_tokens: int = 0
+    gamma_num: int = 0
+    gamma_den: int = 1
+    alpha_ns: Tuple[int, int] = (0, 0)          # [intra-node, inter-node]
+    fs_per_byte: Tuple[int, int] = (0, 0)       # 1/beta in femtoseconds per byte
+    ranks_per_node: int = 0                     # 0 -> every rank in one node
+    expert_bytes: int = 0                       # S(e), uniform ...
+    expert_bytes_table: Optional[Tuple[int, ...]] = None   # ... or one size per expert
+
+
+def budget_ns(t_attn_ns: int, delta_ns: int) -> int:
+    """B = max(0, T_attn - delta) (Eq. 10)."""
+    return max(0, int(t_attn_ns) - int(delta_ns))
+
+
+def link_class(a: int, b: int, ranks_per_node: int) -> int:
+    if ranks_per_node <= 0:
+        return 0
+    return 0 if a // ranks_per_node == b // ranks_per_node else 1
+
+
+def link_id(a: int, b: int, ranks_per_node: int):
+    """Intra-node: the unordered rank pair.  Inter-node: the unordered node pair."""
+    if link_class(a, b, ranks_per_node) == 0:
+        return ("rank", min(a, b), max(a, b))
+    na, nb = a // ranks_per_node, b // ranks_per_node
+    return ("node", min(na, nb), max(na, nb))
+
+
+def swap_cost_ns(bud: Budget, a: int, b: int, e_a: int = 0, e_b: int = 0) -> int:
+    """C(s) = alpha_ab + (S(e_a) + S(e_b)) / beta_ab (Eq. 9) in whole nanoseconds:
+    the transfer term is rounded up and the total is at least 1 ns."""
+    cls = link_class(a, b, bud.ranks_per_node)
+    if bud.expert_bytes_table is not None:
+        size = int(bud.expert_bytes_table[e_a]) + int(bud.expert_bytes_table[e_b])
+    else:
+        size = 2 * bud.expert_bytes
+    transfer = Fraction(size * bud.fs_per_byte[cls], 10**6)
+    ceil_transfer = -((-transfer.numerator) // transfer.denominator)
+    return max(1, bud.alpha_ns[cls] + ceil_transfer)
+
+
+# ----------------------------------------------------------------------------
+# Eq. 8 and Algorithm 1 lines 3-8: the deterministic greedy planner
+# ----------------------------------------------------------------------------
+def objective(L: Sequence[int], gamma: Fraction) -> Fraction:
+    """Phi(L) = max_r L_r + gamma * sum_r (L_r - mean)^2 (Eq. 8), exact."""
+    R = len(L)
+    mean = Fraction(sum(L), R)
+    return Fraction(max(L)) + gamma * sum((Fraction(x) - mean) ** 2 for x in L)
+
+
+def plan_swaps(counts: Sequence[int], expert_to_slot: Sequence[int], R: int, bud: Budget,
+               layer_id: int = 0):
+    """Budgeted greedy expert-swap planning (Algorithm 1 lines 2-8 with the
+    ordering, conflict and budget rules of "Budgeted Expert-Swap Planning").
+
+    Returns (swaps, expert_to_slot_out, load_before, load_after) where each swap
+    is (src_rank a, dst_rank b, expert on a, expert on b).
+
+    One loop iteration = one pass of: take the most and the least loaded rank
+    (the frontier), enumerate their expert pairs, drop pairs containing an expert
+    already moved in this call, drop pairs with non-positive benefit (Eq. 8) or a
+    cost that some residual budget cannot cover, and accept the pair with the
+    largest benefit / cost; ties go to the lexicographically smallest
+    (layer, a, b, e_a, e_b).  Loads and residual budgets are then updated
+    (Eqs. 6, 7).  The loop stops when the imbalance max-min is not above tau, the
+    swap cap is reached, or no pair survives.
+    """
+    E = len(counts)
+    m = E // R
+    n = [int(c) for c in counts]
+    pi = [int(p) for p in expert_to_slot]
+    gamma = Fraction(bud.gamma_num, bud.gamma_den) if bud.gamma_den else Fraction(0)
+    L = rank_loads(n, pi, R)
+    load_before = list(L)
+    selected = [False] * E
+    g_res = bud.global_ns
+    r_res = [bud.rank_ns] * R
+    l_res = {}
+    swaps = []
+    while len(swaps) < bud.max_swaps:
+        a = max(range(R), key=lambda r: (L[r], -r))      # most loaded, lowest index on ties
+        b = min(range(R), key=lambda r: (L[r], r))       # least loaded, lowest index on ties
+        if L[a] - L[b] <= bud.tau_tokens:
+            break
+        phi = objective(L, gamma)
+        lk = link_id(a, b, bud.ranks_per_node)
+        lres = l_res.get(lk, bud.link_ns)
+        on_a = [e for e in range(E) if rank_of_slot(pi[e], m) == a and not selected[e]]
+        on_b = [e for e in range(E) if rank_of_slot(pi[e], m) == b and not selected[e]]
+        best = None          # (benefit/cost, tie-break tuple, cost, new loads)
+        for ea in on_a:
+            for eb in on_b:
+                Ln = list(L)
+                Ln[a] = L[a] - n[ea] + n[eb]                      # Eq. 6
+                Ln[b] = L[b] - n[eb] + n[ea]                      # Eq. 7
+                benefit = phi - objective(Ln, gamma)
+                if benefit <= 0:
+                    continue
+                cost = swap_cost_ns(bud, a, b, ea, eb)            # Eq. 9
+                if bud.global_ns != U64_OFF and cost > g_res:
+                    continue
+                if bud.rank_ns != U64_OFF and (cost > r_res[a] or cost > r_res[b]):
+                    continue
+                if bud.link_ns != U64_OFF and cost > lres:
+                    continue
+                ratio = benefit / cost
+                tie = (layer_id, a, b, ea, eb)
+                if best is None or ratio > best[0] or (ratio == best[0] and tie < best[1]):
+                    best = (ratio, tie, cost, Ln)
+        if best is None:
+            break
+        _, (_, _, _, ea, eb), cost, L = best
+        pi[ea], pi[eb] = pi[eb], pi[ea]
+        selected[ea] = selected[eb] = True
+        if bud.global_ns != U64_OFF:
+            g_res -= cost
+        if bud.rank_ns != U64_OFF:
+            r_res[a] -= cost
+            r_res[b] -= cost
+        if bud.link_ns != U64_OFF:
+            l_res[lk] = lres - cost
+        swaps.append((a, b, ea, eb))
+    return swaps, pi, load_before, list(L)
+
+
+# ----------------------------------------------------------------------------
+# Stage 4: dispatch index under the committed placement
+# ----------------------------------------------------------------------------
+def dispatch_index(ids: np.ndarray, expert_to_slot: Sequence[int], R: int):
+    """Token -> expert dispatch order under placement pi'.
+
+    Assignment (i, j) (token i, j-th chosen expert) goes to physical slot
+    p = pi'[ids[i, j]].  Assignments are laid out by (p, i) ascending, so the
+    tokens of one slot are contiguous, the slots of one rank are contiguous and
+    tokens keep their order inside a slot.
+
+    Returns (slot_offsets [E+1], rank_offsets [R+1], perm [T*k], inv_perm [T*k],
+    rank_load [R]); perm[pos] = i*k + j and inv_perm[i*k + j] = pos.
+    """
+    ids = np.asarray(ids)
+    T, k = ids.shape
+    E = len(expert_to_slot)
+    m = E // R
+    flat = [(int(expert_to_slot[int(ids[i, j])]), i, i * k + j) for i in range(T) for j in range(k)]
+    flat.sort(key=lambda t: (t[0], t[1]))
+    perm = np.array([f for (_, _, f) in flat], dtype=np.int64).reshape(-1)
+    inv_perm = np.zeros(T * k, dtype=np.int64)
+    for pos, f in enumerate(perm):
+        inv_perm[f] = pos
+    slot_count = [0] * E
+    for (p, _, _) in flat:
+        slot_count[p] += 1
+    slot_offsets = [0] * (E + 1)
+    for p in range(E):
+        slot_offsets[p + 1] = slot_offsets[p] + slot_count[p]
+    rank_offsets = [slot_offsets[r * m] for r in range(R)] + [slot_offsets[E]]
+    rank_load = [rank_offsets[r + 1] - rank_offsets[r] for r in range(R)]
+    return (np.array(slot_offsets, dtype=np.int64), np.array(rank_offsets, dtype=np.int64),
+            perm, inv_perm, np.array(rank_load, dtype=np.int64))
+
+
+# ----------------------------------------------------------------------------
+# Evaluation metrics (Evaluation, "Metrics")
+# ----------------------------------------------------------------------------
+def max_over_mean(L: Sequence[int]) -> float:
+    s = sum(int(x) for x in L)
+    return float(max(L)) * len(L) / s if s else 1.0
+
+
+def topk_hit_rate(ids_early: np.ndarray, ids_final: np.ndarray) -> float:
+    """Fraction of final top-k assignments recovered by the early pass."""
+    T, k = ids_final.shape
+    hit = 0
+    for i in range(T):
+        hit += len(set(ids_early[i].tolist()) & set(ids_final[i].tolist()))
+    return hit / (T * k) if T * k else 1.0
+
+
+# ----------------------------------------------------------------------------
+# One layer end to end, in the order of Algorithm 1
+# ----------------------------------------------------------------------------
+def layer_step(h_prev_bits, H_bits, W_bits, gate: Gate, R: int, expert_to_slot, bud: Budget,
+               select_bias=None, logit_bias=None, layer_id: int = 0):
+    """predict -> plan -> (placement committed) -> normal routing -> dispatch index."""
+    z_early = router_logits(h_prev_bits, W_bits, logit_bias)                   # Eq. 2
+    ids_early, _ = select_topk(z_early, gate, select_bias)
+    counts = expert_histogram(ids_early, gate.E)                               # Eq. 5
+    swaps, pi_new, load_before, load_after = plan_swaps(counts, expert_to_slot, R, bud, layer_id)
+    z = router_logits(H_bits, W_bits, logit_bias)                              # Eq. 3
+    ids, w = select_topk(z, gate, select_bias)
+    disp = dispatch_index(ids, pi_new, R)
+    return dict(z_early=z_early, ids_early=ids_early, counts=counts, swaps=swaps, pi_new=pi_new,
+                load_before=load_before, load_after=load_after, z=z, ids=ids, w=w, dispatch=disp)

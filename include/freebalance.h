@@ -1,0 +1,219 @@
+/*
+ * freebalance.h - C ABI of the B200 (sm_100a) FreeBalance hot path.
+ *
+ * One call sequence per MoE layer l, following the paper's four-stage overview
+ * (Method, "Motivation and Overview") and Algorithm 1:
+ *
+ *   1. fb_predict_load      early router pass g_l(h_{l-1}) (Eqs. 2, 4), the model's
+ *                           top-k rule, predicted expert workload n_e (Eq. 5)
+ *   2. fb_plan_swaps        rank loads under the placement pi (Alg. 1 line 2), cost
+ *                           model (Eq. 9), budgets (Eq. 10), deterministic greedy
+ *                           pairwise swaps under the load objective (Eqs. 6-8)
+ *      fb_predict_and_plan  1 + 2 in a single kernel launch
+ *   3. (weight migration: not part of this library)
+ *   4. fb_route_dispatch    normal router pass g_l(H_l) (Eq. 3), authoritative top-k
+ *                           and routing weights, and the token -> expert dispatch
+ *                           index under the committed placement pi'
+ *
+ * Expert-parallel ranks are logical: a placement maps expert e to a physical slot
+ * p = expert_to_slot[e] in [0, E); slot p belongs to rank p / (E / R).  Everything
+ * runs on one GPU.
+ *
+ * Conventions
+ *   - "dev" pointers are device memory owned by the caller, 16-byte aligned,
+ *     dense row-major.  "host" pointers are ordinary host memory.
+ *   - Structs (fb_config, fb_router, fb_budget) are host structs read during the call.
+ *   - Calls enqueue work on `stream` and return without synchronising, except
+ *     fb_layer_step_host and fb_device_status which block until the stream drains.
+ *   - No call throws or aborts.  Argument and shape problems are reported by the
+ *     return value and nothing is launched.  Problems only the device can see (a
+ *     placement that is not a bijection, count sums beyond the planner's range, a
+ *     bounded wait inside a kernel that expired) set a device status word which
+ *     fb_device_status returns; outputs of that call are then unspecified but every
+ *     write stays inside the caller's buffers.
+ *   - There is no CPU fallback: without a CUDA device fb_create fails.
+ */
+#ifndef FREEBALANCE_H_
+#define FREEBALANCE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fb_ctx fb_ctx;              /* opaque; owns a few KB..MB of device scratch */
+typedef void* fb_stream;                   /* a cudaStream_t (NULL = default stream)      */
+
+typedef enum {
+  FB_OK = 0,
+  FB_ERR_INVALID_ARG = 1,                  /* NULL pointer, negative size, bad struct field   */
+  FB_ERR_UNSUPPORTED_SHAPE = 2,            /* shape outside the limits listed at fb_create    */
+  FB_ERR_CUDA = 3,                         /* a CUDA runtime / driver call failed             */
+  FB_ERR_BAD_PLACEMENT = 4,                /* device: expert_to_slot is not a bijection       */
+  FB_ERR_TIMEOUT = 5,                      /* device: a bounded wait inside a kernel expired  */
+  FB_ERR_RANGE = 6                         /* device: sum of counts exceeds FB_MAX_COUNT_SUM  */
+} fb_status;
+
+/* The model's "original top-k rule" applied to the router logits (text after Eq. 4). */
+typedef enum {
+  FB_GATE_SOFTMAX_TOPK = 0,                /* key = logit; weights = softmax probabilities    */
+  FB_GATE_SIGMOID_GROUP_TOPK = 1           /* key = sigmoid(logit) + select_bias, restricted  */
+                                           /* to the topk_group best of n_group expert groups */
+} fb_gate;
+
+#define FB_MAX_EXPERTS   256
+#define FB_MAX_RANKS     64
+#define FB_MAX_TOPK      8
+#define FB_MAX_GROUPS    32
+#define FB_MAX_COUNT_SUM (1u << 21)        /* planner: sum of counts <= 2^21                  */
+#define FB_MAX_GAMMA_NUM (1u << 20)
+#define FB_BUDGET_OFF    UINT64_MAX        /* a residual budget that is not enforced          */
+
+typedef struct {
+  int32_t T_max;        /* largest token count any call will pass                              */
+  int32_t d;            /* hidden size; multiple of 8                                          */
+  int32_t E;            /* routed experts, 1..256                                              */
+  int32_t k;            /* experts per token, 1..min(E, 8)                                     */
+  int32_t R;            /* logical ranks, 1..64, divides E                                     */
+  int32_t gate;         /* fb_gate                                                             */
+  int32_t n_group;      /* sigmoid gate: number of contiguous expert groups (divides E, <=32)  */
+  int32_t topk_group;   /* sigmoid gate: groups kept per token (1..min(n_group, 8))            */
+  int32_t renorm;       /* 1: routing weights divided by their sum over the k chosen           */
+  float   route_scale;  /* sigmoid gate: factor applied to the routing weights                 */
+} fb_config;
+
+/* The frozen router of the target layer, shared by both invocations (Eqs. 2-4). */
+typedef struct {
+  const void*  W;            /* dev bf16 [E][d]: row e = column e of the paper's W (K-major)   */
+  const float* logit_bias;   /* dev fp32 [E] or NULL: b of Eq. 4                               */
+  const float* select_bias;  /* dev fp32 [E] or NULL: added to the sigmoid score for selection */
+                             /* only (never to the routing weight); ignored by the softmax gate */
+} fb_router;
+
+/* Planner parameters: Algorithm 1's budget B and threshold tau, the weight gamma of
+ * Eq. 8 and the cost model of Eq. 9 in integer units so that every rank (and the CPU
+ * oracle) reproduces the same plan bit for bit. */
+typedef struct {
+  uint32_t max_swaps;        /* hard cap on accepted swaps (0 keeps the placement), <= E/2     */
+  uint64_t global_ns;        /* residual budgets, initial value B_l of Eq. 10: one for the     */
+  uint64_t rank_ns;          /*   whole plan, one per rank, one per link.  Every accepted swap */
+  uint64_t link_ns;          /*   is charged C(s) to each it touches; FB_BUDGET_OFF disables.  */
+  uint32_t tau_tokens;       /* loop only while max_r L_r - min_r L_r > tau_tokens             */
+  uint32_t gamma_num;        /* gamma = gamma_num / gamma_den (<= FB_MAX_GAMMA_NUM / any);     */
+  uint32_t gamma_den;        /*   gamma_den == 0 means gamma = 0                               */
+  uint64_t alpha_ns[2];      /* alpha of Eq. 9: [0] same node, [1] different nodes             */
+  uint64_t fs_per_byte[2];   /* 1 / beta of Eq. 9 in femtoseconds per byte, same indexing      */
+  int32_t  ranks_per_node;   /* <= 0: all ranks in one node                                    */
+  uint64_t expert_bytes;     /* S(e) when every expert has the same size                       */
+  const uint64_t* expert_bytes_table; /* dev u64 [E] per-expert S(e), or NULL for the uniform size */
+} fb_budget;
+
+/* One accepted swap: expert_src leaves src_rank (the overloaded one) for dst_rank,
+ * expert_dst travels the other way. */
+typedef struct { int32_t src_rank, dst_rank, expert_src, expert_dst; } fb_swap;
+
+/* ------------------------------------------------------------------------------------
+ * Context.  fb_create allocates all device scratch the other calls need (sized from
+ * T_max and E) on `device`; fb_destroy frees it.  No other call allocates, except the
+ * first fb_layer_step_host (its staging buffers).
+ * Limits (FB_ERR_UNSUPPORTED_SHAPE otherwise): 1 <= E <= 256, 1 <= k <= min(E, 8),
+ * 1 <= R <= 64 with R | E, d >= 8 with 8 | d, 0 <= T <= T_max < 2^31 / max(E, k);
+ * sigmoid gate: n_group | E, n_group <= 32, 1 <= topk_group <= min(n_group, 8),
+ * topk_group * (E / n_group) >= k.
+ * ------------------------------------------------------------------------------------ */
+fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device);
+fb_status fb_destroy(fb_ctx* ctx);
+
+/* Eq. 10: B = max(0, t_attn - delta), all in nanoseconds.  Pure host arithmetic. */
+uint64_t fb_budget_ns(uint64_t t_attn_ns, uint64_t delta_ns);
+
+/* Eq. 9 for a pair of ranks with uniform expert size: C = alpha + 2 S / beta in whole
+ * nanoseconds (transfer term rounded up, total at least 1).  Pure host arithmetic;
+ * returns 0 if the product overflows 64 bits. */
+uint64_t fb_swap_cost_ns(const fb_budget* budget, int32_t rank_a, int32_t rank_b);
+
+/* Stage 1 - residual workload prediction (Eqs. 2, 4, 5).
+ *   x           dev bf16 [T][d]  residual hidden states h_{l-1}
+ *   counts      dev u32 [E]      out: n_e = number of tokens whose top-k contains e
+ *   topk_ids    dev i32 [T][k]   out, optional (NULL to skip): chosen experts per token,
+ *                                descending selection key, equal keys -> lower id first
+ *   logits      dev f32 [T][E]   out, optional debug dump of g(x) (NULL to skip)
+ * T == 0 writes zero counts. */
+fb_status fb_predict_load(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T,
+                          uint32_t* counts, int32_t* topk_ids, float* logits, fb_stream stream);
+
+/* Stage 2 - budgeted expert-swap planning (Algorithm 1 lines 2-8; Eqs. 6-9).
+ * Each iteration takes the most and the least loaded rank (lowest index on ties),
+ * enumerates pairs of their experts not yet moved in this call, drops pairs whose
+ * benefit Phi(L) - Phi(L') (Eq. 8) is not positive or whose cost C(s) exceeds a
+ * residual budget, and accepts the pair with the largest benefit / cost (compared
+ * exactly; ties -> smallest (expert_src, expert_dst)).  It stops when max - min load
+ * <= tau_tokens, after max_swaps swaps, or when no pair survives.
+ *   counts              dev u32 [E]        predicted workload
+ *   expert_to_slot      dev i32 [E]        current placement pi (a bijection onto 0..E-1)
+ *   expert_to_slot_out  dev i32 [E]        out: pi' (may alias expert_to_slot)
+ *   swaps               dev fb_swap [max_swaps]  out: accepted swaps in order
+ *   n_swaps             dev i32 [1]        out
+ *   load_before/after   dev u32 [R]        out: rank loads under pi / pi'
+ * An empty plan leaves pi' == pi. */
+fb_status fb_plan_swaps(fb_ctx* ctx, const uint32_t* counts, const int32_t* expert_to_slot,
+                        const fb_budget* budget, int32_t layer_id,
+                        int32_t* expert_to_slot_out, fb_swap* swaps, int32_t* n_swaps,
+                        uint32_t* load_before, uint32_t* load_after, fb_stream stream);
+
+/* Stages 1 + 2 in one launch: the thread block that finishes last runs the planner. */
+fb_status fb_predict_and_plan(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T,
+                              const int32_t* expert_to_slot, const fb_budget* budget,
+                              int32_t layer_id, uint32_t* counts, int32_t* expert_to_slot_out,
+                              fb_swap* swaps, int32_t* n_swaps,
+                              uint32_t* load_before, uint32_t* load_after, fb_stream stream);
+
+/* Stage 4 - normal routing (Eq. 3) and the dispatch index under pi'.  Never looks at
+ * the prediction: the normal router alone decides the assignments.
+ *   x             dev bf16 [T][d]   H_l, the router's normal input
+ *   topk_ids      dev i32 [T][k]    out: chosen experts (order as in fb_predict_load)
+ *   topk_w        dev f32 [T][k]    out: routing weights of those experts
+ *   slot_offsets  dev u32 [E+1]     out: exclusive prefix sums of tokens per physical slot
+ *   rank_offsets  dev u32 [R+1]     out: rank_offsets[r] = slot_offsets[r * E / R]
+ *   perm          dev i32 [T*k]     out: perm[pos] = i*k + j, ordered by (slot, token i)
+ *   inv_perm      dev i32 [T*k]     out: inv_perm[i*k + j] = pos
+ *   rank_load     dev u32 [R]       out: realised tokens per rank
+ *   logits        dev f32 [T][E]    out, optional debug dump (NULL to skip) */
+fb_status fb_route_dispatch(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T,
+                            const int32_t* expert_to_slot, int32_t* topk_ids, float* topk_w,
+                            uint32_t* slot_offsets, uint32_t* rank_offsets,
+                            int32_t* perm, int32_t* inv_perm, uint32_t* rank_load,
+                            float* logits, fb_stream stream);
+
+/* One whole layer (fb_predict_and_plan, then fb_route_dispatch under the new
+ * placement) with HOST buffers for the per-step tensors: h_prev, H, expert_to_slot
+ * are copied to the device, every output pointer receives host data, and the call
+ * returns after the stream has drained.  The router stays on the device (frozen
+ * weights).  Device staging is allocated on the first call.  Any output pointer may
+ * be NULL to skip its copy.  Pinned host memory makes the copies asynchronous. */
+fb_status fb_layer_step_host(fb_ctx* ctx, const fb_router* router,
+                             const void* h_prev_host, const void* H_host, int32_t T,
+                             const int32_t* expert_to_slot_host, const fb_budget* budget,
+                             int32_t layer_id,
+                             uint32_t* counts, int32_t* expert_to_slot_out, fb_swap* swaps,
+                             int32_t* n_swaps, uint32_t* load_before, uint32_t* load_after,
+                             int32_t* topk_ids, float* topk_w, uint32_t* slot_offsets,
+                             uint32_t* rank_offsets, int32_t* perm, int32_t* inv_perm,
+                             uint32_t* rank_load, fb_stream stream);
+
+/* Synchronises `stream`, returns the device status word in *word (FB_OK, or the
+ * first FB_ERR_BAD_PLACEMENT / FB_ERR_TIMEOUT / FB_ERR_RANGE raised since the last
+ * query) and clears it. */
+fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream);
+
+/* Kernels this library has launched through `ctx` so far (for benchmarks). */
+uint64_t fb_launch_count(const fb_ctx* ctx);
+
+/* Text for a status code; never NULL. */
+const char* fb_status_string(fb_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* FREEBALANCE_H_ */

@@ -1,0 +1,211 @@
+"""ctypes binding of libfreebalance.so: argument marshalling only.
+
+Every function below has the name and meaning of the C entry point declared in
+``include/freebalance.h``; tensors are torch CUDA tensors whose ``data_ptr()`` is
+handed to the library, the stream is torch's current stream unless given.  There
+is no fallback: if the shared library is missing or fails to load this raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+_U64_OFF = 2**64 - 1
+
+
+class FbConfig(ctypes.Structure):
+    _fields_ = [("T_max", ctypes.c_int32), ("d", ctypes.c_int32), ("E", ctypes.c_int32),
+                ("k", ctypes.c_int32), ("R", ctypes.c_int32), ("gate", ctypes.c_int32),
+                ("n_group", ctypes.c_int32), ("topk_group", ctypes.c_int32),
+                ("renorm", ctypes.c_int32), ("route_scale", ctypes.c_float)]
+
+
+class FbRouter(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("logit_bias", ctypes.c_void_p), ("select_bias", ctypes.c_void_p)]
+
+
+class FbBudget(ctypes.Structure):
+    _fields_ = [("max_swaps", ctypes.c_uint32), ("global_ns", ctypes.c_uint64),
+                ("rank_ns", ctypes.c_uint64), ("link_ns", ctypes.c_uint64),
+                ("tau_tokens", ctypes.c_uint32), ("gamma_num", ctypes.c_uint32),
+                ("gamma_den", ctypes.c_uint32), ("alpha_ns", ctypes.c_uint64 * 2),
+                ("fs_per_byte", ctypes.c_uint64 * 2), ("ranks_per_node", ctypes.c_int32),
+                ("expert_bytes", ctypes.c_uint64), ("expert_bytes_table", ctypes.c_void_p)]
+
+
+FB_OK = 0
+FB_ERR_INVALID_ARG = 1
+FB_ERR_UNSUPPORTED_SHAPE = 2
+FB_ERR_CUDA = 3
+FB_ERR_BAD_PLACEMENT = 4
+FB_ERR_TIMEOUT = 5
+FB_ERR_RANGE = 6
+
+EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_predict_load",
+           "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
+           "fb_device_status", "fb_launch_count", "fb_status_string"]
+
+_lib = None
+
+
+class FbError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().fb_status_string(status).decode() if _lib is not None else str(status)
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if the sources are newer) the CUDA library."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if _build.is_stale():
+        path = _build.build()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with paper_2608_14205_b200/build.py")
+    L = ctypes.CDLL(path)
+    vp, i32, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint64
+    L.fb_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(FbConfig), ctypes.c_int]
+    L.fb_destroy.argtypes = [vp]
+    L.fb_budget_ns.argtypes = [u64, u64]
+    L.fb_budget_ns.restype = u64
+    L.fb_swap_cost_ns.argtypes = [ctypes.POINTER(FbBudget), i32, i32]
+    L.fb_swap_cost_ns.restype = u64
+    L.fb_predict_load.argtypes = [vp, ctypes.POINTER(FbRouter), vp, i32, vp, vp, vp, vp]
+    L.fb_plan_swaps.argtypes = [vp, vp, vp, ctypes.POINTER(FbBudget), i32, vp, vp, vp, vp, vp, vp]
+    L.fb_predict_and_plan.argtypes = [vp, ctypes.POINTER(FbRouter), vp, i32, vp, ctypes.POINTER(FbBudget), i32,
+                                      vp, vp, vp, vp, vp, vp, vp]
+    L.fb_route_dispatch.argtypes = [vp, ctypes.POINTER(FbRouter), vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.fb_layer_step_host.argtypes = [vp, ctypes.POINTER(FbRouter), vp, vp, i32, vp, ctypes.POINTER(FbBudget), i32] \
+        + [vp] * 14
+    L.fb_device_status.argtypes = [vp, ctypes.POINTER(i32), vp]
+    L.fb_launch_count.argtypes = [vp]
+    L.fb_launch_count.restype = u64
+    L.fb_status_string.argtypes = [ctypes.c_int]
+    L.fb_status_string.restype = ctypes.c_char_p
+    for name in ("fb_create", "fb_destroy", "fb_predict_load", "fb_plan_swaps", "fb_predict_and_plan",
+                 "fb_route_dispatch", "fb_layer_step_host", "fb_device_status"):
+        getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors handed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return stream or None
+
+
+def _check(status: int, where: str) -> None:
+    if status != FB_OK:
+        raise FbError(status, where)
+
+
+def make_budget(max_swaps=0, global_ns=_U64_OFF, rank_ns=_U64_OFF, link_ns=_U64_OFF, tau_tokens=0,
+                gamma_num=0, gamma_den=1, alpha_ns=(0, 0), fs_per_byte=(0, 0), ranks_per_node=0,
+                expert_bytes=0, expert_bytes_table: Optional[torch.Tensor] = None) -> FbBudget:
+    b = FbBudget()
+    b.max_swaps, b.global_ns, b.rank_ns, b.link_ns = max_swaps, global_ns, rank_ns, link_ns
+    b.tau_tokens, b.gamma_num, b.gamma_den = tau_tokens, gamma_num, gamma_den
+    b.alpha_ns = (ctypes.c_uint64 * 2)(*alpha_ns)
+    b.fs_per_byte = (ctypes.c_uint64 * 2)(*fs_per_byte)
+    b.ranks_per_node, b.expert_bytes = ranks_per_node, expert_bytes
+    b.expert_bytes_table = _ptr(expert_bytes_table)
+    b._keepalive = expert_bytes_table
+    return b
+
+
+def make_router(W: torch.Tensor, logit_bias: Optional[torch.Tensor] = None,
+                select_bias: Optional[torch.Tensor] = None) -> FbRouter:
+    assert W.dtype == torch.bfloat16
+    r = FbRouter(_ptr(W), _ptr(logit_bias), _ptr(select_bias))
+    r._keepalive = (W, logit_bias, select_bias)
+    return r
+
+
+def fb_budget_ns(t_attn_ns: int, delta_ns: int) -> int:
+    return int(lib().fb_budget_ns(t_attn_ns, delta_ns))
+
+
+def fb_swap_cost_ns(budget: FbBudget, rank_a: int, rank_b: int) -> int:
+    return int(lib().fb_swap_cost_ns(ctypes.byref(budget), rank_a, rank_b))
+
+
+class Context:
+    """Owns an fb_ctx; methods mirror the C entry points one to one."""
+
+    def __init__(self, T_max, d, E, k, R, gate=0, n_group=1, topk_group=1, renorm=1, route_scale=1.0,
+                 device: int = 0):
+        self.cfg = FbConfig(T_max, d, E, k, R, gate, n_group, topk_group, renorm, route_scale)
+        self._h = ctypes.c_void_p()
+        _check(lib().fb_create(ctypes.byref(self._h), ctypes.byref(self.cfg), device), "fb_create")
+        self.device = device
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().fb_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def fb_predict_load(self, router, x, T, counts, topk_ids=None, logits=None, stream=None):
+        _check(lib().fb_predict_load(self._h, ctypes.byref(router), _ptr(x), T, _ptr(counts), _ptr(topk_ids),
+                                     _ptr(logits), _stream(stream)), "fb_predict_load")
+
+    def fb_plan_swaps(self, counts, expert_to_slot, budget, layer_id, expert_to_slot_out, swaps, n_swaps,
+                      load_before, load_after, stream=None):
+        _check(lib().fb_plan_swaps(self._h, _ptr(counts), _ptr(expert_to_slot), ctypes.byref(budget), layer_id,
+                                   _ptr(expert_to_slot_out), _ptr(swaps), _ptr(n_swaps), _ptr(load_before),
+                                   _ptr(load_after), _stream(stream)), "fb_plan_swaps")
+
+    def fb_predict_and_plan(self, router, x, T, expert_to_slot, budget, layer_id, counts, expert_to_slot_out,
+                            swaps, n_swaps, load_before, load_after, stream=None):
+        _check(lib().fb_predict_and_plan(self._h, ctypes.byref(router), _ptr(x), T, _ptr(expert_to_slot),
+                                         ctypes.byref(budget), layer_id, _ptr(counts), _ptr(expert_to_slot_out),
+                                         _ptr(swaps), _ptr(n_swaps), _ptr(load_before), _ptr(load_after),
+                                         _stream(stream)), "fb_predict_and_plan")
+
+    def fb_route_dispatch(self, router, x, T, expert_to_slot, topk_ids, topk_w, slot_offsets, rank_offsets,
+                          perm, inv_perm, rank_load, logits=None, stream=None):
+        _check(lib().fb_route_dispatch(self._h, ctypes.byref(router), _ptr(x), T, _ptr(expert_to_slot),
+                                       _ptr(topk_ids), _ptr(topk_w), _ptr(slot_offsets), _ptr(rank_offsets),
+                                       _ptr(perm), _ptr(inv_perm), _ptr(rank_load), _ptr(logits),
+                                       _stream(stream)), "fb_route_dispatch")
+
+    def fb_layer_step_host(self, router, h_prev_host, H_host, T, expert_to_slot_host, budget, layer_id,
+                           counts=None, expert_to_slot_out=None, swaps=None, n_swaps=None, load_before=None,
+                           load_after=None, topk_ids=None, topk_w=None, slot_offsets=None, rank_offsets=None,
+                           perm=None, inv_perm=None, rank_load=None, stream=None):
+        outs = [counts, expert_to_slot_out, swaps, n_swaps, load_before, load_after, topk_ids, topk_w,
+                slot_offsets, rank_offsets, perm, inv_perm, rank_load]
+        _check(lib().fb_layer_step_host(self._h, ctypes.byref(router), _ptr(h_prev_host), _ptr(H_host), T,
+                                        _ptr(expert_to_slot_host), ctypes.byref(budget), layer_id,
+                                        *[_ptr(o) for o in outs], _stream(stream)), "fb_layer_step_host")
+
+    def fb_device_status(self, stream=None) -> int:
+        word = ctypes.c_int32(0)
+        _check(lib().fb_device_status(self._h, ctypes.byref(word), _stream(stream)), "fb_device_status")
+        return int(word.value)
+
+    def fb_launch_count(self) -> int:
+        return int(lib().fb_launch_count(self._h))

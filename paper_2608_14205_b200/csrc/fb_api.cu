@@ -1,0 +1,464 @@
+// Host side of the C ABI declared in include/freebalance.h: argument checks, TMA
+// descriptors, kernel launches.  No computation of the method happens on the host
+// except the two pure helpers fb_budget_ns (Eq. 10) and fb_swap_cost_ns (Eq. 9).
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/freebalance.h"
+#include "fb_dispatch.cuh"
+#include "fb_planner.cuh"
+#include "fb_router.cuh"
+
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct MapEntry {
+  const void* ptr = nullptr;
+  int64_t rows = -1;
+  CUtensorMap map;
+};
+
+constexpr int kMapCache = 8;
+
+}  // namespace
+
+struct fb_ctx {
+  fb_config cfg;
+  int device = 0;
+  int N = 0;                      // experts padded to a multiple of 16 (UMMA N)
+  int stages = 0;
+  int tmem_cols = 0;
+  size_t smem_bytes = 0;
+  int max_tiles = 0;
+  EncodeTiledFn encode = nullptr;
+  // device scratch
+  uint32_t* counts_scratch = nullptr;   // [256], zero between calls
+  uint32_t* ticket = nullptr;           // [1],   zero between calls
+  int32_t* status = nullptr;            // [1]
+  uint32_t* tile_counts = nullptr;      // [max_tiles][E]
+  // descriptor cache
+  MapEntry x_maps[kMapCache];
+  MapEntry w_maps[kMapCache];
+  int x_next = 0, w_next = 0;
+  // staging for fb_layer_step_host (allocated on first use)
+  bool staged = false;
+  void* st_hprev = nullptr; void* st_H = nullptr;
+  int32_t* st_pi = nullptr; int32_t* st_pi_out = nullptr;
+  uint32_t* st_counts = nullptr; fb_swap* st_swaps = nullptr; int32_t* st_nswaps = nullptr;
+  uint32_t* st_load_before = nullptr; uint32_t* st_load_after = nullptr;
+  int32_t* st_ids = nullptr; float* st_w = nullptr;
+  uint32_t* st_slot_offsets = nullptr; uint32_t* st_rank_offsets = nullptr;
+  int32_t* st_perm = nullptr; int32_t* st_inv_perm = nullptr; uint32_t* st_rank_load = nullptr;
+  uint64_t launches = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int next_pow2_at_least_32(int n) {
+  int c = 32;
+  while (c < n) c <<= 1;
+  return c;
+}
+
+fb_status check_config(const fb_config& c) {
+  if (c.T_max < 0 || c.d <= 0 || c.E <= 0 || c.k <= 0 || c.R <= 0) return FB_ERR_INVALID_ARG;
+  if (c.gate != FB_GATE_SOFTMAX_TOPK && c.gate != FB_GATE_SIGMOID_GROUP_TOPK) return FB_ERR_INVALID_ARG;
+  if (c.E > FB_MAX_EXPERTS || c.k > FB_MAX_TOPK || c.k > c.E) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (c.R > FB_MAX_RANKS || c.E % c.R != 0) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (c.d < 8 || c.d % 8 != 0) return FB_ERR_UNSUPPORTED_SHAPE;
+  const int64_t widest = c.E > c.k ? c.E : c.k;
+  if (static_cast<int64_t>(c.T_max) * widest >= (int64_t{1} << 31)) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (c.gate == FB_GATE_SIGMOID_GROUP_TOPK) {
+    if (c.n_group <= 0 || c.topk_group <= 0) return FB_ERR_INVALID_ARG;
+    if (c.n_group > FB_MAX_GROUPS || c.E % c.n_group != 0) return FB_ERR_UNSUPPORTED_SHAPE;
+    if (c.topk_group > c.n_group || c.topk_group > FB_MAX_TOPK) return FB_ERR_UNSUPPORTED_SHAPE;
+    if (static_cast<int64_t>(c.topk_group) * (c.E / c.n_group) < c.k) return FB_ERR_UNSUPPORTED_SHAPE;
+  }
+  return FB_OK;
+}
+
+fb_status make_map(fb_ctx* ctx, MapEntry* cache, int* next, const void* ptr, int64_t rows, uint32_t box_rows,
+                   const CUtensorMap** out) {
+  for (int i = 0; i < kMapCache; ++i)
+    if (cache[i].ptr == ptr && cache[i].rows == rows) { *out = &cache[i].map; return FB_OK; }
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15u) != 0) return FB_ERR_INVALID_ARG;
+  MapEntry& e = cache[*next];
+  *next = (*next + 1) % kMapCache;
+  const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(ctx->cfg.d), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(ctx->cfg.d) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(fb::kBlockK), box_rows};
+  const cuuint32_t estride[2] = {1, 1};
+  const CUresult r = ctx->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride,
+                                 box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { e.ptr = nullptr; e.rows = -1; return FB_ERR_CUDA; }
+  e.ptr = ptr;
+  e.rows = rows;
+  *out = &e.map;
+  return FB_OK;
+}
+
+uint64_t uniform_cost(const fb_budget& b, int cls) {
+  const unsigned __int128 fs = static_cast<unsigned __int128>(b.expert_bytes) * 2u * b.fs_per_byte[cls];
+  const unsigned __int128 ns = (fs + 999999u) / 1000000u + b.alpha_ns[cls];
+  if (ns > UINT64_MAX) return 0;
+  const uint64_t c = static_cast<uint64_t>(ns);
+  return c < 1 ? 1 : c;
+}
+
+fb_status fill_plan(const fb_ctx* ctx, const fb_budget* b, const int32_t* pi, int32_t* pi_out, fb_swap* swaps,
+                    int32_t* n_swaps, uint32_t* load_before, uint32_t* load_after, fb::PlanParams* pp) {
+  if (!b || !pi || !pi_out || !n_swaps || !load_before || !load_after) return FB_ERR_INVALID_ARG;
+  if (b->max_swaps > static_cast<uint32_t>(ctx->cfg.E / 2)) return FB_ERR_INVALID_ARG;
+  if (b->max_swaps > 0 && !swaps) return FB_ERR_INVALID_ARG;
+  if (b->gamma_num > FB_MAX_GAMMA_NUM) return FB_ERR_INVALID_ARG;
+  pp->E = ctx->cfg.E;
+  pp->R = ctx->cfg.R;
+  pp->max_swaps = b->max_swaps;
+  pp->global_ns = b->global_ns;
+  pp->rank_ns = b->rank_ns;
+  pp->link_ns = b->link_ns;
+  pp->tau_tokens = b->tau_tokens;
+  pp->gamma_num = b->gamma_num;
+  pp->gamma_den = b->gamma_den;
+  for (int c = 0; c < 2; ++c) {
+    pp->alpha_ns[c] = b->alpha_ns[c];
+    pp->fs_per_byte[c] = b->fs_per_byte[c];
+    pp->uniform_cost_ns[c] = uniform_cost(*b, c);
+    if (b->expert_bytes_table == nullptr && pp->uniform_cost_ns[c] == 0) return FB_ERR_INVALID_ARG;
+  }
+  pp->ranks_per_node = b->ranks_per_node;
+  pp->expert_bytes_table = b->expert_bytes_table;
+  pp->expert_to_slot = pi;
+  pp->expert_to_slot_out = pi_out;
+  pp->swaps = swaps;
+  pp->n_swaps = n_swaps;
+  pp->load_before = load_before;
+  pp->load_after = load_after;
+  return FB_OK;
+}
+
+// Launch the router kernel in one of its three modes.
+fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T, int mode,
+                        uint32_t* counts_out, int32_t* topk_ids, float* topk_w, float* logits,
+                        const fb::PlanParams* plan, cudaStream_t stream) {
+  const CUtensorMap *mx = nullptr, *mw = nullptr;
+  fb_status st = make_map(ctx, ctx->x_maps, &ctx->x_next, x, T, fb::kTileM, &mx);
+  if (st != FB_OK) return st;
+  st = make_map(ctx, ctx->w_maps, &ctx->w_next, router->W, ctx->cfg.E, static_cast<uint32_t>(ctx->N), &mw);
+  if (st != FB_OK) return st;
+  fb::RouterParams p;
+  memset(&p, 0, sizeof(p));
+  const fb_config& c = ctx->cfg;
+  p.T = T; p.d = c.d; p.E = c.E; p.N = ctx->N; p.k = c.k;
+  p.gate = c.gate; p.n_group = c.gate == FB_GATE_SIGMOID_GROUP_TOPK ? c.n_group : 1;
+  p.topk_group = c.gate == FB_GATE_SIGMOID_GROUP_TOPK ? c.topk_group : 1;
+  p.renorm = c.renorm; p.route_scale = c.route_scale;
+  p.num_kb = (c.d + fb::kBlockK - 1) / fb::kBlockK;
+  p.stages = ctx->stages;
+  p.tmem_cols = ctx->tmem_cols;
+  p.mode = mode;
+  p.logit_bias = router->logit_bias;
+  p.select_bias = c.gate == FB_GATE_SIGMOID_GROUP_TOPK ? router->select_bias : nullptr;
+  p.counts_scratch = ctx->counts_scratch;
+  p.ticket = ctx->ticket;
+  p.status = ctx->status;
+  p.counts_out = counts_out;
+  p.topk_ids = topk_ids;
+  p.topk_w = topk_w;
+  p.logits = logits;
+  p.tile_counts = ctx->tile_counts;
+  if (plan) p.plan = *plan;
+  const int tiles = (T + fb::kTileM - 1) / fb::kTileM;
+  fb::fb_router_kernel<<<tiles, fb::kRouterThreads, ctx->smem_bytes, stream>>>(*mx, *mw, p);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status launch_plan(fb_ctx* ctx, const fb::PlanParams& pp, const uint32_t* counts, cudaStream_t stream) {
+  fb::fb_plan_kernel<<<1, fb::kPlanThreads, 0, stream>>>(pp, counts, ctx->status);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+template <typename Tp>
+bool dev_alloc(Tp** p, size_t count) {
+  return cudaMalloc(reinterpret_cast<void**>(p), (count ? count : 1) * sizeof(Tp)) == cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fb_status_string(fb_status s) {
+  switch (s) {
+    case FB_OK: return "ok";
+    case FB_ERR_INVALID_ARG: return "invalid argument";
+    case FB_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case FB_ERR_CUDA: return "CUDA call failed";
+    case FB_ERR_BAD_PLACEMENT: return "expert_to_slot is not a bijection";
+    case FB_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case FB_ERR_RANGE: return "sum of counts beyond the planner's range";
+  }
+  return "unknown status";
+}
+
+uint64_t fb_budget_ns(uint64_t t_attn_ns, uint64_t delta_ns) {
+  return t_attn_ns > delta_ns ? t_attn_ns - delta_ns : 0;
+}
+
+uint64_t fb_swap_cost_ns(const fb_budget* b, int32_t rank_a, int32_t rank_b) {
+  if (!b) return 0;
+  const int rpn = b->ranks_per_node;
+  const int cls = (rpn <= 0 || rank_a / rpn == rank_b / rpn) ? 0 : 1;
+  return uniform_cost(*b, cls);
+}
+
+fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
+  if (!out || !cfg) return FB_ERR_INVALID_ARG;
+  *out = nullptr;
+  const fb_status cs = check_config(*cfg);
+  if (cs != FB_OK) return cs;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return FB_ERR_CUDA;
+  DeviceGuard guard(device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FB_ERR_CUDA;
+  if (prop.major != 10) return FB_ERR_CUDA;            // built for sm_100a only; no fallback
+  fb_ctx* ctx = new (std::nothrow) fb_ctx();
+  if (!ctx) return FB_ERR_CUDA;
+  ctx->cfg = *cfg;
+  ctx->device = device;
+  ctx->N = (cfg->E + 15) / 16 * 16;
+  ctx->tmem_cols = next_pow2_at_least_32(ctx->N);
+  const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N) * fb::kBlockK * 2;
+  const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
+  int stages = static_cast<int>((budget - 1024) / stage_bytes);
+  if (stages > fb::kMaxStages) stages = fb::kMaxStages;
+  if (stages < 2) { delete ctx; return FB_ERR_UNSUPPORTED_SHAPE; }
+  ctx->stages = stages;
+  ctx->smem_bytes = stages * stage_bytes + 1024;
+  ctx->max_tiles = (cfg->T_max + fb::kTileM - 1) / fb::kTileM;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+    delete ctx;
+    return FB_ERR_CUDA;
+  }
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(ctx->smem_bytes)) == cudaSuccess;
+  ok = ok && dev_alloc(&ctx->counts_scratch, FB_MAX_EXPERTS) && dev_alloc(&ctx->ticket, 1) &&
+       dev_alloc(&ctx->status, 1) &&
+       dev_alloc(&ctx->tile_counts, static_cast<size_t>(ctx->max_tiles) * cfg->E);
+  ok = ok && cudaMemset(ctx->counts_scratch, 0, FB_MAX_EXPERTS * sizeof(uint32_t)) == cudaSuccess &&
+       cudaMemset(ctx->ticket, 0, sizeof(uint32_t)) == cudaSuccess &&
+       cudaMemset(ctx->status, 0, sizeof(int32_t)) == cudaSuccess;
+  if (!ok) { fb_destroy(ctx); return FB_ERR_CUDA; }
+  *out = ctx;
+  return FB_OK;
+}
+
+fb_status fb_destroy(fb_ctx* ctx) {
+  if (!ctx) return FB_OK;
+  DeviceGuard guard(ctx->device);
+  cudaDeviceSynchronize();
+  void* ptrs[] = {ctx->counts_scratch, ctx->ticket, ctx->status, ctx->tile_counts, ctx->st_hprev, ctx->st_H,
+                  ctx->st_pi, ctx->st_pi_out, ctx->st_counts, ctx->st_swaps, ctx->st_nswaps, ctx->st_load_before,
+                  ctx->st_load_after, ctx->st_ids, ctx->st_w, ctx->st_slot_offsets, ctx->st_rank_offsets,
+                  ctx->st_perm, ctx->st_inv_perm, ctx->st_rank_load};
+  for (void* p : ptrs)
+    if (p) cudaFree(p);
+  delete ctx;
+  return FB_OK;
+}
+
+fb_status fb_predict_load(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T, uint32_t* counts,
+                          int32_t* topk_ids, float* logits, fb_stream stream_) {
+  if (!ctx || !router || !router->W || !counts || T < 0) return FB_ERR_INVALID_ARG;
+  if (T > ctx->cfg.T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (T > 0 && !x) return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  if (T == 0)
+    return cudaMemsetAsync(counts, 0, ctx->cfg.E * sizeof(uint32_t), stream) == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+  return launch_router(ctx, router, x, T, fb::kModePredict, counts, topk_ids, nullptr, logits, nullptr, stream);
+}
+
+fb_status fb_plan_swaps(fb_ctx* ctx, const uint32_t* counts, const int32_t* expert_to_slot, const fb_budget* budget,
+                        int32_t layer_id, int32_t* expert_to_slot_out, fb_swap* swaps, int32_t* n_swaps,
+                        uint32_t* load_before, uint32_t* load_after, fb_stream stream_) {
+  (void)layer_id;   // constant within a call: it leads the tie-break tuple but cannot change the order
+  if (!ctx || !counts) return FB_ERR_INVALID_ARG;
+  fb::PlanParams pp;
+  memset(&pp, 0, sizeof(pp));
+  const fb_status st = fill_plan(ctx, budget, expert_to_slot, expert_to_slot_out, swaps, n_swaps, load_before,
+                                 load_after, &pp);
+  if (st != FB_OK) return st;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  return launch_plan(ctx, pp, counts, static_cast<cudaStream_t>(stream_));
+}
+
+fb_status fb_predict_and_plan(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T,
+                              const int32_t* expert_to_slot, const fb_budget* budget, int32_t layer_id,
+                              uint32_t* counts, int32_t* expert_to_slot_out, fb_swap* swaps, int32_t* n_swaps,
+                              uint32_t* load_before, uint32_t* load_after, fb_stream stream_) {
+  (void)layer_id;
+  if (!ctx || !router || !router->W || !counts || T < 0) return FB_ERR_INVALID_ARG;
+  if (T > ctx->cfg.T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (T > 0 && !x) return FB_ERR_INVALID_ARG;
+  fb::PlanParams pp;
+  memset(&pp, 0, sizeof(pp));
+  const fb_status st = fill_plan(ctx, budget, expert_to_slot, expert_to_slot_out, swaps, n_swaps, load_before,
+                                 load_after, &pp);
+  if (st != FB_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  if (T == 0) {
+    if (cudaMemsetAsync(counts, 0, ctx->cfg.E * sizeof(uint32_t), stream) != cudaSuccess) return FB_ERR_CUDA;
+    return launch_plan(ctx, pp, counts, stream);
+  }
+  return launch_router(ctx, router, x, T, fb::kModePredictPlan, counts, nullptr, nullptr, nullptr, &pp, stream);
+}
+
+fb_status fb_route_dispatch(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T,
+                            const int32_t* expert_to_slot, int32_t* topk_ids, float* topk_w, uint32_t* slot_offsets,
+                            uint32_t* rank_offsets, int32_t* perm, int32_t* inv_perm, uint32_t* rank_load,
+                            float* logits, fb_stream stream_) {
+  if (!ctx || !router || !router->W || !expert_to_slot || !slot_offsets || !rank_offsets || !rank_load || T < 0)
+    return FB_ERR_INVALID_ARG;
+  if (T > ctx->cfg.T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (T > 0 && (!x || !topk_ids || !topk_w || !perm || !inv_perm)) return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  const fb_config& c = ctx->cfg;
+  if (T == 0) {
+    if (cudaMemsetAsync(slot_offsets, 0, (c.E + 1) * sizeof(uint32_t), stream) != cudaSuccess ||
+        cudaMemsetAsync(rank_offsets, 0, (c.R + 1) * sizeof(uint32_t), stream) != cudaSuccess ||
+        cudaMemsetAsync(rank_load, 0, c.R * sizeof(uint32_t), stream) != cudaSuccess)
+      return FB_ERR_CUDA;
+    return FB_OK;
+  }
+  const fb_status st = launch_router(ctx, router, x, T, fb::kModeDispatch, nullptr, topk_ids, topk_w, logits,
+                                     nullptr, stream);
+  if (st != FB_OK) return st;
+  fb::DispatchParams dp;
+  dp.T = T; dp.k = c.k; dp.E = c.E; dp.R = c.R;
+  dp.num_tiles = (T + fb::kDispatchTile - 1) / fb::kDispatchTile;
+  dp.topk_ids = topk_ids;
+  dp.tile_counts = ctx->tile_counts;
+  dp.expert_to_slot = expert_to_slot;
+  dp.slot_offsets = slot_offsets;
+  dp.rank_offsets = rank_offsets;
+  dp.perm = perm;
+  dp.inv_perm = inv_perm;
+  dp.rank_load = rank_load;
+  dp.status = ctx->status;
+  fb::fb_dispatch_kernel<<<dp.num_tiles, fb::kDispatchThreads, 0, stream>>>(dp);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status fb_layer_step_host(fb_ctx* ctx, const fb_router* router, const void* h_prev_host, const void* H_host,
+                             int32_t T, const int32_t* expert_to_slot_host, const fb_budget* budget,
+                             int32_t layer_id, uint32_t* counts, int32_t* expert_to_slot_out, fb_swap* swaps,
+                             int32_t* n_swaps, uint32_t* load_before, uint32_t* load_after, int32_t* topk_ids,
+                             float* topk_w, uint32_t* slot_offsets, uint32_t* rank_offsets, int32_t* perm,
+                             int32_t* inv_perm, uint32_t* rank_load, fb_stream stream_) {
+  if (!ctx || !router || !expert_to_slot_host || !budget || T < 0) return FB_ERR_INVALID_ARG;
+  if (T > ctx->cfg.T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (T > 0 && (!h_prev_host || !H_host)) return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  const fb_config& c = ctx->cfg;
+  const size_t Tm = static_cast<size_t>(c.T_max), E = c.E, R = c.R, k = c.k;
+  if (!ctx->staged) {
+    const size_t act = Tm * c.d * 2;
+    bool ok = cudaMalloc(&ctx->st_hprev, act ? act : 16) == cudaSuccess &&
+              cudaMalloc(&ctx->st_H, act ? act : 16) == cudaSuccess;
+    ok = ok && dev_alloc(&ctx->st_pi, E) && dev_alloc(&ctx->st_pi_out, E) && dev_alloc(&ctx->st_counts, E) &&
+         dev_alloc(&ctx->st_swaps, E / 2 + 1) && dev_alloc(&ctx->st_nswaps, 1) &&
+         dev_alloc(&ctx->st_load_before, R) && dev_alloc(&ctx->st_load_after, R) &&
+         dev_alloc(&ctx->st_ids, Tm * k) && dev_alloc(&ctx->st_w, Tm * k) &&
+         dev_alloc(&ctx->st_slot_offsets, E + 1) && dev_alloc(&ctx->st_rank_offsets, R + 1) &&
+         dev_alloc(&ctx->st_perm, Tm * k) && dev_alloc(&ctx->st_inv_perm, Tm * k) &&
+         dev_alloc(&ctx->st_rank_load, R);
+    if (!ok) return FB_ERR_CUDA;
+    ctx->staged = true;
+  }
+  const size_t act_bytes = static_cast<size_t>(T) * c.d * 2;
+  const size_t n_assign = static_cast<size_t>(T) * k;
+  bool ok = true;
+  if (T > 0) {
+    ok = ok && cudaMemcpyAsync(ctx->st_hprev, h_prev_host, act_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ctx->st_H, H_host, act_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(ctx->st_pi, expert_to_slot_host, E * sizeof(int32_t), cudaMemcpyHostToDevice, stream) ==
+                 cudaSuccess;
+  if (!ok) return FB_ERR_CUDA;
+  fb_status st = fb_predict_and_plan(ctx, router, ctx->st_hprev, T, ctx->st_pi, budget, layer_id, ctx->st_counts,
+                                     ctx->st_pi_out, ctx->st_swaps, ctx->st_nswaps, ctx->st_load_before,
+                                     ctx->st_load_after, stream);
+  if (st != FB_OK) return st;
+  st = fb_route_dispatch(ctx, router, ctx->st_H, T, ctx->st_pi_out, ctx->st_ids, ctx->st_w, ctx->st_slot_offsets,
+                         ctx->st_rank_offsets, ctx->st_perm, ctx->st_inv_perm, ctx->st_rank_load, nullptr, stream);
+  if (st != FB_OK) return st;
+  auto back = [&](void* dst, const void* src, size_t bytes) {
+    if (dst && bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  };
+  back(counts, ctx->st_counts, E * sizeof(uint32_t));
+  back(expert_to_slot_out, ctx->st_pi_out, E * sizeof(int32_t));
+  back(swaps, ctx->st_swaps, budget->max_swaps * sizeof(fb_swap));
+  back(n_swaps, ctx->st_nswaps, sizeof(int32_t));
+  back(load_before, ctx->st_load_before, R * sizeof(uint32_t));
+  back(load_after, ctx->st_load_after, R * sizeof(uint32_t));
+  back(topk_ids, ctx->st_ids, n_assign * sizeof(int32_t));
+  back(topk_w, ctx->st_w, n_assign * sizeof(float));
+  back(slot_offsets, ctx->st_slot_offsets, (E + 1) * sizeof(uint32_t));
+  back(rank_offsets, ctx->st_rank_offsets, (R + 1) * sizeof(uint32_t));
+  back(perm, ctx->st_perm, n_assign * sizeof(int32_t));
+  back(inv_perm, ctx->st_inv_perm, n_assign * sizeof(int32_t));
+  back(rank_load, ctx->st_rank_load, R * sizeof(uint32_t));
+  if (!ok) return FB_ERR_CUDA;
+  return cudaStreamSynchronize(stream) == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream_) {
+  if (!ctx || !word) return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return FB_ERR_CUDA;
+  if (cudaMemcpy(word, ctx->status, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return FB_ERR_CUDA;
+  if (*word != 0 && cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) return FB_ERR_CUDA;
+  return FB_OK;
+}
+
+uint64_t fb_launch_count(const fb_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the FreeBalance per-layer hot path on B200.
+
+One "step" = the whole hot path for one MoE layer on one prefill batch:
+fb_predict_and_plan on h_{l-1} (early router pass, gating, top-k, histogram, rank
+loads, swap planner - one kernel launch) followed by fb_route_dispatch on H_l under
+the new placement (normal router pass, routing weights, dispatch index - two
+launches).  The metric is tokens per second through that path, per layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload dsv3] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica on its own GPU - the path has no exchange step - and the time is the
+maximum over ranks.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_14205_b200 import inputs as I  # noqa: E402
+
+METRIC = "predicted-routing tokens/sec per layer"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 2**20
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def budget_kwargs(wl: I.Workload, T: int):
+    gn, gd = I.default_gamma(T, wl.k, wl.R)
+    return dict(max_swaps=min(wl.max_swaps, wl.E // 2), global_ns=wl.global_ns, rank_ns=wl.rank_ns,
+                link_ns=wl.link_ns, tau_tokens=0, gamma_num=gn, gamma_den=gd,
+                alpha_ns=(wl.alpha_ns, wl.alpha_ns), fs_per_byte=(wl.fs_per_byte, wl.fs_per_byte),
+                ranks_per_node=wl.ranks_per_node, expert_bytes=wl.expert_bytes)
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _loop(self):
+        nv = self._nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons", None)
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                if get_reasons is not None:
+                    r = int(get_reasons(self._h))
+                    for name, bit in names.items():
+                        if r & bit:
+                            self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self._period)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def oracle_layer_seconds(wl, layer, bkw, steps, warmup):
+    """Time the CPU oracle, as it stands, on whole layers of the workload."""
+    import numpy as np
+    from oracle import freebalance_oracle as O
+    def bits(t): return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    gate = O.Gate(E=wl.E, k=wl.k, gate=wl.gate, n_group=wl.n_group, topk_group=wl.topk_group,
+                  renorm=wl.renorm, route_scale=wl.route_scale)
+    bud = O.Budget(**bkw)
+    args = (bits(layer.h_prev), bits(layer.H), bits(layer.W), gate, wl.R, layer.expert_to_slot.tolist(), bud,
+            None if layer.select_bias is None else layer.select_bias.numpy(),
+            None if layer.logit_bias is None else layer.logit_bias.numpy())
+    for _ in range(warmup):
+        O.layer_step(*args)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        O.layer_step(*args)
+    return (time.perf_counter() - t0) / max(1, steps)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args, wl, rank):
+    if rank != 0:
+        return
+    # one whole layer of the workload per step is a few seconds of CPU work for the
+    # 16k-token shape; longer shapes are cut to 16k tokens to keep the run bounded
+    T_s = min(wl.T, 16384)
+    layer = I.make_layer(wl, 0, 0, T=T_s)
+    bkw = budget_kwargs(wl, T_s)
+    steps = max(1, min(args.steps, 5))
+    warmup = min(args.warmup, 1)
+    sec = oracle_layer_seconds(wl, layer, bkw, steps, warmup)
+    value = T_s / sec
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "T": T_s, "d": wl.d, "E": wl.E, "k": wl.k, "R": wl.R},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{steps} whole layer(s) of {T_s} tokens, full chain"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="dsv3", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ring", type=int, default=2, help="distinct layers cycled through")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    wl = I.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    from paper_2608_14205_b200 import binding as B
+
+    import torch.distributed as dist
+    distributed = world > 1
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if distributed:
+        dist.init_process_group("nccl", device_id=dev)
+
+    T, E, R, k, d = wl.T, wl.E, wl.R, wl.k, wl.d
+    bkw = budget_kwargs(wl, T)
+    budget = B.make_budget(**bkw)
+    ctx = B.Context(T, d, E, k, R, wl.gate, wl.n_group, wl.topk_group, wl.renorm, wl.route_scale, device=local_rank)
+
+    # ---- inputs: a ring of distinct layers, resident in HBM before the timed region
+    ring = max(1, args.ring)
+    layers_cpu = [I.make_layer(wl, layer=l, seed=rank) for l in range(ring)]
+    layers = []
+    for li in layers_cpu:
+        W = li.W.to(dev)
+        sb = li.select_bias.to(dev) if li.select_bias is not None else None
+        layers.append(dict(router=B.make_router(W, None, sb), h_prev=li.h_prev.to(dev), H=li.H.to(dev),
+                           pi=li.expert_to_slot.to(dev)))
+    i32 = lambda n: torch.zeros(max(1, n), dtype=torch.int32, device=dev)
+    out = dict(counts=i32(E), pi_out=i32(E), swaps=i32(4 * max(1, bkw["max_swaps"])), n_swaps=i32(1),
+               load_before=i32(R), load_after=i32(R), ids=i32(T * k), w=torch.zeros(max(1, T * k), device=dev),
+               slot_offsets=i32(E + 1), rank_offsets=i32(R + 1), perm=i32(T * k), inv_perm=i32(T * k),
+               rank_load=i32(R))
+
+    def step(L):
+        ctx.fb_predict_and_plan(L["router"], L["h_prev"], T, L["pi"], budget, 0, out["counts"], out["pi_out"],
+                                out["swaps"], out["n_swaps"], out["load_before"], out["load_after"])
+        ctx.fb_route_dispatch(L["router"], L["H"], T, out["pi_out"], out["ids"], out["w"], out["slot_offsets"],
+                              out["rank_offsets"], out["perm"], out["inv_perm"], out["rank_load"])
+
+    def barrier():
+        if distributed:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for i in range(args.warmup):
+        step(layers[i % ring])
+    barrier()
+    if ctx.fb_device_status() != 0:
+        raise SystemExit("device status non-zero after warm-up")
+
+    # ---- timed region: exactly K steps; events on the launching (current) stream
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    launches0 = ctx.fb_launch_count()
+    barrier()
+    sampler.start()
+    for i in range(K):
+        L = layers[i % ring]
+        ev[i][0].record()
+        ctx.fb_predict_and_plan(L["router"], L["h_prev"], T, L["pi"], budget, 0, out["counts"], out["pi_out"],
+                                out["swaps"], out["n_swaps"], out["load_before"], out["load_after"])
+        ev[i][1].record()
+        ctx.fb_route_dispatch(L["router"], L["H"], T, out["pi_out"], out["ids"], out["w"], out["slot_offsets"],
+                              out["rank_offsets"], out["perm"], out["inv_perm"], out["rank_load"])
+        ev[i][2].record()
+    barrier()
+    clocks = sampler.stop()
+    launches = ctx.fb_launch_count() - launches0
+    total_ms = ev[0][0].elapsed_time(ev[K - 1][2])
+    predict_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
+    dispatch_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(K)]
+    if distributed:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    status = ctx.fb_device_status()
+
+    # ---- end to end through the host-buffer entry point (copies inside the timed region)
+    L0 = layers_cpu[0]
+    pin = lambda t: t.contiguous().pin_memory()
+    h_prev_h, H_h, pi_h = pin(L0.h_prev), pin(L0.H), pin(L0.expert_to_slot)
+    hi32 = lambda n: torch.zeros(max(1, n), dtype=torch.int32).pin_memory()
+    hout = dict(counts=hi32(E), expert_to_slot_out=hi32(E), swaps=hi32(4 * max(1, bkw["max_swaps"])),
+                n_swaps=hi32(1), load_before=hi32(R), load_after=hi32(R), topk_ids=hi32(T * k),
+                topk_w=torch.zeros(max(1, T * k)).pin_memory(), slot_offsets=hi32(E + 1),
+                rank_offsets=hi32(R + 1), perm=hi32(T * k), inv_perm=hi32(T * k), rank_load=hi32(R))
+    h2d = h_prev_h.numel() * 2 + H_h.numel() * 2 + pi_h.numel() * 4
+    d2h = sum(v.numel() * v.element_size() for v in hout.values())
+    e2e_steps = max(3, min(K, 20))
+    for _ in range(2):
+        ctx.fb_layer_step_host(layers[0]["router"], h_prev_h, H_h, T, pi_h, budget, 0, **hout)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        ctx.fb_layer_step_host(layers[0]["router"], h_prev_h, H_h, T, pi_h, budget, 0, **hout)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if distributed:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    if rank == 0:
+        peaks = measured_peaks()
+        ms_per_step = total_ms / K
+        value = world * T * K / (total_ms * 1e-3)
+        # roofline of the dominant kernel (the fused router kernel of fb_predict_and_plan)
+        alg_bytes = 2 * T * d + 2 * d * E + 4 * E
+        alg_flops = 2 * T * d * E
+        k1_ms = statistics.mean(predict_ms)
+        achieved_gbs = alg_bytes / (k1_ms * 1e-3) / 1e9
+        achieved_tf = alg_flops / (k1_ms * 1e-3) / 1e12
+        t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+        t_tensor = alg_flops / (peaks["bf16_tflops"] * 1e12)
+        roof = {"kernel": "fb_router_kernel (fb_predict_and_plan)", "bound": "hbm" if t_hbm >= t_tensor else "tensor",
+                "achieved": achieved_gbs if t_hbm >= t_tensor else achieved_tf,
+                "peak": peaks["hbm_gbs"] if t_hbm >= t_tensor else peaks["bf16_tflops"],
+                "unit": "GB/s" if t_hbm >= t_tensor else "TFLOP/s",
+                "frac": (achieved_gbs / peaks["hbm_gbs"]) if t_hbm >= t_tensor else (achieved_tf / peaks["bf16_tflops"]),
+                "peak_source": peaks["source"], "traffic": None, "kernel_us": k1_ms * 1e3,
+                "kernel_us_median": statistics.median(predict_ms) * 1e3,
+                "t_roof_us": max(t_hbm, t_tensor) * 1e6, "tensor_tflops": achieved_tf,
+                "tensor_frac_of_burst": achieved_tf / peaks["bf16_tflops"],
+                "dispatch_us": statistics.mean(dispatch_ms) * 1e3}
+        traffic_file = os.path.join(ROOT, "profiles", "router_kernel_traffic.json")
+        if os.path.exists(traffic_file):
+            with open(traffic_file) as f:
+                tr = json.load(f)
+            if wl.name in tr:
+                roof["traffic"] = tr[wl.name]
+
+        lb, la = out["load_before"].cpu().tolist(), out["load_after"].cpu().tolist()
+        pi_new = out["pi_out"].cpu().tolist()
+        so = out["slot_offsets"].cpu().tolist()
+        m = E // R
+        realized = [so[pi_new[e] + 1] - so[pi_new[e]] for e in range(E)]
+        pi_old = layers_cpu[(K - 1) % ring].expert_to_slot.tolist()
+        real_before = [0] * R
+        for e in range(E):
+            real_before[pi_old[e] // m] += realized[e]
+        real_after = out["rank_load"].cpu().tolist()
+        mom = lambda L: (max(L) * len(L) / sum(L)) if sum(L) else 1.0
+
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": wl.name, "T": T, "d": d, "E": E, "k": k, "R": R,
+                           "gate": "sigmoid_group_topk" if wl.gate else "softmax_topk",
+                           "layers_in_ring": ring, "parallelism": f"replicas x{world}",
+                           "l2": "each input matrix (%.0f MB) exceeds L2 (126 MB); consecutive launches read different matrices"
+                                 % (T * d * 2 / 1e6) if T * d * 2 > L2_BYTES else
+                                 "ring of layers; inputs may be L2-resident"},
+                "clocks": clocks,
+                "e2e": {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
+                "gpu_launches": int(launches), "device_status": status,
+                "roofline": roof,
+                "load_balance": {"predicted_max_over_mean": [mom(lb), mom(la)],
+                                 "realized_max_over_mean": [mom(real_before), mom(real_after)],
+                                 "n_swaps": int(out["n_swaps"].item())}}
+        if not args.no_cpu_baseline:
+            T_s = min(T, 16384)
+            sample_layer = layers_cpu[0] if T_s == T else I.make_layer(wl, 0, rank, T=T_s)
+            sec = oracle_layer_seconds(wl, sample_layer, budget_kwargs(wl, T_s), 1, 0)
+            line["cpu_baseline"] = {"value": T_s / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                    "sample": f"1 whole layer of {T_s} tokens, full chain, {sec:.2f} s"}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if distributed:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

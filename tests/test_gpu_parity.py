@@ -1,0 +1,288 @@
+"""GPU parity: every entry point of the C-ABI library against the CPU oracle on the
+same seeded inputs (see tests/parity_util.py for the comparison rules)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import freebalance_oracle as O
+from paper_2608_14205_b200 import binding as B
+from paper_2608_14205_b200 import inputs as I
+from tests import parity_util as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(wl, T, layer=0, seed=0, with_logit_bias=False, placement=None, want_logits=True, sample=None, **bud):
+    li = I.make_layer(wl, layer, seed, T=T, with_logit_bias=with_logit_bias)
+    ctx = P.make_context(wl, max(T, 1))
+    bkw = P.budget_kwargs(wl, max(T, 1), **bud)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=want_logits, placement=placement)
+    rep = P.compare_layer(wl, li, bkw, gpu, placement=placement, sample_rows=sample)
+    ctx.close()
+    return rep, gpu
+
+
+# ------------------------------------------------------------------ the paper-shaped configs, reduced T
+@pytest.mark.parametrize("name,T,layer", [
+    ("tiny", 512, 0), ("tiny", 512, 1), ("tiny", 500, 0), ("tiny", 1, 0), ("tiny", 129, 1),
+    ("mixtral", 300, 0), ("mixtral", 1000, 3),
+    ("qwen3", 1000, 0), ("qwen3", 2500, 7),
+    ("dsv3", 777, 0), ("dsv3", 1500, 11),
+    ("sweep32k", 900, 0),
+])
+def test_config_shapes_small(name, T, layer):
+    rep, gpu = _run(I.WORKLOADS[name], T, layer)
+    assert rep["n_swaps"] <= I.WORKLOADS[name].max_swaps
+
+
+def test_mixtral_one_expert_per_rank_never_swaps():
+    rep, gpu = _run(I.WORKLOADS["mixtral"], 640)
+    assert rep["n_swaps"] == 0 and gpu["pi_out"] == list(range(8))
+
+
+def test_dsv3_cost_model_admits_five_swaps():
+    rep, gpu = _run(I.WORKLOADS["dsv3"], 2048)
+    assert rep["n_swaps"] == 5
+    assert rep["pred_max_over_mean_after"] < rep["pred_max_over_mean_before"]
+
+
+def test_empty_batch():
+    wl = I.WORKLOADS["tiny"]
+    rep, gpu = _run(wl, 0)
+    assert gpu["counts"].sum() == 0 and rep["n_swaps"] == 0 and gpu["slot_offsets"].tolist() == [0] * 9
+
+
+# ------------------------------------------------------------------ gating / shape edge cases
+def _wl(**kw):
+    base = dict(name="edge", T=300, d=256, E=16, k=2, R=4, layers=1, max_swaps=4, skew="zipf", zipf_s=1.0)
+    base.update(kw)
+    return I.Workload(**base)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(k=1), dict(E=8, k=8, R=2), dict(E=24, k=3, R=3), dict(E=40, k=4, R=5, d=1000), dict(E=200, k=8, R=8, d=8),
+    dict(d=72), dict(E=256, k=8, R=64, d=512), dict(E=64, k=6, R=8, d=2048),
+    dict(gate=1, n_group=16, topk_group=3, k=3),                  # groups of one expert
+    dict(gate=1, n_group=4, topk_group=2, k=8, E=16),              # k = all eligible experts
+    dict(gate=1, n_group=1, topk_group=1, k=2),                    # one group: plain sigmoid top-k
+    dict(gate=1, n_group=8, topk_group=8, k=5, E=64, R=8),         # every group kept
+    dict(gate=1, n_group=32, topk_group=8, k=8, E=256, R=32, d=512),
+    dict(gate=1, n_group=2, topk_group=1, k=3, E=24, R=4, route_scale=2.5),
+    dict(renorm=0), dict(gate=1, n_group=4, topk_group=2, k=2, renorm=0, route_scale=2.5),
+])
+def test_edge_shapes(kw):
+    _run(_wl(**kw), 300, with_logit_bias=True)
+
+
+def test_select_bias_large_enough_to_change_the_selection():
+    wl = _wl(gate=1, n_group=4, topk_group=2, k=2)
+    li = I.make_layer(wl, 0, 0, T=200)
+    li.select_bias = torch.zeros(wl.E)
+    li.select_bias[13] = 4.0                       # expert 13 now wins everywhere, its group is kept
+    ctx = P.make_context(wl, 200)
+    bkw = P.budget_kwargs(wl, 200)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw)
+    P.compare_layer(wl, li, bkw, gpu)
+    assert (gpu["ids"][:, 0] == 13).all() and gpu["counts"][13] == 200
+    assert (gpu["w"] < 1.0).all()                  # weights use the unbiased score
+
+
+def test_exact_ties_go_to_the_lowest_ids():
+    wl = _wl(E=16, k=3)
+    li = I.make_layer(wl, 0, 0, T=150)
+    li.W = torch.zeros_like(li.W)                  # all logits equal
+    ctx = P.make_context(wl, 150)
+    bkw = P.budget_kwargs(wl, 150)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw)
+    assert (gpu["ids"] == np.array([0, 1, 2])).all()
+    assert gpu["counts"].tolist() == [150, 150, 150] + [0] * 13
+    assert np.allclose(gpu["w"], 1 / 3, atol=1e-6)
+    wl2 = _wl(gate=1, n_group=4, topk_group=2, k=3)
+    li2 = I.make_layer(wl2, 0, 0, T=150)
+    li2.W = torch.zeros_like(li2.W)
+    li2.select_bias = torch.zeros(wl2.E)
+    gpu2 = P.run_gpu_layer(P.make_context(wl2, 150), wl2, li2, P.budget_kwargs(wl2, 150))
+    assert (gpu2["ids"] == np.array([0, 1, 2])).all()
+
+
+# ------------------------------------------------------------------ planner variants through the kernel
+@pytest.mark.parametrize("bud", [
+    dict(tau_tokens=10**6), dict(max_swaps=0), dict(global_ns=0), dict(gamma_num=0, gamma_den=1),
+    dict(gamma_num=3, gamma_den=0),
+    dict(ranks_per_node=2, alpha_ns=(100, 900), fs_per_byte=(2000, 9000), expert_bytes=100_000,
+         global_ns=3000, rank_ns=2500, link_ns=1500, max_swaps=8),
+    dict(alpha_ns=(50, 50), fs_per_byte=(10**6, 10**6), global_ns=900, max_swaps=8,
+         expert_bytes_table=[(7 * e * e + 13) % 400 + 1 for e in range(32)]),
+])
+def test_planner_budget_variants(bud):
+    wl = _wl(E=32, k=4, R=4, max_swaps=8)
+    _run(wl, 400, placement=I.random_placement(32, seed=5), **bud)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_plan_swaps_alone_on_random_counts(seed):
+    rng = np.random.default_rng(seed)
+    R = int(rng.choice([2, 4, 8, 16, 32, 64]))
+    m = int(rng.choice([1, 2, 4, 8, 16]))
+    E = R * m
+    if E > 256:
+        m = 256 // R
+        E = R * m
+    counts = I.random_counts(E, int(rng.integers(0, 200_000)), seed, zipf_s=float(rng.choice([0.5, 1.0, 1.5])))
+    pi = I.random_placement(E, seed)
+    bkw = dict(max_swaps=int(rng.integers(0, E // 2 + 1)), gamma_num=int(rng.choice([0, 1, 5])),
+               gamma_den=int(rng.choice([1, 64, 100_000])), tau_tokens=int(rng.choice([0, 0, 50])),
+               alpha_ns=(int(rng.integers(0, 500)), int(rng.integers(0, 5000))),
+               fs_per_byte=(int(rng.integers(0, 3000)), int(rng.integers(0, 20000))),
+               expert_bytes=int(rng.integers(0, 10**7)), ranks_per_node=int(rng.choice([0, 2, 8])),
+               global_ns=[O.U64_OFF, 10**5, 10**6][int(rng.integers(0, 3))],
+               rank_ns=[O.U64_OFF, 10**5][int(rng.integers(0, 2))],
+               link_ns=[O.U64_OFF, 5 * 10**4][int(rng.integers(0, 2))])
+    ctx = B.Context(128, 64, E, 1, R)
+    dev = torch.device("cuda")
+    ms = max(1, bkw["max_swaps"])
+    out_pi = torch.zeros(E, dtype=torch.int32, device=dev)
+    swaps = torch.zeros(4 * ms, dtype=torch.int32, device=dev)
+    n = torch.zeros(1, dtype=torch.int32, device=dev)
+    lb = torch.zeros(R, dtype=torch.int32, device=dev)
+    la = torch.zeros(R, dtype=torch.int32, device=dev)
+    ctx.fb_plan_swaps(counts.to(torch.int32).to(dev), pi.to(dev), B.make_budget(**bkw), seed, out_pi, swaps, n, lb, la)
+    assert ctx.fb_device_status() == 0
+    want = O.plan_swaps(counts.tolist(), pi.tolist(), R, O.Budget(**bkw), layer_id=seed)
+    got_swaps = [tuple(r) for r in swaps.cpu().numpy().reshape(-1, 4)[:int(n.item())].tolist()]
+    assert (got_swaps, out_pi.cpu().tolist(), lb.cpu().tolist(), la.cpu().tolist()) == want
+
+
+def test_planner_worked_examples_on_gpu(golden):
+    for name in ["planner_two_swaps_one_tie.json", "planner_tie_then_stop.json"]:
+        gd = golden(name)
+        E, R = gd["E"], gd["R"]
+        ctx = B.Context(128, 64, E, 1, R)
+        dev = torch.device("cuda")
+        t = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
+        out_pi, swaps, n, lb, la = t([0] * E), t([0] * 12), t([0]), t([0] * R), t([0] * R)
+        bud = B.make_budget(max_swaps=gd["max_swaps"], gamma_num=gd["gamma_num"], gamma_den=gd["gamma_den"])
+        ctx.fb_plan_swaps(t(gd["counts"]), t(gd["expert_to_slot"]), bud, 0, out_pi, swaps, n, lb, la)
+        assert ctx.fb_device_status() == 0
+        k = int(n.item())
+        assert swaps.cpu().numpy().reshape(-1, 4)[:k].tolist() == gd["swaps"]
+        assert out_pi.cpu().tolist() == gd["expert_to_slot_out"]
+        assert lb.cpu().tolist() == gd["load_before"] and la.cpu().tolist() == gd["load_after"]
+
+
+# ------------------------------------------------------------------ errors and repeatability
+def test_device_detected_errors_and_recovery():
+    wl = I.WORKLOADS["tiny"]
+    li = I.make_layer(wl, 0, 0, T=256)
+    ctx = P.make_context(wl, 256)
+    bkw = P.budget_kwargs(wl, 256)
+    bad = torch.tensor([0, 1, 2, 3, 4, 5, 6, 6], dtype=torch.int32)          # slot 6 twice
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw, placement=bad)
+    assert gpu["status"] == B.FB_ERR_BAD_PLACEMENT
+    assert gpu["swaps"] == [] and gpu["fused"]["swaps"] == []
+    out_of_range = torch.tensor([0, 1, 2, 3, 4, 5, 6, 99], dtype=torch.int32)
+    assert P.run_gpu_layer(ctx, wl, li, bkw, placement=out_of_range)["status"] == B.FB_ERR_BAD_PLACEMENT
+    # the context stays usable and the scratch histogram was left clean
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw)
+    P.compare_layer(wl, li, bkw, gpu)
+    # counts beyond the planner's range
+    dev = torch.device("cuda")
+    big = torch.full((8,), 2**20, dtype=torch.int32, device=dev)
+    z = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
+    ctx.fb_plan_swaps(big, li.expert_to_slot.to(dev), B.make_budget(max_swaps=2), 0, z(8), z(8), z(1), z(4), z(4))
+    assert ctx.fb_device_status() == B.FB_ERR_RANGE
+    assert ctx.fb_device_status() == 0
+
+
+def test_host_detected_errors():
+    wl = I.WORKLOADS["tiny"]
+    ctx = P.make_context(wl, 128)
+    dev = torch.device("cuda")
+    li = I.make_layer(wl, 0, 0, T=256)
+    router = B.make_router(li.W.to(dev))
+    counts = torch.zeros(8, dtype=torch.int32, device=dev)
+    with pytest.raises(B.FbError) as e:
+        ctx.fb_predict_load(router, li.h_prev.to(dev), 256, counts)            # T > T_max
+    assert e.value.status == B.FB_ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(B.FbError) as e:
+        ctx.fb_predict_load(router, None, 64, counts)
+    assert e.value.status == B.FB_ERR_INVALID_ARG
+    with pytest.raises(B.FbError) as e:
+        ctx.fb_predict_load(router, li.h_prev.to(dev), -1, counts)
+    assert e.value.status == B.FB_ERR_INVALID_ARG
+    z = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
+    with pytest.raises(B.FbError) as e:                                        # max_swaps > E/2
+        ctx.fb_plan_swaps(counts, z(8), B.make_budget(max_swaps=5), 0, z(8), z(20), z(1), z(4), z(4))
+    assert e.value.status == B.FB_ERR_INVALID_ARG
+    with pytest.raises(B.FbError) as e:                                        # gamma out of range
+        ctx.fb_plan_swaps(counts, z(8), B.make_budget(max_swaps=1, gamma_num=2**21), 0, z(8), z(4), z(1), z(4), z(4))
+    assert e.value.status == B.FB_ERR_INVALID_ARG
+    with pytest.raises(B.FbError):
+        B.Context(128, 64, 300, 2, 4)
+
+
+def test_repeated_calls_are_bit_identical():
+    wl = I.WORKLOADS["qwen3"]
+    li = I.make_layer(wl, 2, 0, T=1111)
+    ctx = P.make_context(wl, 1111)
+    bkw = P.budget_kwargs(wl, 1111)
+    a = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False)
+    b = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False)
+    for key in ("counts", "ids_early", "ids", "perm", "inv_perm", "slot_offsets", "rank_load"):
+        assert np.array_equal(a[key], b[key]), key
+    assert a["swaps"] == b["swaps"] and a["fused"]["swaps"] == b["fused"]["swaps"]
+    assert np.array_equal(a["w"], b["w"])
+
+
+def test_host_buffer_entry_point_matches_device_entry_points():
+    wl = I.WORKLOADS["qwen3"]
+    T = 700
+    li = I.make_layer(wl, 1, 0, T=T)
+    ctx = P.make_context(wl, T)
+    bkw = P.budget_kwargs(wl, T)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False)
+    dev = torch.device("cuda")
+    router = B.make_router(li.W.to(dev))
+    E, R, k = wl.E, wl.R, wl.k
+    pin = lambda t: t.contiguous().pin_memory()
+    i32 = lambda n: torch.zeros(n, dtype=torch.int32).pin_memory()
+    outs = dict(counts=i32(E), expert_to_slot_out=i32(E), swaps=i32(4 * bkw["max_swaps"]), n_swaps=i32(1),
+                load_before=i32(R), load_after=i32(R), topk_ids=i32(T * k),
+                topk_w=torch.zeros(T * k).pin_memory(), slot_offsets=i32(E + 1), rank_offsets=i32(R + 1),
+                perm=i32(T * k), inv_perm=i32(T * k), rank_load=i32(R))
+    ctx.fb_layer_step_host(router, pin(li.h_prev), pin(li.H), T, pin(li.expert_to_slot), B.make_budget(**bkw), 0,
+                           **outs)
+    assert ctx.fb_device_status() == 0
+    assert outs["counts"].tolist() == gpu["counts"].tolist()
+    n = int(outs["n_swaps"].item())
+    assert [tuple(r) for r in outs["swaps"].numpy().reshape(-1, 4)[:n].tolist()] == gpu["swaps"]
+    assert outs["expert_to_slot_out"].tolist() == gpu["pi_out"]
+    assert np.array_equal(outs["topk_ids"].numpy().reshape(T, k), gpu["ids"])
+    assert np.array_equal(outs["perm"].numpy(), gpu["perm"]) and np.array_equal(outs["inv_perm"].numpy(), gpu["inv_perm"])
+    assert outs["rank_load"].tolist() == gpu["rank_load"].tolist()
+    assert np.allclose(outs["topk_w"].numpy().reshape(T, k), gpu["w"], atol=0, rtol=0)
+
+
+# ------------------------------------------------------------------ full size, the benchmark's launch configuration
+def test_dsv3_full_size_every_output():
+    wl = I.WORKLOADS["dsv3"]
+    rep, gpu = _run(wl, wl.T, layer=0, want_logits=False)
+    assert rep["n_swaps"] == 5
+    assert rep["real_max_over_mean_after"] < rep["real_max_over_mean_before"]
+
+
+@pytest.mark.parametrize("name", ["sweep32k", "sweep64k"])
+def test_long_prefill_sweep_sampled(name):
+    wl = I.WORKLOADS[name]
+    rows = np.random.default_rng(0).choice(wl.T, size=2048, replace=False)
+    rows.sort()
+    rep, gpu = _run(wl, wl.T, layer=0, want_logits=False, sample=rows)
+    assert rep["n_swaps"] <= wl.max_swaps
+
+
+@pytest.mark.parametrize("name", ["mixtral", "qwen3"])
+def test_mid_configs_full_size(name):
+    wl = I.WORKLOADS[name]
+    _run(wl, wl.T, layer=0, want_logits=False)

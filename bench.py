@@ -178,6 +178,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ring", type=int, default=2, help="distinct layers cycled through")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -277,8 +278,8 @@ def main():
                 rank_offsets=hi32(R + 1), perm=hi32(T * k), inv_perm=hi32(T * k), rank_load=hi32(R))
     h2d = h_prev_h.numel() * 2 + H_h.numel() * 2 + pi_h.numel() * 4
     d2h = sum(v.numel() * v.element_size() for v in hout.values())
-    e2e_steps = max(3, min(K, 20))
-    for _ in range(2):
+    e2e_steps = 0 if args.no_e2e else max(3, min(K, 20))
+    for _ in range(0 if args.no_e2e else 2):
         ctx.fb_layer_step_host(layers[0]["router"], h_prev_h, H_h, T, pi_h, budget, 0, **hout)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -287,7 +288,7 @@ def main():
         ctx.fb_layer_step_host(layers[0]["router"], h_prev_h, H_h, T, pi_h, budget, 0, **hout)
     e1.record()
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
+    e2e_ms = max(e0.elapsed_time(e1), 1e-9)
     if distributed:
         t = torch.tensor([e2e_ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -344,7 +345,8 @@ def main():
                                  % (T * d * 2 / 1e6) if T * d * 2 > L2_BYTES else
                                  "ring of layers; inputs may be L2-resident"},
                 "clocks": clocks,
-                "e2e": {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "e2e": None if args.no_e2e else
+                       {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
                 "gpu_launches": int(launches), "device_status": status,
                 "roofline": roof,

@@ -255,7 +255,10 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   if (stages > fb::kMaxStages) stages = fb::kMaxStages;
   if (stages < 2) { delete ctx; return FB_ERR_UNSUPPORTED_SHAPE; }
   ctx->stages = stages;
-  ctx->smem_bytes = stages * stage_bytes + 1024;
+  size_t dyn = stages * stage_bytes;
+  if (dyn < fb::epilogue_scratch_bytes(ctx->N)) dyn = fb::epilogue_scratch_bytes(ctx->N);
+  if (dyn + 1024 > budget) { delete ctx; return FB_ERR_UNSUPPORTED_SHAPE; }
+  ctx->smem_bytes = dyn + 1024;
   ctx->max_tiles = (cfg->T_max + fb::kTileM - 1) / fb::kTileM;
 
   void* fn = nullptr;

@@ -1,7 +1,7 @@
-// Budgeted greedy expert-swap planner (Algorithm 1 lines 2-8, Eqs. 6-9) for one
-// group of kPlanThreads threads: either a stand-alone one-block kernel or the tail of
-// the router kernel, run by the block that finished last.  Integer arithmetic only, so
-// every rank that replays it on the same count vector gets the same plan.
+// Budgeted greedy expert-swap planner (Algorithm 1 lines 2-8, Eqs. 6-9), run by one
+// warp: either a stand-alone one-warp kernel or the tail of the router kernel, in the
+// block that finished last.  Integer arithmetic only, so every rank that replays it on
+// the same count vector gets the same plan.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -11,8 +11,8 @@
 
 namespace fb {
 
-constexpr int kPlanThreads = 128;
-constexpr uint32_t kPlanBarrierId = 1;
+constexpr int kPlanThreads = 32;          // the stand-alone planner kernel is one warp
+constexpr uint32_t kPlanBarrierId = 1;    // named barrier of the router kernel's epilogue warps
 
 struct PlanParams {
   int32_t E, R;
@@ -48,7 +48,6 @@ struct PlanShared {
   unsigned long long rank_spent[FB_MAX_RANKS];
   uint32_t link_key[FB_MAX_EXPERTS / 2]; // one entry per accepted swap
   unsigned long long link_cost[FB_MAX_EXPERTS / 2];
-  PlanCandidate warp_best[kPlanThreads / 32];
   int32_t bad;
 };
 
@@ -74,76 +73,100 @@ __device__ __forceinline__ unsigned long long plan_cost_ns(const PlanParams& p, 
   return c < 1 ? 1 : c;
 }
 
-// Called by exactly kPlanThreads threads with t = 0..kPlanThreads-1; sh.cnt must hold
-// the count vector.  Synchronises with the named barrier kPlanBarrierId.
-__device__ __noinline__ void plan_swaps_block(const PlanParams& p, PlanShared& sh, int t, int* status) {
-  const int E = p.E, R = p.R, m = E / R;
-  // ---- placement: load, invert, check that it is a bijection
-  if (t == 0) sh.bad = 0;
-  for (int e = t; e < E; e += kPlanThreads) { sh.expert_at[e] = -1; sh.moved[e] = 0; }
-  for (int r = t; r < R; r += kPlanThreads) sh.rank_spent[r] = 0;
-  named_bar_sync(kPlanBarrierId, kPlanThreads);
-  for (int e = t; e < E; e += kPlanThreads) {
+// Load the placement into shared memory, invert it and check that it is a bijection.
+// Called by `nthreads` threads (t = 0..nthreads-1); the caller synchronises afterwards.
+// sh.bad must have been cleared and sh.expert_at filled with -1 beforehand.
+__device__ __forceinline__ void plan_load_placement(const PlanParams& p, PlanShared& sh, int t, int nthreads) {
+  for (int e = t; e < p.E; e += nthreads) {
     const int s = p.expert_to_slot[e];
     sh.slot_of[e] = s;
-    if (s < 0 || s >= E) sh.bad = 1;
+    sh.moved[e] = 0;
+    if (s < 0 || s >= p.E) sh.bad = 1;
     else if (atomicExch(&sh.expert_at[s], e) != -1) sh.bad = 1;
   }
-  named_bar_sync(kPlanBarrierId, kPlanThreads);
+}
+__device__ __forceinline__ void plan_clear(PlanShared& sh, int t, int nthreads) {
+  if (t == 0) sh.bad = 0;
+  for (int e = t; e < FB_MAX_EXPERTS; e += nthreads) sh.expert_at[e] = -1;
+}
+
+// The greedy loop, run by ONE warp (all 32 lanes) once sh.cnt holds the count vector and
+// plan_load_placement has filled the placement arrays.  A single warp keeps the rank
+// loads in registers (lane r holds ranks r and r + 32) and needs no block barrier: every
+// step is a handful of shuffles.
+__device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh, int lane, int* status) {
+  const int E = p.E, R = p.R, m = E / R;
+  const uint32_t full = 0xffffffffu;
+  __syncwarp();
   unsigned long long total = 0;
-  if (t == 0) {
-    for (int e = 0; e < E; ++e) total += sh.cnt[e];
-    if (total > FB_MAX_COUNT_SUM) sh.bad = 2;
-  }
-  named_bar_sync(kPlanBarrierId, kPlanThreads);
-  if (sh.bad) {
+  for (int e = lane; e < E; e += 32) total += sh.cnt[e];
+  for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(full, total, off);
+  int bad = sh.bad;
+  if (!bad && total > FB_MAX_COUNT_SUM) bad = 2;
+  if (bad) {
     // Unusable input: report it, keep the placement as given, empty plan.
-    if (t == 0) {
-      atomicCAS(status, 0, sh.bad == 1 ? FB_ERR_BAD_PLACEMENT : FB_ERR_RANGE);
+    if (lane == 0) {
+      atomicCAS(status, 0, bad == 1 ? FB_ERR_BAD_PLACEMENT : FB_ERR_RANGE);
       *p.n_swaps = 0;
     }
-    for (int e = t; e < E; e += kPlanThreads) p.expert_to_slot_out[e] = p.expert_to_slot[e];
-    for (int r = t; r < R; r += kPlanThreads) { p.load_before[r] = 0; p.load_after[r] = 0; }
+    for (int e = lane; e < E; e += 32) p.expert_to_slot_out[e] = p.expert_to_slot[e];
+    for (int r = lane; r < R; r += 32) { p.load_before[r] = 0; p.load_after[r] = 0; }
     return;
   }
-  // ---- rank loads (Algorithm 1 line 2)
-  for (int r = t; r < R; r += kPlanThreads) {
-    uint32_t s = 0;
-    for (int j = 0; j < m; ++j) s += sh.cnt[sh.expert_at[r * m + j]];
-    sh.load[r] = s;
-    p.load_before[r] = s;
+  // ---- rank loads (Algorithm 1 line 2): lane holds L[lane] and L[lane + 32]
+  long long L0 = -1, L1 = -1;                  // -1 marks "no such rank"
+  if (lane < R) {
+    uint32_t s0 = 0;
+    for (int j = 0; j < m; ++j) s0 += sh.cnt[sh.expert_at[lane * m + j]];
+    L0 = s0;
+    p.load_before[lane] = s0;
   }
-  named_bar_sync(kPlanBarrierId, kPlanThreads);
+  if (lane + 32 < R) {
+    uint32_t s1 = 0;
+    for (int j = 0; j < m; ++j) s1 += sh.cnt[sh.expert_at[(lane + 32) * m + j]];
+    L1 = s1;
+    p.load_before[lane + 32] = s1;
+  }
+  if (lane == 0) { for (int r = 0; r < R; ++r) sh.rank_spent[r] = 0; }
+  __syncwarp();
 
   const long long gnum = p.gamma_den ? p.gamma_num : 0;
   const long long gden = p.gamma_den ? p.gamma_den : 1;
+  const int rpn = p.ranks_per_node;
   unsigned long long global_spent = 0;
   uint32_t n = 0;
   while (n < p.max_swaps) {
-    // frontier: most and least loaded rank, lowest index on ties (every thread computes it)
-    int a = 0, b = 0;
-    for (int r = 1; r < R; ++r) {
-      if (sh.load[r] > sh.load[a]) a = r;
-      if (sh.load[r] < sh.load[b]) b = r;
-    }
-    const long long La = sh.load[a], Lb = sh.load[b];
+    // frontier: most and least loaded rank, lowest index on ties.  Loads are below 2^22
+    // (checked above), so (load, rank) packs into 32 bits and one warp reduction finds
+    // each extreme: max of load<<6 | (63 - rank), min of load<<6 | rank.
+    const uint32_t none_hi = 0u, none_lo = 0xffffffffu;
+    const uint32_t h0 = L0 >= 0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(63 - lane)) : none_hi;
+    const uint32_t h1 = L1 >= 0 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(31 - lane)) : none_hi;
+    const uint32_t l0 = L0 >= 0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(lane)) : none_lo;
+    const uint32_t l1 = L1 >= 0 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(lane + 32)) : none_lo;
+    const uint32_t hi_key = __reduce_max_sync(full, h0 > h1 ? h0 : h1);
+    const uint32_t lo_key = __reduce_min_sync(full, l0 < l1 ? l0 : l1);
+    const int a = 63 - static_cast<int>(hi_key & 63u), b = static_cast<int>(lo_key & 63u);
+    const long long La = hi_key >> 6, Lb = lo_key >> 6;
     if (La - Lb <= static_cast<long long>(p.tau_tokens)) break;
-    long long M2 = 0;
-    for (int r = 0; r < R; ++r)
-      if (r != a && r != b && static_cast<long long>(sh.load[r]) > M2) M2 = sh.load[r];
-    const int rpn = p.ranks_per_node;
+    uint32_t m2 = 0;                               // largest load among the other ranks
+    if (lane != a && lane != b && L0 > 0) m2 = static_cast<uint32_t>(L0);
+    if (lane + 32 != a && lane + 32 != b && L1 > static_cast<long long>(m2)) m2 = static_cast<uint32_t>(L1);
+    const long long M2 = __reduce_max_sync(full, m2);
     const int cls = (rpn <= 0 || a / rpn == b / rpn) ? 0 : 1;
     const int lo = a < b ? a : b, hi = a < b ? b : a;
     const uint32_t lkey = cls == 0 ? (static_cast<uint32_t>(lo) << 8 | static_cast<uint32_t>(hi))
                                    : (0x10000u | static_cast<uint32_t>(lo / rpn) << 8 | static_cast<uint32_t>(hi / rpn));
     unsigned long long link_spent = 0;
-    for (uint32_t i = 0; i < n; ++i)
-      if (sh.link_key[i] == lkey) link_spent += sh.link_cost[i];
-    const unsigned long long rank_spent = sh.rank_spent[a] > sh.rank_spent[b] ? sh.rank_spent[a] : sh.rank_spent[b];
+    if (p.link_ns != FB_BUDGET_OFF)
+      for (uint32_t i = 0; i < n; ++i)
+        if (sh.link_key[i] == lkey) link_spent += sh.link_cost[i];
+    const unsigned long long rs_a = sh.rank_spent[a], rs_b = sh.rank_spent[b];
+    const unsigned long long rank_spent = rs_a > rs_b ? rs_a : rs_b;
 
     PlanCandidate best;
     best.benefit = 0; best.cost = 1; best.ea = -1; best.eb = -1;
-    for (int c = t; c < m * m; c += kPlanThreads) {
+    for (int c = lane; c < m * m; c += 32) {
       const int ea = sh.expert_at[a * m + c / m];
       const int eb = sh.expert_at[b * m + c % m];
       if (sh.moved[ea] || sh.moved[eb]) continue;
@@ -164,42 +187,60 @@ __device__ __noinline__ void plan_swaps_block(const PlanParams& p, PlanShared& s
       if (p.link_ns != FB_BUDGET_OFF && (cand.cost > p.link_ns || link_spent > p.link_ns - cand.cost)) continue;
       if (plan_better(cand, best)) best = cand;
     }
-    // block arg-max
-    for (int off = 16; off > 0; off >>= 1) {
-      PlanCandidate o;
-      o.benefit = __shfl_xor_sync(0xffffffffu, best.benefit, off);
-      o.cost = __shfl_xor_sync(0xffffffffu, best.cost, off);
-      o.ea = __shfl_xor_sync(0xffffffffu, best.ea, off);
-      o.eb = __shfl_xor_sync(0xffffffffu, best.eb, off);
-      if (plan_better(o, best)) best = o;
+    if (p.expert_bytes_table == nullptr) {
+      // every candidate of this iteration has the same cost: the largest benefit wins,
+      // ties go to the smallest (ea, eb).  Three 32-bit warp reductions.
+      const unsigned long long ben = best.ea >= 0 ? static_cast<unsigned long long>(best.benefit) : 0ull;
+      const uint32_t top_hi = __reduce_max_sync(full, static_cast<uint32_t>(ben >> 32));
+      const uint32_t lo_part = static_cast<uint32_t>(ben >> 32) == top_hi ? static_cast<uint32_t>(ben) : 0u;
+      const uint32_t top_lo = __reduce_max_sync(full, lo_part);
+      const unsigned long long top_ben = static_cast<unsigned long long>(top_hi) << 32 | top_lo;
+      const uint32_t pair = (best.ea >= 0 && ben == top_ben)
+                                ? (static_cast<uint32_t>(best.ea) << 16 | static_cast<uint32_t>(best.eb)) : 0xffffffffu;
+      const uint32_t win = __reduce_min_sync(full, pair);
+      if (top_ben == 0 || win == 0xffffffffu) { best.ea = -1; }
+      else {
+        best.benefit = static_cast<long long>(top_ben);
+        best.cost = p.uniform_cost_ns[cls];
+        best.ea = static_cast<int32_t>(win >> 16);
+        best.eb = static_cast<int32_t>(win & 0xffffu);
+      }
+    } else {
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        PlanCandidate o;
+        o.benefit = __shfl_xor_sync(full, best.benefit, off);
+        o.cost = __shfl_xor_sync(full, best.cost, off);
+        o.ea = __shfl_xor_sync(full, best.ea, off);
+        o.eb = __shfl_xor_sync(full, best.eb, off);
+        if (plan_better(o, best)) best = o;
+      }
     }
-    if ((t & 31) == 0) sh.warp_best[t >> 5] = best;
-    named_bar_sync(kPlanBarrierId, kPlanThreads);
-    best = sh.warp_best[0];
-    for (int w = 1; w < kPlanThreads / 32; ++w)
-      if (plan_better(sh.warp_best[w], best)) best = sh.warp_best[w];
     if (best.ea < 0) break;                                     // Algorithm 1 lines 6-7
-    named_bar_sync(kPlanBarrierId, kPlanThreads);               // everyone has read warp_best / load
-    if (t == 0) {
-      const long long dlt = static_cast<long long>(sh.cnt[best.ea]) - static_cast<long long>(sh.cnt[best.eb]);
-      sh.load[a] = static_cast<uint32_t>(La - dlt);
-      sh.load[b] = static_cast<uint32_t>(Lb + dlt);
+    const long long dlt = static_cast<long long>(sh.cnt[best.ea]) - static_cast<long long>(sh.cnt[best.eb]);
+    __syncwarp();                                               // all lanes are done reading the tables
+    if (lane == 0) {
       const int sa = sh.slot_of[best.ea], sb = sh.slot_of[best.eb];
       sh.slot_of[best.ea] = sb; sh.slot_of[best.eb] = sa;
       sh.expert_at[sa] = best.eb; sh.expert_at[sb] = best.ea;
       sh.moved[best.ea] = 1; sh.moved[best.eb] = 1;
-      sh.rank_spent[a] += best.cost; sh.rank_spent[b] += best.cost;
+      sh.rank_spent[a] = rs_a + best.cost; sh.rank_spent[b] = rs_b + best.cost;
       sh.link_key[n] = lkey; sh.link_cost[n] = best.cost;
       fb_swap s; s.src_rank = a; s.dst_rank = b; s.expert_src = best.ea; s.expert_dst = best.eb;
       p.swaps[n] = s;
     }
+    if (lane == a) L0 -= dlt;
+    if (lane + 32 == a) L1 -= dlt;
+    if (lane == b) L0 += dlt;
+    if (lane + 32 == b) L1 += dlt;
     global_spent += best.cost;
     ++n;
-    named_bar_sync(kPlanBarrierId, kPlanThreads);
+    __syncwarp();
   }
-  if (t == 0) *p.n_swaps = static_cast<int32_t>(n);
-  for (int e = t; e < E; e += kPlanThreads) p.expert_to_slot_out[e] = sh.slot_of[e];
-  for (int r = t; r < R; r += kPlanThreads) p.load_after[r] = sh.load[r];
+  if (lane == 0) *p.n_swaps = static_cast<int32_t>(n);
+  for (int e = lane; e < E; e += 32) p.expert_to_slot_out[e] = sh.slot_of[e];
+  if (lane < R) p.load_after[lane] = static_cast<uint32_t>(L0);
+  if (lane + 32 < R) p.load_after[lane + 32] = static_cast<uint32_t>(L1);
 }
 
 }  // namespace fb

@@ -5,7 +5,20 @@
 //
 // One block owns 128 token rows and all N = pad16(E) expert columns.
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the TMEM allocation),
-// warps 2..5 = epilogue, one thread per token row.
+// warps 2..17 = epilogue.  A warp may only read the 32 TMEM lanes (token rows) selected
+// by warp_id % 4, so the 16 epilogue warps form 4 "row quarters" x 4 "subs"; the subs of
+// a quarter split the expert columns between them in 32-column chunks, one thread per
+// token row, and sub 0 merges the partial results.
+//
+// Epilogue outline (after the accumulator is complete the pipeline's shared memory is
+// idle and is reused as scratch):
+//   pass 1  TMEM -> registers, 32 independent columns at a time: logit (+bias), selection
+//           key (logit, or sigmoid + bias); keys are parked in shared memory; the sigmoid
+//           gate also records each group's score (sum of its two largest keys).
+//   choose  every thread picks its row's best groups and a lower bound for the k-th key.
+//   pass 2  keys are re-read from shared memory; per chunk the few that can still enter
+//           the top-k are compacted, then inserted (one insertion routine, rolled loops:
+//           the code stays small enough for the instruction cache).
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -20,8 +33,9 @@ constexpr int kTileM = 128;            // token rows per block
 constexpr int kBlockK = 64;            // bf16 elements per k-block = one 128-byte swizzled row
 constexpr int kUmmaK = 16;             // K of one tcgen05.mma for 16-bit inputs
 constexpr int kMaxStages = 8;
-constexpr int kRouterThreads = 192;
-constexpr int kEpilogueThreads = 128;
+constexpr int kEpiSubs = 4;            // epilogue warps per row quarter
+constexpr int kEpilogueThreads = 128 * kEpiSubs;
+constexpr int kRouterThreads = 64 + kEpilogueThreads;
 constexpr int kATileBytes = kTileM * kBlockK * 2;
 
 enum RouterMode : int {
@@ -72,11 +86,40 @@ struct TopK {
       if (x > v[0]) { v[0] = x; i[0] = id; }
     }
   }
+  // Same list, candidates in any order: equal keys are ordered by ascending id.
+  __device__ __forceinline__ void insert_any_order(float x, int32_t id) {
+    const bool enters = x > v[FB_MAX_TOPK - 1] || (x == v[FB_MAX_TOPK - 1] && id < i[FB_MAX_TOPK - 1]);
+    if (enters) {
+#pragma unroll
+      for (int j = FB_MAX_TOPK - 1; j > 0; --j) {
+        const bool above_prev = x > v[j - 1] || (x == v[j - 1] && id < i[j - 1]);
+        const bool above_cur = x > v[j] || (x == v[j] && id < i[j]);
+        v[j] = above_prev ? v[j - 1] : (above_cur ? x : v[j]);
+        i[j] = above_prev ? i[j - 1] : (above_cur ? id : i[j]);
+      }
+      if (x > v[0] || (x == v[0] && id < i[0])) { v[0] = x; i[0] = id; }
+    }
+  }
 };
 
+// 1 / (1 + 2^(-z log2 e)) with the two hardware approximations (relative error ~1e-7).
+// 2^x overflows to +inf for z < -88 and the reciprocal of +inf is 0, as it should be.
 __device__ __forceinline__ float fb_sigmoid(float z) {
-  return __fdividef(1.0f, 1.0f + __expf(-z));
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * -1.4426950408889634f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return r;
 }
+
+// Shared-memory scratch of the epilogue (it reuses the pipeline stages): keys [N][128],
+// group scores and group lower bounds [32][128] each, partial top-k lists of subs 1..,
+// partial softmax sums.
+constexpr int kCandCap = 32;           // candidates per row the fast selection path can hold
+__host__ __device__ constexpr size_t epilogue_scratch_bytes(int N) {
+  return (static_cast<size_t>(N) * kTileM + 2 * FB_MAX_GROUPS * kTileM + 2 * kCandCap * kTileM) * 4;
+}
+
+static_assert(2 * kCandCap >= 2 * (kEpiSubs - 1) * FB_MAX_TOPK + kEpiSubs * 2, "merge area must fit in the candidate area");
 
 struct RouterShared {
   uint64_t full_bar[kMaxStages];
@@ -85,9 +128,10 @@ struct RouterShared {
   uint32_t tmem_base;
   int32_t abort_flag;
   int32_t is_last;
-  float logit_bias[FB_MAX_EXPERTS];
-  float select_bias[FB_MAX_EXPERTS];
+  float logit_bias[FB_MAX_EXPERTS + 32];     // + 32: a partial last chunk is read in full
+  float select_bias[FB_MAX_EXPERTS + 32];
   uint32_t hist[FB_MAX_EXPERTS];
+  uint32_t cand_count[kTileM];               // fast selection path: candidates claimed per row
   PlanShared plan;
 };
 
@@ -130,11 +174,13 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   }
   if (warp >= 2) {
     const int et = threadIdx.x - 64;
-    for (int e = et; e < FB_MAX_EXPERTS; e += kEpilogueThreads) {
-      sh.hist[e] = 0;
+    for (int e = et; e < FB_MAX_EXPERTS + 32; e += kEpilogueThreads) {
+      if (e < FB_MAX_EXPERTS) sh.hist[e] = 0;
+      if (e < kTileM) sh.cand_count[e] = 0;
       sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
       sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
     }
+    if (p.mode == kModePredictPlan) plan_clear(sh.plan, et, kEpilogueThreads);
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -181,88 +227,369 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       umma_commit_1cta(smem_u32(&sh.accum_bar));          // accumulator complete
     }
   } else {
-    // ------------------------------------------------------------ epilogue: one thread per row
-    const int et = threadIdx.x - 64;                       // 0..127
+    // ------------------------------------------------------------ epilogue
+    const int et = threadIdx.x - 64;                       // 0 .. kEpilogueThreads-1
     const int quarter = warp & 3;                          // TMEM lanes this warp may touch
+    const int sub = (warp - 2) >> 2;                       // which share of the columns
     const int row_in_tile = quarter * 32 + lane;
     const long long row = static_cast<long long>(tile) * kTileM + row_in_tile;
     const bool valid = row < p.T;
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     const int E = p.E, N = p.N, k = p.k;
+    const bool sigmoid_gate = p.gate != FB_GATE_SOFTMAX_TOPK;
+    const int gs = sigmoid_gate ? E / p.n_group : E;       // experts per group
+    // Which sub owns chunk c: whole groups must stay with one sub.
+    const int n_chunks = (N + 31) >> 5;
+    const int chunks_per_group = (sigmoid_gate && gs % 32 == 0) ? gs / 32 : 1;
+    const bool splittable = !sigmoid_gate || gs % 32 == 0 || 32 % gs == 0;
+    // DeepSeek-V3-like gate (groups of exactly one chunk, few groups kept): selection by
+    // ranking a short candidate list instead of insertion.
+    const bool fast_select = sigmoid_gate && gs == 32 && p.n_group <= 8 && p.topk_group <= kEpiSubs &&
+                             p.topk_group * 2 >= k;
 
+    // While the main loop runs, stage the placement for the planner (any block may turn
+    // out to be the last one).
+    if (p.mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
     const bool got = mbar_wait(smem_u32(&sh.accum_bar), 0u, abort_flag);
     tcgen05_fence_after();
+
+    // scratch carved out of the (now idle) pipeline stages
+    float* key_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // [N][128]
+    float* gscore_s = key_s + static_cast<size_t>(N) * kTileM;                               // [32][128]
+    float* glow_s = gscore_s + FB_MAX_GROUPS * kTileM;                                       // [32][128]
+    float* merge_v = glow_s + FB_MAX_GROUPS * kTileM;                                        // [subs-1][8][128]
+    int32_t* merge_i = reinterpret_cast<int32_t*>(merge_v + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);
+    float* part_s = reinterpret_cast<float*>(merge_i + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);   // [subs][2][128]
+
     TopK top;
     top.init();
-    float sm_max = -INFINITY, sm_sum = 0.0f;               // online softmax (weights without renorm)
+    float sm_max = -INFINITY, sm_sum = 0.0f;               // softmax denominator (weights without renorm)
+    const bool has_lb = p.logit_bias != nullptr;
+    const bool want_sum = p.topk_w != nullptr && !p.renorm && !sigmoid_gate;
     if (got) {
-      uint32_t r[32];
-      if (p.gate == FB_GATE_SOFTMAX_TOPK) {
-        for (int c0 = 0; c0 < N; c0 += 32) {
-          load_chunk(taddr, c0, N, r);
+      // ---------------- pass 1
+      float m1 = -INFINITY, m2 = -INFINITY;
+      for (int c = 0; c < n_chunks; ++c) {
+        const int owner = splittable ? (c / chunks_per_group) % kEpiSubs : 0;
+        if (owner != sub) continue;
+        const int c0 = c * 32;
+        uint32_t r[32];
+        float q[32];
+        load_chunk(taddr, c0, N, r);
+        if (p.logits != nullptr && valid) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < E)
+              p.logits[row * E + c0 + j] = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
+        }
+        if (sigmoid_gate) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const int e = c0 + j;
-            if (e < E) {
-              const float z = __uint_as_float(r[j]) + sh.logit_bias[e];
-              if (p.logits != nullptr && valid) p.logits[row * E + e] = z;
-              if (z > sm_max) { sm_sum = sm_sum * __expf(sm_max - z) + 1.0f; sm_max = z; }
-              else sm_sum += __expf(z - sm_max);
-              top.insert(z, e);
-            }
+            const float z = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
+            q[j] = (c0 + j < E) ? fb_sigmoid(z) + sh.select_bias[c0 + j] : -INFINITY;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float z = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
+            q[j] = (c0 + j < E) ? z : -INFINITY;
           }
         }
-      } else {
-        // pass 1: score every group by the sum of its two largest keys, keep the best groups
-        const int gs = E / p.n_group;
-        TopK gtop;                                           // FB_MAX_TOPK >= topk_group
-        gtop.init();
-        int pos = 0, g = 0;
-        float m1 = -INFINITY, m2 = -INFINITY;
-        for (int c0 = 0; c0 < N; c0 += 32) {
-          load_chunk(taddr, c0, N, r);
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (c0 + j < N) key_s[(c0 + j) * kTileM + row_in_tile] = q[j];
+        if (want_sum) {
+          float cmax = q[0];
+#pragma unroll
+          for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, q[j]);
+          const float nmax = fmaxf(sm_max, cmax);
+          float part = 0.0f;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) part += __expf(q[j] - nmax);     // exp(-inf) = 0 for padding
+          sm_sum = sm_sum * __expf(sm_max - nmax) + part;
+          sm_max = nmax;
+        }
+        if (sigmoid_gate && gs % 32 == 0) {
+          // the chunk lies inside one group: branch-free top-2 of its 32 keys by a merge tree
+          float a1[16], a2[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) { a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); }
+#pragma unroll
+          for (int w = 8; w >= 1; w >>= 1) {
+#pragma unroll
+            for (int j = 0; j < w; ++j) {
+              const float hi = fmaxf(a1[j], a1[j + w]);
+              a2[j] = fmaxf(fminf(a1[j], a1[j + w]), fmaxf(a2[j], a2[j + w]));
+              a1[j] = hi;
+            }
+          }
+          m2 = fmaxf(fminf(m1, a1[0]), fmaxf(m2, a2[0]));
+          m1 = fmaxf(m1, a1[0]);
+          if ((c0 + 32) % gs == 0) {                          // last chunk of the group
+            const int g = c0 / gs;
+            gscore_s[g * kTileM + row_in_tile] = m1 + m2;
+            glow_s[g * kTileM + row_in_tile] = m2;
+            m1 = -INFINITY; m2 = -INFINITY;
+          }
+        } else if (sigmoid_gate) {
+          int g = c0 / gs, pos = c0 % gs;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const int e = c0 + j;
-            if (e < E) {
-              const float z = __uint_as_float(r[j]) + sh.logit_bias[e];
-              if (p.logits != nullptr && valid) p.logits[row * E + e] = z;
-              const float q = fb_sigmoid(z) + sh.select_bias[e];
-              if (q > m1) { m2 = m1; m1 = q; }
-              else if (q > m2) m2 = q;
-              if (++pos == gs) {
-                gtop.insert(gs >= 2 ? m1 + m2 : m1, g);
+            if (c0 + j < E) {
+              m2 = fmaxf(m2, fminf(m1, q[j]));
+              m1 = fmaxf(m1, q[j]);
+              if (++pos == gs) {                              // group complete (uniform branch)
+                gscore_s[g * kTileM + row_in_tile] = gs >= 2 ? m1 + m2 : m1;
+                glow_s[g * kTileM + row_in_tile] = gs >= 2 ? m2 : m1;
                 ++g; pos = 0; m1 = -INFINITY; m2 = -INFINITY;
               }
-            }
-          }
-        }
-        uint32_t keep = 0;
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j < p.topk_group) keep |= 1u << gtop.i[j];
-        // pass 2: top-k among the experts of the kept groups
-        pos = 0; g = 0;
-        for (int c0 = 0; c0 < N; c0 += 32) {
-          load_chunk(taddr, c0, N, r);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int e = c0 + j;
-            if (e < E) {
-              if ((keep >> g) & 1u) {
-                const float z = __uint_as_float(r[j]) + sh.logit_bias[e];
-                top.insert(fb_sigmoid(z) + sh.select_bias[e], e);
-              }
-              if (++pos == gs) { ++g; pos = 0; }
             }
           }
         }
       }
     }
     tcgen05_fence_before();
+    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    if (got && fast_select) {
+      // ---------------- choose: rank the (at most 8) group scores of this row
+      uint32_t* cand_hi = reinterpret_cast<uint32_t*>(merge_v);             // [kCandCap][128] ordered key bits
+      uint32_t* cand_lo = cand_hi + kCandCap * kTileM;                       // [kCandCap][128] ~expert id
+      float sc[8];
+#pragma unroll
+      for (int g = 0; g < 8; ++g) sc[g] = g < p.n_group ? gscore_s[g * kTileM + row_in_tile] : -INFINITY;
+      int my_group = -1;
+      float floor_key = INFINITY;
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        int rank = 0;
+#pragma unroll
+        for (int h = 0; h < 8; ++h)
+          if (h != g) rank += (sc[h] > sc[g] || (sc[h] == sc[g] && h < g)) ? 1 : 0;
+        if (g < p.n_group && rank < p.topk_group) {
+          floor_key = fminf(floor_key, glow_s[g * kTileM + row_in_tile]);
+          if (rank == sub) my_group = g;
+        }
+      }
+      // ---------------- collect: sub s scans the row's s-th best group for keys >= floor
+      // (the kept groups' two best keys are >= floor, so at least k keys qualify)
+      if (sub < p.topk_group) {
+        const int base = my_group * 32;
+        uint32_t mask = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          mask |= (key_s[(base + j) * kTileM + row_in_tile] >= floor_key) ? (1u << j) : 0u;
+        const uint32_t mine = __popc(mask);
+        const uint32_t first = atomicAdd(&sh.cand_count[row_in_tile], mine);
+        const uint32_t most = __reduce_max_sync(0xffffffffu, mine);
+#pragma unroll 1
+        for (uint32_t i = 0; i < most; ++i) {
+          if (mask != 0 && first + i < kCandCap) {
+            const int j = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const uint32_t bits = __float_as_uint(key_s[(base + j) * kTileM + row_in_tile]);
+            // order-preserving map of the float onto unsigned integers
+            cand_hi[(first + i) * kTileM + row_in_tile] = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
+            cand_lo[(first + i) * kTileM + row_in_tile] = ~static_cast<uint32_t>(base + j);
+          }
+        }
+      }
+    }
+    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    uint32_t* out_hi = reinterpret_cast<uint32_t*>(gscore_s);               // [8][128], group scores are dead now
+    uint32_t* out_lo = out_hi + FB_MAX_TOPK * kTileM;
+    bool overflow = false;
+    if (got && fast_select) {
+      // ---------------- rank: candidate c beats d if its key is larger, or equal with a
+      // lower expert id; a candidate with fewer than k better ones is the rank-th choice
+      const uint32_t* cand_hi = reinterpret_cast<const uint32_t*>(merge_v);
+      const uint32_t* cand_lo = cand_hi + kCandCap * kTileM;
+      const uint32_t n_all = sh.cand_count[row_in_tile];
+      overflow = n_all > kCandCap;
+      const uint32_t n = overflow ? 0u : n_all;
+      const uint32_t n_most = __reduce_max_sync(0xffffffffu, n);
+#pragma unroll 1
+      for (uint32_t tier = 0; tier * 4 * kEpiSubs < n_most; ++tier) {
+        unsigned long long mykey[4];
+        uint32_t rank[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
+          const uint32_t cc = c < n ? c : 0;
+          mykey[t] = (static_cast<unsigned long long>(cand_hi[cc * kTileM + row_in_tile]) << 32) |
+                     cand_lo[cc * kTileM + row_in_tile];
+          rank[t] = 0;
+        }
+#pragma unroll 2
+        for (uint32_t d = 0; d < n_most; ++d) {
+          const uint32_t dd = d < n ? d : 0;
+          const unsigned long long other = d < n
+              ? (static_cast<unsigned long long>(cand_hi[dd * kTileM + row_in_tile]) << 32) | cand_lo[dd * kTileM + row_in_tile]
+              : 0ull;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) rank[t] += other > mykey[t] ? 1u : 0u;
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
+          if (c < n && rank[t] < static_cast<uint32_t>(FB_MAX_TOPK)) {
+            out_hi[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t] >> 32);
+            out_lo[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t]);
+          }
+        }
+      }
+    }
+    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    if (got && fast_select && sub == 0) {
+      if (!overflow) {
+#pragma unroll
+        for (int j = 0; j < FB_MAX_TOPK; ++j) {
+          if (j < k) {
+            const uint32_t u = out_hi[j * kTileM + row_in_tile];
+            top.v[j] = __uint_as_float(u ^ ((u >> 31) ? 0x80000000u : 0xffffffffu));
+            top.i[j] = static_cast<int32_t>(~out_lo[j * kTileM + row_in_tile]);
+          }
+        }
+      }
+      if (__any_sync(0xffffffffu, overflow)) {
+        // More than kCandCap keys reached the floor (many equal keys): plain scan of the
+        // kept groups for the rows concerned.
+        if (overflow) {
+          float sc[8];
+#pragma unroll
+          for (int g = 0; g < 8; ++g) sc[g] = -INFINITY;
+          // group scores were overwritten by the output area: recompute them from the keys
+          for (int g = 0; g < p.n_group; ++g) {
+            float a1 = -INFINITY, a2 = -INFINITY;
+            for (int j = 0; j < 32; ++j) {
+              const float x = key_s[(g * 32 + j) * kTileM + row_in_tile];
+              a2 = fmaxf(a2, fminf(a1, x));
+              a1 = fmaxf(a1, x);
+            }
+#pragma unroll
+            for (int h = 0; h < 8; ++h) if (h == g) sc[h] = a1 + a2;
+          }
+          top.init();
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            int rank = 0;
+#pragma unroll
+            for (int h = 0; h < 8; ++h)
+              if (h != g) rank += (sc[h] > sc[g] || (sc[h] == sc[g] && h < g)) ? 1 : 0;
+            if (g < p.n_group && rank < p.topk_group) {
+              for (int j = 0; j < 32; ++j) {
+                const float x = key_s[(g * 32 + j) * kTileM + row_in_tile];
+                if (x > top.v[FB_MAX_TOPK - 1] || x == top.v[FB_MAX_TOPK - 1]) top.insert_any_order(x, g * 32 + j);
+              }
+            }
+          }
+        }
+      }
+    }
+    if (got && !fast_select) {
+      // ---------------- choose the groups; lower bound for the k-th key
+      uint32_t keep = 1u;
+      float floor_key = -INFINITY;
+      if (sigmoid_gate) {
+        TopK gtop;                                          // FB_MAX_TOPK >= topk_group
+        gtop.init();
+        for (int g = 0; g < p.n_group; ++g) {
+          const float sc = gscore_s[g * kTileM + row_in_tile];
+          if (sc > gtop.v[FB_MAX_TOPK - 1]) gtop.insert(sc, g);
+        }
+        keep = 0;
+        float low = INFINITY;
+#pragma unroll
+        for (int j = 0; j < FB_MAX_TOPK; ++j) {
+          if (j < p.topk_group) {
+            keep |= 1u << gtop.i[j];
+            low = fminf(low, glow_s[gtop.i[j] * kTileM + row_in_tile]);
+          }
+        }
+        // The kept groups' best (two) keys are eligible; if there are at least k of
+        // them, the smallest is a lower bound for the k-th largest eligible key.
+        if (p.topk_group * (gs >= 2 ? 2 : 1) >= k) floor_key = low;
+      }
+      // ---------------- pass 2
+      for (int c = 0; c < n_chunks; ++c) {
+        const int owner = splittable ? (c / chunks_per_group) % kEpiSubs : 0;
+        if (owner != sub) continue;
+        const int c0 = c * 32;
+        int g = sigmoid_gate ? c0 / gs : 0, pos = sigmoid_gate ? c0 % gs : 0;
+        const int g_start = g, pos_start = pos;
+        uint32_t cnt = 0;
+        unsigned long long packed = 0;                      // up to 8 column offsets, one byte each
+#pragma unroll 4
+        for (int j = 0; j < 32; ++j) {
+          const int e = c0 + j;
+          if (e < E) {
+            const float x = key_s[e * kTileM + row_in_tile];
+            if (((keep >> g) & 1u) && x >= floor_key && x > top.v[FB_MAX_TOPK - 1]) {
+              if (cnt < 8) packed |= static_cast<unsigned long long>(j) << (8 * cnt);
+              ++cnt;
+            }
+            if (++pos == gs) { ++g; pos = 0; }
+          }
+        }
+        const uint32_t most = __reduce_max_sync(0xffffffffu, cnt);
+        if (most > 8) {
+          // too many candidates for the packed list somewhere in the warp: plain scan
+          g = g_start; pos = pos_start;
+#pragma unroll 1
+          for (int j = 0; j < 32; ++j) {
+            const int e = c0 + j;
+            if (e < E) {
+              const float x = key_s[e * kTileM + row_in_tile];
+              if (((keep >> g) & 1u) && x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+              if (++pos == gs) { ++g; pos = 0; }
+            }
+          }
+        } else {
+#pragma unroll 1
+          for (uint32_t i = 0; i < most; ++i) {
+            if (i < cnt) {
+              const int e = c0 + static_cast<int>((packed >> (8 * i)) & 0xffu);
+              const float x = key_s[e * kTileM + row_in_tile];
+              if (x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+            }
+          }
+        }
+      }
+      // ---------------- hand the partial lists to sub 0
+      if (sub != 0) {
+#pragma unroll
+        for (int j = 0; j < FB_MAX_TOPK; ++j) {
+          merge_v[((sub - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile] = top.v[j];
+          merge_i[((sub - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile] = top.i[j];
+        }
+      }
+      if (want_sum) {
+        part_s[(sub * 2 + 0) * kTileM + row_in_tile] = sm_max;
+        part_s[(sub * 2 + 1) * kTileM + row_in_tile] = sm_sum;
+      }
+    }
+    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    const bool writer = got && valid && sub == 0;
+    if (got && sub == 0 && !fast_select) {
+#pragma unroll 1
+      for (int s2 = 1; s2 < kEpiSubs; ++s2) {
+#pragma unroll 1
+        for (int j = 0; j < FB_MAX_TOPK; ++j) {
+          const float x = merge_v[((s2 - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile];
+          if (x > -INFINITY) top.insert_any_order(x, merge_i[((s2 - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile]);
+        }
+      }
+      if (want_sum) {
+        float mx = -INFINITY;
+        for (int s2 = 0; s2 < kEpiSubs; ++s2) mx = fmaxf(mx, part_s[(s2 * 2 + 0) * kTileM + row_in_tile]);
+        float sum = 0.0f;
+        for (int s2 = 0; s2 < kEpiSubs; ++s2)
+          sum += part_s[(s2 * 2 + 1) * kTileM + row_in_tile] * __expf(part_s[(s2 * 2 + 0) * kTileM + row_in_tile] - mx);
+        sm_max = mx; sm_sum = sum;
+      }
+    }
 
     // ---- outputs per row
-    if (got && valid) {
+    if (writer) {
       if (p.topk_ids != nullptr) {
 #pragma unroll
         for (int j = 0; j < FB_MAX_TOPK; ++j)
@@ -271,14 +598,15 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       if (p.topk_w != nullptr) {
         float w[FB_MAX_TOPK];
         float wsum = 0.0f;
+        const float ref = top.v[0];                         // row maximum of the keys
 #pragma unroll
         for (int j = 0; j < FB_MAX_TOPK; ++j) {
-          if (p.gate == FB_GATE_SOFTMAX_TOPK) w[j] = (j < k) ? __expf(top.v[j] - sm_max) : 0.0f;
+          if (!sigmoid_gate) w[j] = (j < k) ? __expf(top.v[j] - ref) : 0.0f;
           else w[j] = (j < k) ? top.v[j] - sh.select_bias[top.i[j]] : 0.0f;   // unbiased sigmoid score
           wsum += w[j];
         }
         float scale;
-        if (p.gate == FB_GATE_SOFTMAX_TOPK) scale = p.renorm ? 1.0f / wsum : 1.0f / sm_sum;
+        if (!sigmoid_gate) scale = p.renorm ? 1.0f / wsum : 1.0f / (sm_sum * __expf(sm_max - ref));
         else scale = p.renorm ? p.route_scale / wsum : p.route_scale;
 #pragma unroll
         for (int j = 0; j < FB_MAX_TOPK; ++j)
@@ -286,12 +614,22 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
     }
     // ---- histogram: one shared-memory atomic per distinct expert per warp (Eq. 5)
+    if (sub == 0) {
+      if (E > 32) {
+        // many bins: lanes rarely collide, plain shared-memory atomics are cheapest
 #pragma unroll
-    for (int j = 0; j < FB_MAX_TOPK; ++j) {
-      if (j < k) {
-        const int e = (got && valid) ? top.i[j] : -1;
-        const uint32_t same = __match_any_sync(0xffffffffu, e);
-        if (e >= 0 && lane == __ffs(same) - 1) atomicAdd(&sh.hist[e], __popc(same));
+        for (int j = 0; j < FB_MAX_TOPK; ++j)
+          if (j < k && writer) atomicAdd(&sh.hist[top.i[j]], 1u);
+      } else {
+        // few bins: add once per distinct expert per warp
+#pragma unroll
+        for (int j = 0; j < FB_MAX_TOPK; ++j) {
+          if (j < k) {
+            const int e = writer ? top.i[j] : -1;
+            const uint32_t same = __match_any_sync(0xffffffffu, e);
+            if (e >= 0 && lane == __ffs(same) - 1) atomicAdd(&sh.hist[e], __popc(same));
+          }
+        }
       }
     }
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
@@ -322,7 +660,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (et == 0) *p.ticket = 0;
         if (sh.abort_flag) { if (et == 0) atomicCAS(p.status, 0, FB_ERR_TIMEOUT); }
         named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-        if (p.mode == kModePredictPlan) plan_swaps_block(p.plan, sh.plan, et, p.status);
+        if (p.mode == kModePredictPlan && warp == 2) plan_swaps_warp(p.plan, sh.plan, lane, p.status);
       }
     }
   }
@@ -336,14 +674,16 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   }
 }
 
-// Stand-alone planner: one block of kPlanThreads threads.
+// Stand-alone planner: one warp.
 __global__ void __launch_bounds__(kPlanThreads, 1)
 fb_plan_kernel(const __grid_constant__ PlanParams p, const uint32_t* __restrict__ counts, int32_t* status) {
   __shared__ PlanShared sh;
   const int t = threadIdx.x;
+  plan_clear(sh, t, kPlanThreads);
   for (int e = t; e < p.E; e += kPlanThreads) sh.cnt[e] = counts[e];
-  named_bar_sync(kPlanBarrierId, kPlanThreads);
-  plan_swaps_block(p, sh, t, status);
+  __syncwarp();
+  plan_load_placement(p, sh, t, kPlanThreads);
+  plan_swaps_warp(p, sh, t, status);
 }
 
 }  // namespace fb

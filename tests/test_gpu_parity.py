@@ -163,7 +163,7 @@ def test_planner_worked_examples_on_gpu(golden):
         dev = torch.device("cuda")
         t = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
         out_pi, swaps, n, lb, la = t([0] * E), t([0] * 12), t([0]), t([0] * R), t([0] * R)
-        bud = B.make_budget(max_swaps=gd["max_swaps"], gamma_num=gd["gamma_num"], gamma_den=gd["gamma_den"])
+        bud = B.make_budget(max_swaps=min(gd["max_swaps"], E // 2), gamma_num=gd["gamma_num"], gamma_den=gd["gamma_den"])
         ctx.fb_plan_swaps(t(gd["counts"]), t(gd["expert_to_slot"]), bud, 0, out_pi, swaps, n, lb, la)
         assert ctx.fb_device_status() == 0
         k = int(n.item())

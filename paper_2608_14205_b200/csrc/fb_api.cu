@@ -22,6 +22,7 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 struct MapEntry {
   const void* ptr = nullptr;
   int64_t rows = -1;
+  uint32_t box_rows = 0;
   CUtensorMap map;
 };
 
@@ -33,9 +34,9 @@ struct fb_ctx {
   fb_config cfg;
   int device = 0;
   int N = 0;                      // experts padded to a multiple of 16 (UMMA N)
-  int stages = 0;
+  int stages[2] = {0, 0};         // pipeline depth for the single-block and the pair kernel
   int tmem_cols = 0;
-  size_t smem_bytes = 0;
+  size_t smem_bytes[2] = {0, 0};
   int max_tiles = 0;
   EncodeTiledFn encode = nullptr;
   // device scratch
@@ -97,7 +98,10 @@ fb_status check_config(const fb_config& c) {
 fb_status make_map(fb_ctx* ctx, MapEntry* cache, int* next, const void* ptr, int64_t rows, uint32_t box_rows,
                    const CUtensorMap** out) {
   for (int i = 0; i < kMapCache; ++i)
-    if (cache[i].ptr == ptr && cache[i].rows == rows) { *out = &cache[i].map; return FB_OK; }
+    if (cache[i].ptr == ptr && cache[i].rows == rows && cache[i].box_rows == box_rows) {
+      *out = &cache[i].map;
+      return FB_OK;
+    }
   if ((reinterpret_cast<uintptr_t>(ptr) & 15u) != 0) return FB_ERR_INVALID_ARG;
   MapEntry& e = cache[*next];
   *next = (*next + 1) % kMapCache;
@@ -111,6 +115,7 @@ fb_status make_map(fb_ctx* ctx, MapEntry* cache, int* next, const void* ptr, int
   if (r != CUDA_SUCCESS) { e.ptr = nullptr; e.rows = -1; return FB_ERR_CUDA; }
   e.ptr = ptr;
   e.rows = rows;
+  e.box_rows = box_rows;
   *out = &e.map;
   return FB_OK;
 }
@@ -162,7 +167,10 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   const CUtensorMap *mx = nullptr, *mw = nullptr;
   fb_status st = make_map(ctx, ctx->x_maps, &ctx->x_next, x, T, fb::kTileM, &mx);
   if (st != FB_OK) return st;
-  st = make_map(ctx, ctx->w_maps, &ctx->w_next, router->W, ctx->cfg.E, static_cast<uint32_t>(ctx->N), &mw);
+  const int tiles = (T + fb::kTileM - 1) / fb::kTileM;
+  const int pair = (tiles > 1 && ctx->stages[1] >= 2) ? 1 : 0;   // a single tile gains nothing from a partner
+  st = make_map(ctx, ctx->w_maps, &ctx->w_next, router->W, ctx->cfg.E,
+                static_cast<uint32_t>(pair ? ctx->N / 2 : ctx->N), &mw);
   if (st != FB_OK) return st;
   fb::RouterParams p;
   memset(&p, 0, sizeof(p));
@@ -172,7 +180,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.topk_group = c.gate == FB_GATE_SIGMOID_GROUP_TOPK ? c.topk_group : 1;
   p.renorm = c.renorm; p.route_scale = c.route_scale;
   p.num_kb = (c.d + fb::kBlockK - 1) / fb::kBlockK;
-  p.stages = ctx->stages;
+  p.stages = ctx->stages[pair];
   p.tmem_cols = ctx->tmem_cols;
   p.mode = mode;
   p.logit_bias = router->logit_bias;
@@ -186,10 +194,28 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.logits = logits;
   p.tile_counts = ctx->tile_counts;
   if (plan) p.plan = *plan;
-  const int tiles = (T + fb::kTileM - 1) / fb::kTileM;
-  fb::fb_router_kernel<<<tiles, fb::kRouterThreads, ctx->smem_bytes, stream>>>(*mx, *mw, p);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(fb::kRouterThreads, 1, 1);
+  cfg.dynamicSmemBytes = ctx->smem_bytes[pair];
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  cudaError_t err;
+  if (pair) {
+    cfg.gridDim = dim3(static_cast<unsigned>((tiles + 1) / 2 * 2), 1, 1);
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mw, p);
+  } else {
+    cfg.gridDim = dim3(static_cast<unsigned>(tiles), 1, 1);
+    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1>, *mx, *mw, p);
+  }
   ++ctx->launches;
-  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+  return err == cudaSuccess ? FB_OK : FB_ERR_CUDA;
 }
 
 fb_status launch_plan(fb_ctx* ctx, const fb::PlanParams& pp, const uint32_t* counts, cudaStream_t stream) {
@@ -249,16 +275,20 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   ctx->device = device;
   ctx->N = (cfg->E + 15) / 16 * 16;
   ctx->tmem_cols = next_pow2_at_least_32(ctx->N);
-  const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N) * fb::kBlockK * 2;
   const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
-  int stages = static_cast<int>((budget - 1024) / stage_bytes);
-  if (stages > fb::kMaxStages) stages = fb::kMaxStages;
-  if (stages < 2) { delete ctx; return FB_ERR_UNSUPPORTED_SHAPE; }
-  ctx->stages = stages;
-  size_t dyn = stages * stage_bytes;
-  if (dyn < fb::epilogue_scratch_bytes(ctx->N)) dyn = fb::epilogue_scratch_bytes(ctx->N);
-  if (dyn + 1024 > budget) { delete ctx; return FB_ERR_UNSUPPORTED_SHAPE; }
-  ctx->smem_bytes = dyn + 1024;
+  for (int pair = 0; pair < 2; ++pair) {
+    const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N / (pair + 1)) * fb::kBlockK * 2;
+    int stages = static_cast<int>((budget - 1024) / stage_bytes);
+    if (stages > fb::kMaxStages) stages = fb::kMaxStages;
+    size_t dyn = stages * stage_bytes;
+    if (dyn < fb::epilogue_scratch_bytes(ctx->N)) dyn = fb::epilogue_scratch_bytes(ctx->N);
+    if (stages < 2 || dyn + 1024 > budget) {
+      if (pair == 0) { delete ctx; return FB_ERR_UNSUPPORTED_SHAPE; }
+      stages = 0;                                      // pair kernel not usable for this shape
+    }
+    ctx->stages[pair] = stages;
+    ctx->smem_bytes[pair] = dyn + 1024;
+  }
   ctx->max_tiles = (cfg->T_max + fb::kTileM - 1) / fb::kTileM;
 
   void* fn = nullptr;
@@ -269,8 +299,11 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
     return FB_ERR_CUDA;
   }
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(ctx->smem_bytes)) == cudaSuccess;
+  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(ctx->smem_bytes[0])) == cudaSuccess;
+  if (ctx->stages[1] >= 2)
+    ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(ctx->smem_bytes[1])) == cudaSuccess;
   ok = ok && dev_alloc(&ctx->counts_scratch, FB_MAX_EXPERTS) && dev_alloc(&ctx->ticket, 1) &&
        dev_alloc(&ctx->status, 1) &&
        dev_alloc(&ctx->tile_counts, static_cast<size_t>(ctx->max_tiles) * cfg->E);

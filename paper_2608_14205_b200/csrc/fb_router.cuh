@@ -142,6 +142,13 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32
   tmem_ld_wait();
 }
 
+// kCtas == 1: every block computes its 128 x N tile alone.
+// kCtas == 2: launched in clusters of two; the pair shares one 256 x N MMA
+// (tcgen05 cta_group::2).  Each block still loads its own 128 rows of x, but only half
+// of the W tile, which halves the W traffic out of L2 and leaves room for more pipeline
+// stages.  The even block of the pair issues the MMAs and owns the "full" barriers;
+// both blocks get their stage-free and accumulator-ready signals from its commits.
+template <int kCtas>
 __global__ void __launch_bounds__(kRouterThreads, 1)
 fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                  const __grid_constant__ RouterParams p) {
@@ -151,7 +158,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int tile = blockIdx.x;
-  const uint32_t b_tile_bytes = static_cast<uint32_t>(p.N) * kBlockK * 2;
+  const uint32_t cta_rank = kCtas == 2 ? cluster_ctarank() : 0u;
+  const uint32_t b_tile_bytes = static_cast<uint32_t>(p.N / kCtas) * kBlockK * 2;
   const uint32_t stage_bytes = kATileBytes + b_tile_bytes;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzle atoms need 1024-byte alignment
   volatile int* abort_flag = &sh.abort_flag;
@@ -169,8 +177,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     prefetch_tensormap(&tmap_w);
   }
   if (warp == 1) {
-    tmem_alloc<1>(smem_u32(&sh.tmem_base), static_cast<uint32_t>(p.tmem_cols));
-    tmem_relinquish<1>();
+    tmem_alloc<kCtas>(smem_u32(&sh.tmem_base), static_cast<uint32_t>(p.tmem_cols));
+    tmem_relinquish<kCtas>();
   }
   if (warp >= 2) {
     const int et = threadIdx.x - 64;
@@ -184,6 +192,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   }
   tcgen05_fence_before();
   __syncthreads();
+  if (kCtas == 2) { cluster_arrive(); cluster_wait(); }   // the partner's barriers and TMEM are ready too
   tcgen05_fence_after();
   const uint32_t tmem_base = sh.tmem_base;
 
@@ -195,23 +204,33 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       for (int kb = 0; kb < p.num_kb; ++kb) {
         const int s = kb % p.stages;
         const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
-        if (!mbar_wait(smem_u32(&sh.empty_bar[s]), phase ^ 1u, abort_flag)) break;
-        const uint32_t full = smem_u32(&sh.full_bar[s]);
-        mbar_arrive_expect_tx(full, stage_bytes);
+        if (!mbar_wait<kCtas == 2>(smem_u32(&sh.empty_bar[s]), phase ^ 1u, abort_flag)) break;
         const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
-        tma_load_2d(a_dst, &tmap_x, full, kb * kBlockK, tile * kTileM, pol_x);
-        tma_load_2d(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK, 0, pol_w);
+        if (kCtas == 1) {
+          const uint32_t full = smem_u32(&sh.full_bar[s]);
+          mbar_arrive_expect_tx(full, stage_bytes);
+          tma_load_2d(a_dst, &tmap_x, full, kb * kBlockK, tile * kTileM, pol_x);
+          tma_load_2d(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK, 0, pol_w);
+        } else {
+          // both blocks report their bytes to the even block's barrier, which expects
+          // the bytes of the whole pair
+          const uint32_t full = map_to_cta(smem_u32(&sh.full_bar[s]), 0u);
+          if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&sh.full_bar[s]), 2u * stage_bytes);
+          tma_load_2d_pair(a_dst, &tmap_x, full, kb * kBlockK, tile * kTileM, pol_x);
+          tma_load_2d_pair(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK,
+                           static_cast<int32_t>(cta_rank) * (p.N / 2), pol_w);
+        }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16_f32(kTileM, static_cast<uint32_t>(p.N));
+    if (lane == 0 && cta_rank == 0) {
+      const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.N));
       bool ok = true;
       for (int kb = 0; kb < p.num_kb && ok; ++kb) {
         const int s = kb % p.stages;
         const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
-        ok = mbar_wait(smem_u32(&sh.full_bar[s]), phase, abort_flag);
+        ok = mbar_wait<kCtas == 2>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
         if (!ok) break;
         tcgen05_fence_after();
         const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
@@ -220,11 +239,15 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 #pragma unroll
         for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
           // advance 16 elements = 32 bytes inside the swizzled row: +2 in the address field
-          umma_bf16<1>(tmem_base, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          umma_bf16<kCtas>(tmem_base, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
         }
-        umma_commit_1cta(smem_u32(&sh.empty_bar[s]));     // frees the stage when these MMAs retire
+        // frees the stage (in both blocks of a pair) when these MMAs retire
+        if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.empty_bar[s]));
+        else umma_commit_2cta(smem_u32(&sh.empty_bar[s]), 0x3);
       }
-      umma_commit_1cta(smem_u32(&sh.accum_bar));          // accumulator complete
+      // accumulator complete
+      if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.accum_bar));
+      else umma_commit_2cta(smem_u32(&sh.accum_bar), 0x3);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -250,7 +273,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // While the main loop runs, stage the placement for the planner (any block may turn
     // out to be the last one).
     if (p.mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
-    const bool got = mbar_wait(smem_u32(&sh.accum_bar), 0u, abort_flag);
+    const bool got = mbar_wait<kCtas == 2>(smem_u32(&sh.accum_bar), 0u, abort_flag);
     tcgen05_fence_after();
 
     // scratch carved out of the (now idle) pipeline stages
@@ -634,8 +657,9 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
     if (p.mode == kModeDispatch) {
-      for (int e = et; e < E; e += kEpilogueThreads)
-        p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
+      if (static_cast<long long>(tile) * kTileM < p.T)       // the padding block of an odd pair owns no tile
+        for (int e = et; e < E; e += kEpilogueThreads)
+          p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
     } else {
       for (int e = et; e < E; e += kEpilogueThreads) {
         const uint32_t c = sh.hist[e];
@@ -666,11 +690,13 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   }
 
   // ---------------------------------------------------------------- teardown
+  tcgen05_fence_before();
   __syncthreads();
+  if (kCtas == 2) { cluster_arrive(); cluster_wait(); }   // nobody leaves while the partner may still signal it
   if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(p.status, 0, FB_ERR_TIMEOUT);
   if (warp == 1) {
     tcgen05_fence_after();
-    tmem_dealloc<1>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+    tmem_dealloc<kCtas>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
   }
 }
 

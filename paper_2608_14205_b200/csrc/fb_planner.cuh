@@ -133,6 +133,17 @@ __device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh
   const long long gnum = p.gamma_den ? p.gamma_num : 0;
   const long long gden = p.gamma_den ? p.gamma_den : 1;
   const int rpn = p.ranks_per_node;
+  const bool uniform = p.expert_bytes_table == nullptr;     // one cost per link class
+  // Candidate c (0 <= c < m*m) pairs slot c / m of the heavy rank with slot c % m of the
+  // light one.  A lane's first candidates are fixed for the whole call: divide once.
+  constexpr int kSlotsPerLane = 8;                          // covers m <= 16 without a loop
+  int cand_ia[kSlotsPerLane], cand_ib[kSlotsPerLane];
+#pragma unroll
+  for (int t = 0; t < kSlotsPerLane; ++t) {
+    const int c = lane + 32 * t;
+    cand_ia[t] = c / m;
+    cand_ib[t] = c % m;
+  }
   unsigned long long global_spent = 0;
   uint32_t n = 0;
   while (n < p.max_swaps) {
@@ -164,29 +175,49 @@ __device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh
     const unsigned long long rs_a = sh.rank_spent[a], rs_b = sh.rank_spent[b];
     const unsigned long long rank_spent = rs_a > rs_b ? rs_a : rs_b;
 
+    if (uniform) {
+      // same cost for every candidate of this iteration: one budget test decides for all
+      const unsigned long long c_ns = p.uniform_cost_ns[cls];
+      if (p.global_ns != FB_BUDGET_OFF && (c_ns > p.global_ns || global_spent > p.global_ns - c_ns)) break;
+      if (p.rank_ns != FB_BUDGET_OFF && (c_ns > p.rank_ns || rank_spent > p.rank_ns - c_ns)) break;
+      if (p.link_ns != FB_BUDGET_OFF && (c_ns > p.link_ns || link_spent > p.link_ns - c_ns)) break;
+    }
     PlanCandidate best;
     best.benefit = 0; best.cost = 1; best.ea = -1; best.eb = -1;
-    for (int c = lane; c < m * m; c += 32) {
-      const int ea = sh.expert_at[a * m + c / m];
-      const int eb = sh.expert_at[b * m + c % m];
-      if (sh.moved[ea] || sh.moved[eb]) continue;
-      const long long dlt = static_cast<long long>(sh.cnt[ea]) - static_cast<long long>(sh.cnt[eb]);
+    const int D = static_cast<int>(La - Lb);                    // > tau >= 0, below 2^22
+    const int mm = m * m;
+    auto consider = [&](int ia, int ib) {
+      const int ea = sh.expert_at[a * m + ia];
+      const int eb = sh.expert_at[b * m + ib];
+      if (sh.moved[ea] || sh.moved[eb]) return;
+      const int dlt = static_cast<int>(sh.cnt[ea]) - static_cast<int>(sh.cnt[eb]);   // tokens moved a -> b
       long long Mn = La - dlt;                                  // Eq. 6
       if (Lb + dlt > Mn) Mn = Lb + dlt;                         // Eq. 7
       if (M2 > Mn) Mn = M2;
       // gamma_den * (Phi(L) - Phi(L')): the mean is unchanged by a swap, so the
       // variance term reduces to 2 dlt (La - Lb - dlt).
-      const long long benefit = gden * (La - Mn) + gnum * 2 * dlt * (La - Lb - dlt);
-      if (benefit <= 0) continue;
+      const long long var2 = static_cast<long long>(dlt) * static_cast<long long>(D - dlt);
+      const long long benefit = gden * (La - Mn) + 2 * gnum * var2;
+      if (benefit <= 0) return;
       PlanCandidate cand;
       cand.benefit = benefit;
-      cand.cost = plan_cost_ns(p, cls, ea, eb);                 // Eq. 9
       cand.ea = ea; cand.eb = eb;
-      if (p.global_ns != FB_BUDGET_OFF && (cand.cost > p.global_ns || global_spent > p.global_ns - cand.cost)) continue;
-      if (p.rank_ns != FB_BUDGET_OFF && (cand.cost > p.rank_ns || rank_spent > p.rank_ns - cand.cost)) continue;
-      if (p.link_ns != FB_BUDGET_OFF && (cand.cost > p.link_ns || link_spent > p.link_ns - cand.cost)) continue;
-      if (plan_better(cand, best)) best = cand;
-    }
+      if (uniform) {
+        cand.cost = 1;                                          // equal for all: compare benefits only
+        if (best.ea < 0 || benefit > best.benefit ||
+            (benefit == best.benefit && (ea < best.ea || (ea == best.ea && eb < best.eb)))) best = cand;
+      } else {
+        cand.cost = plan_cost_ns(p, cls, ea, eb);               // Eq. 9
+        if (p.global_ns != FB_BUDGET_OFF && (cand.cost > p.global_ns || global_spent > p.global_ns - cand.cost)) return;
+        if (p.rank_ns != FB_BUDGET_OFF && (cand.cost > p.rank_ns || rank_spent > p.rank_ns - cand.cost)) return;
+        if (p.link_ns != FB_BUDGET_OFF && (cand.cost > p.link_ns || link_spent > p.link_ns - cand.cost)) return;
+        if (plan_better(cand, best)) best = cand;
+      }
+    };
+#pragma unroll
+    for (int t = 0; t < kSlotsPerLane; ++t)
+      if (lane + 32 * t < mm) consider(cand_ia[t], cand_ib[t]);
+    for (int c = lane + 32 * kSlotsPerLane; c < mm; c += 32) consider(c / m, c % m);
     if (p.expert_bytes_table == nullptr) {
       // every candidate of this iteration has the same cost: the largest benefit wins,
       // ties go to the smallest (ea, eb).  Three 32-bit warp reductions.

@@ -37,6 +37,7 @@ constexpr int kEpiSubs = 4;            // epilogue warps per row quarter
 constexpr int kEpilogueThreads = 128 * kEpiSubs;
 constexpr int kRouterThreads = 64 + kEpilogueThreads;
 constexpr int kATileBytes = kTileM * kBlockK * 2;
+constexpr uint32_t kAccumBarrierId = 2;      // named barrier: accumulator finished (MMA warp -> epilogue warps)
 
 enum RouterMode : int {
   kModePredict = 0,        // histogram -> counts
@@ -121,6 +122,20 @@ __host__ __device__ constexpr size_t epilogue_scratch_bytes(int N) {
 
 static_assert(2 * kCandCap >= 2 * (kEpiSubs - 1) * FB_MAX_TOPK + kEpiSubs * 2, "merge area must fit in the candidate area");
 
+// Same value with the reciprocal computed on the FMA pipe: a bit-trick first guess
+// (12% off) refined by three Newton steps to ~1e-7 relative error.  The argument of the
+// reciprocal is 1 + 2^x in [1, 2^116] thanks to the clamp, far from overflow.
+__device__ __forceinline__ float fb_sigmoid_fma(float z) {
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaxf(z, -80.0f) * -1.4426950408889634f));
+  const float y = 1.0f + e;
+  float r = __int_as_float(0x7EF311C7 - __float_as_int(y));
+  r = r * (2.0f - y * r);
+  r = r * (2.0f - y * r);
+  r = r * (2.0f - y * r);
+  return r;
+}
+
 struct RouterShared {
   uint64_t full_bar[kMaxStages];
   uint64_t empty_bar[kMaxStages];
@@ -128,8 +143,9 @@ struct RouterShared {
   uint32_t tmem_base;
   int32_t abort_flag;
   int32_t is_last;
+  int32_t accum_ok;
   float logit_bias[FB_MAX_EXPERTS + 32];     // + 32: a partial last chunk is read in full
-  float select_bias[FB_MAX_EXPERTS + 32];
+  alignas(16) float select_bias[FB_MAX_EXPERTS + 32];
   uint32_t hist[FB_MAX_EXPERTS];
   uint32_t cand_count[kTileM];               // fast selection path: candidates claimed per row
   PlanShared plan;
@@ -249,6 +265,11 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.accum_bar));
       else umma_commit_2cta(smem_u32(&sh.accum_bar), 0x3);
     }
+    // One thread polls for the finished accumulator on behalf of the 16 epilogue warps,
+    // which sleep at a hardware barrier meanwhile (no issue slots, no power).
+    if (lane == 0) sh.accum_ok = mbar_wait<kCtas == 2>(smem_u32(&sh.accum_bar), 0u, abort_flag) ? 1 : 0;
+    __syncwarp();
+    named_bar_arrive(kAccumBarrierId, kEpilogueThreads + 32);
   } else {
     // ------------------------------------------------------------ epilogue
     const int et = threadIdx.x - 64;                       // 0 .. kEpilogueThreads-1
@@ -273,7 +294,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // While the main loop runs, stage the placement for the planner (any block may turn
     // out to be the last one).
     if (p.mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
-    const bool got = mbar_wait<kCtas == 2>(smem_u32(&sh.accum_bar), 0u, abort_flag);
+    named_bar_sync(kAccumBarrierId, kEpilogueThreads + 32);
+    const bool got = sh.accum_ok != 0;
     tcgen05_fence_after();
 
     // scratch carved out of the (now idle) pipeline stages
@@ -305,7 +327,20 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             if (c0 + j < E)
               p.logits[row * E + c0 + j] = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
         }
-        if (sigmoid_gate) {
+        if (sigmoid_gate && c0 + 32 <= E && !has_lb) {
+          // whole chunk valid, no logit bias (the common case).  The sigmoid needs two
+          // special-function results per key and that unit is the bottleneck here, so
+          // every other key gets its reciprocal from Newton steps on the FMA pipe instead.
+          const float4* sb4 = reinterpret_cast<const float4*>(&sh.select_bias[c0]);
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4) {
+            const float4 b = sb4[j4];
+            q[4 * j4 + 0] = fb_sigmoid(__uint_as_float(r[4 * j4 + 0])) + b.x;
+            q[4 * j4 + 1] = fb_sigmoid_fma(__uint_as_float(r[4 * j4 + 1])) + b.y;
+            q[4 * j4 + 2] = fb_sigmoid(__uint_as_float(r[4 * j4 + 2])) + b.z;
+            q[4 * j4 + 3] = fb_sigmoid_fma(__uint_as_float(r[4 * j4 + 3])) + b.w;
+          }
+        } else if (sigmoid_gate) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const float z = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);

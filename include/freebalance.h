@@ -202,6 +202,36 @@ fb_status fb_layer_step_host(fb_ctx* ctx, const fb_router* router,
                              uint32_t* rank_offsets, int32_t* perm, int32_t* inv_perm,
                              uint32_t* rank_load, fb_stream stream);
 
+/* fb_predict_load for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of stage 1, same computation.)
+ *
+ * Who needs it: code that runs after an inference server has frozen its memory pool
+ * and forbids any further cudaMalloc (allocations there synchronise the device and
+ * fragment the pool), code inside a region where allocation is illegal, and hosts that
+ * link the library but may not create an fb_ctx because fb_create allocates.  This call
+ * takes no context and performs no cudaMalloc / cudaFree and calls no allocating library
+ * routine; the caller passes inputs and outputs as for fb_predict_load (`logits` is not
+ * offered).
+ *
+ * The kernel's scratch - FB_STATIC_MAX_EXPERTS histogram counters, the finished-block
+ * ticket and a status word, 1280 bytes - is a fixed array inside the library image, so
+ * every GPU that loads the library holds those bytes until the process exits.
+ *   - cfg->E above FB_STATIC_MAX_EXPERTS is refused with FB_ERR_UNSUPPORTED_SHAPE; the
+ *     other limits are those of fb_create.
+ *   - The first call on a device looks up the array's device address and sets kernel
+ *     attributes (once per device; the shape-dependent part again when cfg changes).
+ *     Make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  Each call clears it on `stream` before
+ *     its kernel, so a call is not disturbed by what an earlier one left behind, but two
+ *     calls that overlap on the GPU (different streams) race on it: serialise them.
+ *   - status_word: dev i32 [1] or NULL.  If given (zeroed by the caller), device-detected
+ *     problems are recorded there as by fb_device_status; if NULL they go unreported.
+ * Not thread-safe. */
+#define FB_STATIC_MAX_EXPERTS 256
+fb_status fb_predict_load_static(const fb_config* cfg, int device, const fb_router* router,
+                                 const void* x, int32_t T, uint32_t* counts, int32_t* topk_ids,
+                                 int32_t* status_word, fb_stream stream);
+
 /* Synchronises `stream`, returns the device status word in *word (FB_OK, or the
  * first FB_ERR_BAD_PLACEMENT / FB_ERR_TIMEOUT / FB_ERR_RANGE raised since the last
  * query) and clears it. */

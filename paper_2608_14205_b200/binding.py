@@ -48,7 +48,7 @@ FB_ERR_RANGE = 6
 
 EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_predict_load",
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
-           "fb_device_status", "fb_launch_count", "fb_status_string"]
+           "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static"]
 
 _lib = None
 
@@ -85,6 +85,9 @@ def lib() -> ctypes.CDLL:
     L.fb_route_dispatch.argtypes = [vp, ctypes.POINTER(FbRouter), vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.fb_layer_step_host.argtypes = [vp, ctypes.POINTER(FbRouter), vp, vp, i32, vp, ctypes.POINTER(FbBudget), i32] \
         + [vp] * 14
+    L.fb_predict_load_static.argtypes = [ctypes.POINTER(FbConfig), ctypes.c_int, ctypes.POINTER(FbRouter), vp, i32,
+                                         vp, vp, vp, vp]
+    L.fb_predict_load_static.restype = ctypes.c_int
     L.fb_device_status.argtypes = [vp, ctypes.POINTER(i32), vp]
     L.fb_launch_count.argtypes = [vp]
     L.fb_launch_count.restype = u64
@@ -145,6 +148,14 @@ def fb_budget_ns(t_attn_ns: int, delta_ns: int) -> int:
 
 def fb_swap_cost_ns(budget: FbBudget, rank_a: int, rank_b: int) -> int:
     return int(lib().fb_swap_cost_ns(ctypes.byref(budget), rank_a, rank_b))
+
+
+def fb_predict_load_static(cfg: FbConfig, device: int, router: FbRouter, x, T: int, counts, topk_ids=None,
+                           status_word=None, stream=None) -> None:
+    """Context-free prediction pass that allocates nothing (scratch lives in the library image)."""
+    _check(lib().fb_predict_load_static(ctypes.byref(cfg), device, ctypes.byref(router), _ptr(x), T, _ptr(counts),
+                                        _ptr(topk_ids), _ptr(status_word), _stream(stream)),
+           "fb_predict_load_static")
 
 
 class Context:

@@ -498,3 +498,101 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream_) {
 uint64_t fb_launch_count(const fb_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------
+// fb_predict_load_static: the prediction pass for callers that must not allocate.
+// Its scratch (the cross-block histogram, the finished-block ticket and a status word)
+// lives in a fixed array inside the library image instead of in an fb_ctx.
+// ---------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticScratchWords = FB_STATIC_MAX_EXPERTS + 64;
+constexpr int kStaticMaxDevices = 64;
+
+// Every GPU that loads the library holds this array until the process exits.
+static __device__ __align__(256) uint32_t g_static_scratch[kStaticScratchWords];
+
+struct StaticState {
+  bool ready = false;
+  uint32_t* scratch = nullptr;      // device address of g_static_scratch on this device
+  fb_ctx ctx;                       // host-side launch state only; owns no device memory
+};
+StaticState g_static_state[kStaticMaxDevices];
+
+}  // namespace
+
+extern "C" fb_status fb_predict_load_static(const fb_config* cfg, int device, const fb_router* router,
+                                            const void* x, int32_t T, uint32_t* counts, int32_t* topk_ids,
+                                            int32_t* status_word, fb_stream stream_) {
+  if (!cfg || !router || !router->W || !counts || T < 0) return FB_ERR_INVALID_ARG;
+  if (cfg->E > FB_STATIC_MAX_EXPERTS) return FB_ERR_UNSUPPORTED_SHAPE;   // scratch array too small
+  const fb_status cs = check_config(*cfg);
+  if (cs != FB_OK) return cs;
+  if (T > cfg->T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (T > 0 && !x) return FB_ERR_INVALID_ARG;
+  if (device < 0 || device >= kStaticMaxDevices) return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  StaticState& st = g_static_state[device];
+  if (!st.ready) {
+    // One-time set-up for this device, with the device current.  In host code the name
+    // of a __device__ array is only a handle: the address a kernel can use has to be
+    // asked for.
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess || prop.major != 10) return FB_ERR_CUDA;
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || addr == nullptr) return FB_ERR_CUDA;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr)
+      return FB_ERR_CUDA;
+    st.scratch = static_cast<uint32_t*>(addr);
+    st.ctx.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    st.ctx.device = device;
+    st.ctx.cfg.E = -1;                                   // forces the shape-dependent part below
+    st.ready = true;
+  }
+  fb_ctx& ctx = st.ctx;
+  if (memcmp(&ctx.cfg, cfg, sizeof(fb_config)) != 0) {
+    // shape-dependent launch parameters (host arithmetic and function attributes only)
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FB_ERR_CUDA;
+    ctx.cfg = *cfg;
+    ctx.N = (cfg->E + 15) / 16 * 16;
+    ctx.tmem_cols = next_pow2_at_least_32(ctx.N);
+    const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
+    for (int pair = 0; pair < 2; ++pair) {
+      const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx.N / (pair + 1)) * fb::kBlockK * 2;
+      int stages = static_cast<int>((budget - 1024) / stage_bytes);
+      if (stages > fb::kMaxStages) stages = fb::kMaxStages;
+      size_t dyn = stages * stage_bytes;
+      if (dyn < fb::epilogue_scratch_bytes(ctx.N)) dyn = fb::epilogue_scratch_bytes(ctx.N);
+      if (stages < 2 || dyn + 1024 > budget) {
+        if (pair == 0) { ctx.cfg.E = -1; return FB_ERR_UNSUPPORTED_SHAPE; }
+        stages = 0;
+      }
+      ctx.stages[pair] = stages;
+      ctx.smem_bytes[pair] = dyn + 1024;
+    }
+    bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   static_cast<int>(ctx.smem_bytes[0])) == cudaSuccess;
+    if (ctx.stages[1] >= 2)
+      ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(ctx.smem_bytes[1])) == cudaSuccess;
+    if (!ok) { ctx.cfg.E = -1; return FB_ERR_CUDA; }
+    for (int i = 0; i < kMapCache; ++i) { ctx.x_maps[i] = MapEntry(); ctx.w_maps[i] = MapEntry(); }
+    ctx.max_tiles = (cfg->T_max + fb::kTileM - 1) / fb::kTileM;
+  }
+  ctx.counts_scratch = st.scratch;
+  ctx.ticket = st.scratch + FB_STATIC_MAX_EXPERTS;
+  ctx.status = status_word ? status_word : reinterpret_cast<int32_t*>(st.scratch + FB_STATIC_MAX_EXPERTS + 1);
+  ctx.tile_counts = nullptr;                             // unused by the prediction pass
+  if (T == 0)
+    return cudaMemsetAsync(counts, 0, cfg->E * sizeof(uint32_t), stream) == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+  // The array keeps whatever the previous call (possibly one that was cut short) left in it.
+  if (cudaMemsetAsync(st.scratch, 0, kStaticScratchWords * sizeof(uint32_t), stream) != cudaSuccess)
+    return FB_ERR_CUDA;
+  return launch_router(&ctx, router, x, T, fb::kModePredict, counts, topk_ids, nullptr, nullptr, nullptr, stream);
+}

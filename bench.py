@@ -105,6 +105,21 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """The slowest rank's time decides: MAX all-reduce (identity when not distributed)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(world: int, tokens_per_step: int, steps: int, total_ms: float) -> float:
+    """Replicas process world * tokens per step; the job takes the slowest rank's time."""
+    return world * tokens_per_step * steps / (total_ms * 1e-3)
+
+
 def physical_gpu_index(local_rank: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -261,10 +276,7 @@ def main():
     total_ms = ev[0][0].elapsed_time(ev[K - 1][2])
     predict_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
     dispatch_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(K)]
-    if distributed:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev)
     status = ctx.fb_device_status()
 
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
@@ -289,15 +301,12 @@ def main():
     e1.record()
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), 1e-9)
-    if distributed:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dev)
 
     if rank == 0:
         peaks = measured_peaks()
         ms_per_step = total_ms / K
-        value = world * T * K / (total_ms * 1e-3)
+        value = whole_job_throughput(world, T, K, total_ms)
         # roofline of the dominant kernel (the fused router kernel of fb_predict_and_plan)
         alg_bytes = 2 * T * d + 2 * d * E + 4 * E
         alg_flops = 2 * T * d * E

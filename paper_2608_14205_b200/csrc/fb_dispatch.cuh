@@ -13,7 +13,7 @@
 
 namespace fb {
 
-constexpr int kDispatchThreads = 256;
+constexpr int kDispatchThreads = 1024;   // 4 threads per expert column for the tile sums
 constexpr int kDispatchTile = 128;     // must equal the router kernel's tile height
 
 struct DispatchParams {
@@ -35,9 +35,11 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
   __shared__ int32_t owner[FB_MAX_EXPERTS];
   __shared__ uint32_t before[FB_MAX_EXPERTS];      // assignments to this slot in earlier tiles
   __shared__ uint32_t total[FB_MAX_EXPERTS];       // assignments to this slot in all tiles
+  __shared__ uint32_t part_before[kDispatchThreads / FB_MAX_EXPERTS][FB_MAX_EXPERTS];
+  __shared__ uint32_t part_total[kDispatchThreads / FB_MAX_EXPERTS][FB_MAX_EXPERTS];
   __shared__ uint32_t offs[FB_MAX_EXPERTS + 1];    // exclusive prefix of total over slots
   __shared__ uint32_t mask[FB_MAX_EXPERTS][kDispatchTile / 32];
-  __shared__ uint32_t warp_sum[kDispatchThreads / 32];
+  __shared__ uint32_t warp_sum[FB_MAX_EXPERTS / 32];
   __shared__ int32_t bad;
 
   const int t = threadIdx.x;
@@ -61,18 +63,37 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
     if (t == 0 && tile == 0) atomicCAS(p.status, 0, FB_ERR_BAD_PLACEMENT);
     return;
   }
-  // column sums of the per-tile histogram, split at this tile
-  for (int e = t; e < E; e += kDispatchThreads) {
+  // Column sums of the per-tile histogram, split at this tile.  The loop is bound by L2
+  // latency, so each column is shared by 4 threads and the loads are issued 32 at a time.
+  {
+    constexpr int kParts = kDispatchThreads / FB_MAX_EXPERTS;
+    const int e = t % FB_MAX_EXPERTS, part = t / FB_MAX_EXPERTS;
     uint32_t bef = 0, tot = 0;
-    const uint32_t* col = p.tile_counts + e;
-#pragma unroll 8
-    for (int tt = 0; tt < p.num_tiles; ++tt) {
-      const uint32_t c = col[static_cast<size_t>(tt) * E];
-      tot += c;
-      if (tt < tile) bef += c;
+    if (e < E) {
+      const int per = (p.num_tiles + kParts - 1) / kParts;
+      const int t0 = part * per, t1 = min(p.num_tiles, t0 + per);
+      const uint32_t* col = p.tile_counts + e;
+      for (int base = t0; base < t1; base += 32) {
+        uint32_t c[32];
+#pragma unroll
+        for (int u = 0; u < 32; ++u) c[u] = (base + u < t1) ? __ldg(col + static_cast<size_t>(base + u) * E) : 0u;
+#pragma unroll
+        for (int u = 0; u < 32; ++u) {
+          tot += c[u];
+          if (base + u < tile) bef += c[u];
+        }
+      }
     }
-    before[slot_of[e]] = bef;
-    total[slot_of[e]] = tot;
+    part_before[part][e] = bef;
+    part_total[part][e] = tot;
+    __syncthreads();
+    if (part == 0 && e < E) {
+      uint32_t b = 0, a = 0;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) { b += part_before[q][e]; a += part_total[q][e]; }
+      before[slot_of[e]] = b;
+      total[slot_of[e]] = a;
+    }
   }
   __syncthreads();
   // exclusive scan of total[] over slots (thread s owns slot s)
@@ -84,12 +105,14 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
       const uint32_t o = __shfl_up_sync(0xffffffffu, incl, off);
       if ((t & 31) >= off) incl += o;
     }
-    if ((t & 31) == 31) warp_sum[t >> 5] = incl;
+    if (t < FB_MAX_EXPERTS && (t & 31) == 31) warp_sum[t >> 5] = incl;
     __syncthreads();
-    uint32_t base = 0;
-    for (int w = 0; w < (t >> 5); ++w) base += warp_sum[w];
-    if (t < E) offs[t] = base + incl - v;
-    if (t == E - 1) offs[E] = base + incl;
+    if (t < FB_MAX_EXPERTS) {
+      uint32_t base = 0;
+      for (int w = 0; w < (t >> 5); ++w) base += warp_sum[w];
+      if (t < E) offs[t] = base + incl - v;
+      if (t == E - 1) offs[E] = base + incl;
+    }
   }
   __syncthreads();
   if (tile == 0) {
@@ -98,39 +121,29 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
     for (int r = t; r <= p.R; r += kDispatchThreads) p.rank_offsets[r] = offs[r * m];
     for (int r = t; r < p.R; r += kDispatchThreads) p.rank_load[r] = offs[(r + 1) * m] - offs[r * m];
   }
-  // rank of each assignment among the rows of this tile that go to the same slot
-  const long long i = static_cast<long long>(tile) * kDispatchTile + t;
-  const bool active = t < kDispatchTile && i < p.T;
-  int32_t my_slot[FB_MAX_TOPK];
-#pragma unroll
-  for (int j = 0; j < FB_MAX_TOPK; ++j) my_slot[j] = 0;
+  // Rank of each assignment among the rows of this tile that go to the same slot.
+  // Thread (row, j) = (t % 128, t / 128) owns assignment j of the tile's row.
+  static_assert(kDispatchThreads == kDispatchTile * FB_MAX_TOPK, "one thread per assignment of a tile");
+  const int row = t % kDispatchTile, j = t / kDispatchTile;
+  const long long i = static_cast<long long>(tile) * kDispatchTile + row;
+  const bool active = j < k && i < p.T;
+  int my_slot = 0;
   if (active) {
-#pragma unroll
-    for (int j = 0; j < FB_MAX_TOPK; ++j) {
-      if (j < k) {
-        int e = p.topk_ids[i * k + j];
-        e = (e < 0 || e >= E) ? 0 : e;
-        my_slot[j] = slot_of[e];
-        atomicOr(&mask[my_slot[j]][t >> 5], 1u << (t & 31));
-      }
-    }
+    int e = p.topk_ids[i * k + j];
+    e = (e < 0 || e >= E) ? 0 : e;
+    my_slot = slot_of[e];
+    atomicOr(&mask[my_slot][row >> 5], 1u << (row & 31));
   }
   __syncthreads();
   if (active) {
     const long long n_assign = static_cast<long long>(p.T) * k;
-#pragma unroll
-    for (int j = 0; j < FB_MAX_TOPK; ++j) {
-      if (j < k) {
-        const int s = my_slot[j];
-        uint32_t ahead = __popc(mask[s][t >> 5] & ((1u << (t & 31)) - 1u));
-        for (int w = 0; w < (t >> 5); ++w) ahead += __popc(mask[s][w]);
-        const long long pos = static_cast<long long>(offs[s]) + before[s] + ahead;
-        const long long flat = i * k + j;
-        if (pos < n_assign) {
-          p.perm[pos] = static_cast<int32_t>(flat);
-          p.inv_perm[flat] = static_cast<int32_t>(pos);
-        }
-      }
+    uint32_t ahead = __popc(mask[my_slot][row >> 5] & ((1u << (row & 31)) - 1u));
+    for (int w = 0; w < (row >> 5); ++w) ahead += __popc(mask[my_slot][w]);
+    const long long pos = static_cast<long long>(offs[my_slot]) + before[my_slot] + ahead;
+    const long long flat = i * k + j;
+    if (pos < n_assign) {
+      p.perm[pos] = static_cast<int32_t>(flat);
+      p.inv_perm[flat] = static_cast<int32_t>(pos);
     }
   }
 }

@@ -274,7 +274,7 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   ctx->cfg = *cfg;
   ctx->device = device;
   ctx->N = (cfg->E + 15) / 16 * 16;
-  ctx->tmem_cols = next_pow2_at_least_32(ctx->N);
+  ctx->tmem_cols = next_pow2_at_least_32(2 * ctx->N)   /* two accumulators */;
   const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
   for (int pair = 0; pair < 2; ++pair) {
     const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N / (pair + 1)) * fb::kBlockK * 2;
@@ -561,7 +561,7 @@ extern "C" fb_status fb_predict_load_static(const fb_config* cfg, int device, co
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FB_ERR_CUDA;
     ctx.cfg = *cfg;
     ctx.N = (cfg->E + 15) / 16 * 16;
-    ctx.tmem_cols = next_pow2_at_least_32(ctx.N);
+    ctx.tmem_cols = next_pow2_at_least_32(2 * ctx.N);
     const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
     for (int pair = 0; pair < 2; ++pair) {
       const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx.N / (pair + 1)) * fb::kBlockK * 2;

@@ -4,8 +4,14 @@
 // finishes last publishes the count vector and, when asked, runs the swap planner.
 //
 // One block owns 128 token rows and all N = pad16(E) expert columns.
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the TMEM allocation),
-// warps 2..17 = epilogue.  A warp may only read the 32 TMEM lanes (token rows) selected
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer for the even k-blocks (owns the
+// TMEM allocation), warp 18 = MMA issuer for the odd k-blocks, warps 2..17 = epilogue.
+// A thread that issues tcgen05.mma gets the next one accepted only ~175 cycles later,
+// whatever the MMA's shape, which is slower than the tensor pipe and than the x stream
+// from HBM; two issuing threads, each accumulating its own k-blocks into its own TMEM
+// accumulator (columns [0, N) and [N, 2N)), remove that limit and keep the summation
+// order fixed.  The epilogue adds the two accumulators.
+// Epilogue warps:  A warp may only read the 32 TMEM lanes (token rows) selected
 // by warp_id % 4, so the 16 epilogue warps form 4 "row quarters" x 4 "subs"; the subs of
 // a quarter split the expert columns between them in 32-column chunks, one thread per
 // token row, and sub 0 merges the partial results.
@@ -35,7 +41,8 @@ constexpr int kUmmaK = 16;             // K of one tcgen05.mma for 16-bit inputs
 constexpr int kMaxStages = 8;
 constexpr int kEpiSubs = 4;            // epilogue warps per row quarter
 constexpr int kEpilogueThreads = 128 * kEpiSubs;
-constexpr int kRouterThreads = 64 + kEpilogueThreads;
+constexpr int kRouterThreads = 64 + kEpilogueThreads + 32;
+constexpr int kSecondIssuerWarp = kRouterThreads / 32 - 1;
 constexpr int kATileBytes = kTileM * kBlockK * 2;
 constexpr uint32_t kAccumBarrierId = 2;      // named barrier: accumulator finished (MMA warp -> epilogue warps)
 
@@ -51,7 +58,7 @@ struct RouterParams {
   float route_scale;
   int32_t num_kb;                    // ceil(d / 64)
   int32_t stages;
-  int32_t tmem_cols;                 // power of two >= max(32, N)
+  int32_t tmem_cols;                 // power of two >= max(32, 2 N): two accumulators
   int32_t mode;
   const float* logit_bias;           // [E] or nullptr
   const float* select_bias;          // [E] or nullptr
@@ -187,7 +194,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       mbar_init(smem_u32(&sh.full_bar[s]), 1);
       mbar_init(smem_u32(&sh.empty_bar[s]), 1);
     }
-    mbar_init(smem_u32(&sh.accum_bar), 1);
+    mbar_init(smem_u32(&sh.accum_bar), 2);                 // one commit per MMA issuer
     fence_mbar_init();
     prefetch_tensormap(&tmap_x);
     prefetch_tensormap(&tmap_w);
@@ -238,12 +245,16 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 || warp == kSecondIssuerWarp) {
+    // ------------------------------------------------------------ MMA issuers
+    // warp 1: k-blocks 0, 2, 4, ... into accumulator 0; the last warp: 1, 3, 5, ... into
+    // accumulator 1 (N columns further).  In a pair only the even block issues.
     if (lane == 0 && cta_rank == 0) {
+      const int first_kb = warp == 1 ? 0 : 1;
+      const uint32_t acc = tmem_base + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
       const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.N));
       bool ok = true;
-      for (int kb = 0; kb < p.num_kb && ok; ++kb) {
+      for (int kb = first_kb; kb < p.num_kb && ok; kb += 2) {
         const int s = kb % p.stages;
         const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
         ok = mbar_wait<kCtas == 2>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
@@ -255,21 +266,23 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 #pragma unroll
         for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
           // advance 16 elements = 32 bytes inside the swizzled row: +2 in the address field
-          umma_bf16<kCtas>(tmem_base, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          umma_bf16<kCtas>(acc, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb != first_kb || kk != 0) ? 1u : 0u);
         }
         // frees the stage (in both blocks of a pair) when these MMAs retire
         if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.empty_bar[s]));
         else umma_commit_2cta(smem_u32(&sh.empty_bar[s]), 0x3);
       }
-      // accumulator complete
+      // this issuer's accumulator is complete
       if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.accum_bar));
       else umma_commit_2cta(smem_u32(&sh.accum_bar), 0x3);
     }
+    if (warp == 1) {
     // One thread polls for the finished accumulator on behalf of the 16 epilogue warps,
     // which sleep at a hardware barrier meanwhile (no issue slots, no power).
     if (lane == 0) sh.accum_ok = mbar_wait<kCtas == 2>(smem_u32(&sh.accum_bar), 0u, abort_flag) ? 1 : 0;
     __syncwarp();
     named_bar_arrive(kAccumBarrierId, kEpilogueThreads + 32);
+    }
   } else {
     // ------------------------------------------------------------ epilogue
     const int et = threadIdx.x - 64;                       // 0 .. kEpilogueThreads-1
@@ -321,6 +334,21 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         uint32_t r[32];
         float q[32];
         load_chunk(taddr, c0, N, r);
+        if (p.num_kb > 1) {                                  // add the odd k-blocks' accumulator
+          const int halves = (N - c0 >= 32) ? 2 : 1;         // 16 columns at a time keeps registers low
+          for (int h = 0; h < halves; ++h) {
+            uint32_t r2[32];
+            tmem_ld_32x32b_x16(taddr + N + c0 + 16 * h, r2);
+            tmem_ld_wait();
+            if (h == 0) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) r[16 + j] = __float_as_uint(__uint_as_float(r[16 + j]) + __uint_as_float(r2[j]));
+            }
+          }
+        }
         if (p.logits != nullptr && valid) {
 #pragma unroll
           for (int j = 0; j < 32; ++j)

@@ -44,6 +44,9 @@ struct PlanShared {
   int32_t slot_of[FB_MAX_EXPERTS];       // expert -> slot (current placement)
   int32_t expert_at[FB_MAX_EXPERTS];     // slot -> expert
   uint8_t moved[FB_MAX_EXPERTS];
+  uint32_t slot_cnt[FB_MAX_EXPERTS];     // fast loop: count of the expert in each slot, bit 31 = already moved
+  uint8_t cand_a[FB_MAX_EXPERTS];        // fast loop: candidate c pairs slot c / m of the heavy rank ...
+  uint8_t cand_b[FB_MAX_EXPERTS];        // ... with slot c % m of the light rank
   uint32_t load[FB_MAX_RANKS];
   unsigned long long rank_spent[FB_MAX_RANKS];
   uint32_t link_key[FB_MAX_EXPERTS / 2]; // one entry per accepted swap
@@ -84,10 +87,121 @@ __device__ __forceinline__ void plan_load_placement(const PlanParams& p, PlanSha
     if (s < 0 || s >= p.E) sh.bad = 1;
     else if (atomicExch(&sh.expert_at[s], e) != -1) sh.bad = 1;
   }
+  const int m = p.E / p.R;
+  for (int c = t; c < FB_MAX_EXPERTS; c += nthreads) {
+    sh.cand_a[c] = static_cast<uint8_t>(c / m);
+    sh.cand_b[c] = static_cast<uint8_t>(c % m);
+  }
 }
 __device__ __forceinline__ void plan_clear(PlanShared& sh, int t, int nthreads) {
   if (t == 0) sh.bad = 0;
   for (int e = t; e < FB_MAX_EXPERTS; e += nthreads) sh.expert_at[e] = -1;
+}
+
+// Greedy loop specialised for the common case: one cost per link class (no per-expert
+// size table) and at most 256 candidate pairs per iteration (m <= 16), so every lane owns
+// at most 8 fixed (slot, slot) pairs.  Same decisions as the general loop below; the
+// arithmetic is kept in 32-bit registers where the ranges allow (loads < 2^22).
+// L0 / L1: this lane's rank loads (ranks lane and lane + 32, -1 if absent).
+__device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanShared& sh, int lane,
+                                                      int& L0, int& L1) {
+  const int R = p.R, m = p.E / R, mm = m * m;
+  const uint32_t full = 0xffffffffu;
+  int cand_sa[8], cand_sb[8];                                   // slot offsets inside the two ranks
+#pragma unroll
+  for (int t = 0; t < 8; ++t) { cand_sa[t] = sh.cand_a[lane + 32 * t]; cand_sb[t] = sh.cand_b[lane + 32 * t]; }
+  const uint32_t gden = p.gamma_den ? p.gamma_den : 1u;
+  const uint32_t gnum2 = p.gamma_den ? 2u * p.gamma_num : 0u;   // <= 2^21
+  const int rpn = p.ranks_per_node;
+  unsigned long long global_spent = 0;
+  uint32_t n = 0;
+  __syncwarp();
+  while (n < p.max_swaps) {
+    // frontier (lowest index on ties): max of load<<6 | (63 - rank), min of load<<6 | rank
+    const uint32_t h0 = L0 >= 0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(63 - lane)) : 0u;
+    const uint32_t h1 = L1 >= 0 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(31 - lane)) : 0u;
+    const uint32_t l0 = L0 >= 0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(lane)) : 0xffffffffu;
+    const uint32_t l1 = L1 >= 0 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(lane + 32)) : 0xffffffffu;
+    const uint32_t hi_key = __reduce_max_sync(full, h0 > h1 ? h0 : h1);
+    const uint32_t lo_key = __reduce_min_sync(full, l0 < l1 ? l0 : l1);
+    const int a = 63 - static_cast<int>(hi_key & 63u), b = static_cast<int>(lo_key & 63u);
+    const int La = static_cast<int>(hi_key >> 6), Lb = static_cast<int>(lo_key >> 6);
+    const int D = La - Lb;
+    if (static_cast<uint32_t>(D) <= p.tau_tokens) break;
+    int m2l = 0;
+    if (lane != a && lane != b && L0 > m2l) m2l = L0;
+    if (lane + 32 != a && lane + 32 != b && L1 > m2l) m2l = L1;
+    const int M2 = static_cast<int>(__reduce_max_sync(full, static_cast<uint32_t>(m2l)));
+    // budgets: the cost is the same for every pair of this iteration
+    const int cls = (rpn <= 0 || a / rpn == b / rpn) ? 0 : 1;
+    const unsigned long long c_ns = p.uniform_cost_ns[cls];
+    const int lo = a < b ? a : b, hi = a < b ? b : a;
+    const uint32_t lkey = cls == 0 ? (static_cast<uint32_t>(lo) << 8 | static_cast<uint32_t>(hi))
+                                   : (0x10000u | static_cast<uint32_t>(lo / rpn) << 8 | static_cast<uint32_t>(hi / rpn));
+    const unsigned long long rs_a = sh.rank_spent[a], rs_b = sh.rank_spent[b];
+    if (p.global_ns != FB_BUDGET_OFF && (c_ns > p.global_ns || global_spent > p.global_ns - c_ns)) break;
+    if (p.rank_ns != FB_BUDGET_OFF) {
+      const unsigned long long rs = rs_a > rs_b ? rs_a : rs_b;
+      if (c_ns > p.rank_ns || rs > p.rank_ns - c_ns) break;
+    }
+    if (p.link_ns != FB_BUDGET_OFF) {
+      unsigned long long link_spent = 0;
+      for (uint32_t i = 0; i < n; ++i)
+        if (sh.link_key[i] == lkey) link_spent += sh.link_cost[i];
+      if (c_ns > p.link_ns || link_spent > p.link_ns - c_ns) break;
+    }
+    // candidates of this lane
+    long long best_ben = 0;
+    uint32_t best_pair = 0xffffffffu;
+    const int base_a = a * m, base_b = b * m;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if (lane + 32 * t < mm) {
+        const int sa = base_a + cand_sa[t], sb = base_b + cand_sb[t];
+        const uint32_t ca = sh.slot_cnt[sa], cb = sh.slot_cnt[sb];
+        const uint32_t pair = static_cast<uint32_t>(sh.expert_at[sa]) << 16 | static_cast<uint32_t>(sh.expert_at[sb]);
+        if (((ca | cb) >> 31) == 0) {                             // neither expert moved yet
+          const int dlt = static_cast<int>(ca) - static_cast<int>(cb);   // tokens moved a -> b
+          int Mn = La - dlt;                                      // Eq. 6
+          if (Lb + dlt > Mn) Mn = Lb + dlt;                       // Eq. 7
+          if (M2 > Mn) Mn = M2;
+          // gamma_den * (Phi(L) - Phi(L')), variance term 2 dlt (La - Lb - dlt)
+          const long long ben = static_cast<long long>(gden) * (La - Mn) +
+                                static_cast<long long>(gnum2) * (static_cast<long long>(dlt) * (D - dlt));
+          if (ben > best_ben || (ben == best_ben && ben > 0 && pair < best_pair)) { best_ben = ben; best_pair = pair; }
+        }
+      }
+    }
+    // largest benefit, ties -> smallest (expert on a, expert on b)
+    const unsigned long long ben = static_cast<unsigned long long>(best_ben);
+    const uint32_t top_hi = __reduce_max_sync(full, static_cast<uint32_t>(ben >> 32));
+    const uint32_t top_lo = __reduce_max_sync(full, static_cast<uint32_t>(ben >> 32) == top_hi ? static_cast<uint32_t>(ben) : 0u);
+    const unsigned long long top_ben = static_cast<unsigned long long>(top_hi) << 32 | top_lo;
+    if (top_ben == 0) break;                                      // Algorithm 1 lines 6-7
+    const uint32_t win = __reduce_min_sync(full, ben == top_ben ? best_pair : 0xffffffffu);
+    const int ea = static_cast<int>(win >> 16), eb = static_cast<int>(win & 0xffffu);
+    const int sa = sh.slot_of[ea], sb = sh.slot_of[eb];
+    const int dlt = static_cast<int>(sh.slot_cnt[sa]) - static_cast<int>(sh.slot_cnt[sb]);
+    __syncwarp();                                                 // all lanes are done reading the tables
+    if (lane == 0) {
+      const uint32_t ca = sh.slot_cnt[sa], cb = sh.slot_cnt[sb];
+      sh.slot_cnt[sa] = cb | 0x80000000u; sh.slot_cnt[sb] = ca | 0x80000000u;
+      sh.slot_of[ea] = sb; sh.slot_of[eb] = sa;
+      sh.expert_at[sa] = eb; sh.expert_at[sb] = ea;
+      sh.rank_spent[a] = rs_a + c_ns; sh.rank_spent[b] = rs_b + c_ns;
+      sh.link_key[n] = lkey; sh.link_cost[n] = c_ns;
+      fb_swap sw; sw.src_rank = a; sw.dst_rank = b; sw.expert_src = ea; sw.expert_dst = eb;
+      p.swaps[n] = sw;
+    }
+    if (lane == a) L0 -= dlt;
+    if (lane + 32 == a) L1 -= dlt;
+    if (lane == b) L0 += dlt;
+    if (lane + 32 == b) L1 += dlt;
+    global_spent += c_ns;
+    ++n;
+    __syncwarp();
+  }
+  return n;
 }
 
 // The greedy loop, run by ONE warp (all 32 lanes) once sh.cnt holds the count vector and
@@ -98,9 +212,13 @@ __device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh
   const int E = p.E, R = p.R, m = E / R;
   const uint32_t full = 0xffffffffu;
   __syncwarp();
-  unsigned long long total = 0;
-  for (int e = lane; e < E; e += 32) total += sh.cnt[e];
-  for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(full, total, off);
+  // counts per slot, and their sum (clamped per lane so that 32 lanes cannot overflow)
+  unsigned long long mine = 0;
+  if (!sh.bad)
+    for (int sl = lane; sl < E; sl += 32) { const uint32_t c = sh.cnt[sh.expert_at[sl]]; sh.slot_cnt[sl] = c; mine += c; }
+  const uint32_t clamped = mine > (1u << 22) ? (1u << 22) : static_cast<uint32_t>(mine);
+  const uint32_t total = __reduce_add_sync(full, clamped);
+  __syncwarp();
   int bad = sh.bad;
   if (!bad && total > FB_MAX_COUNT_SUM) bad = 2;
   if (bad) {
@@ -117,19 +235,29 @@ __device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh
   long long L0 = -1, L1 = -1;                  // -1 marks "no such rank"
   if (lane < R) {
     uint32_t s0 = 0;
-    for (int j = 0; j < m; ++j) s0 += sh.cnt[sh.expert_at[lane * m + j]];
+    for (int j = 0; j < m; ++j) s0 += sh.slot_cnt[lane * m + j];
     L0 = s0;
     p.load_before[lane] = s0;
+    sh.rank_spent[lane] = 0;
   }
   if (lane + 32 < R) {
     uint32_t s1 = 0;
-    for (int j = 0; j < m; ++j) s1 += sh.cnt[sh.expert_at[(lane + 32) * m + j]];
+    for (int j = 0; j < m; ++j) s1 += sh.slot_cnt[(lane + 32) * m + j];
     L1 = s1;
     p.load_before[lane + 32] = s1;
+    sh.rank_spent[lane + 32] = 0;
   }
-  if (lane == 0) { for (int r = 0; r < R; ++r) sh.rank_spent[r] = 0; }
   __syncwarp();
 
+  if (p.expert_bytes_table == nullptr && m <= 16) {
+    int l0 = static_cast<int>(L0), l1 = static_cast<int>(L1);
+    const uint32_t n_fast = plan_loop_uniform(p, sh, lane, l0, l1);
+    if (lane == 0) *p.n_swaps = static_cast<int32_t>(n_fast);
+    for (int e = lane; e < E; e += 32) p.expert_to_slot_out[e] = sh.slot_of[e];
+    if (lane < R) p.load_after[lane] = static_cast<uint32_t>(l0);
+    if (lane + 32 < R) p.load_after[lane + 32] = static_cast<uint32_t>(l1);
+    return;
+  }
   const long long gnum = p.gamma_den ? p.gamma_num : 0;
   const long long gden = p.gamma_den ? p.gamma_den : 1;
   const int rpn = p.ranks_per_node;

@@ -304,6 +304,18 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const bool fast_select = sigmoid_gate && gs == 32 && p.n_group <= 8 && p.topk_group <= kEpiSubs &&
                              p.topk_group * 2 >= k;
 
+    // Chunk bookkeeping, worked out while the main loop runs (integer divisions by run-time
+    // values are slow and would otherwise sit between the chunks of the epilogue):
+    // which chunks this warp owns, which of them end a group, and each chunk's group.
+    uint32_t owned_chunks = 0, group_end_chunks = 0, chunk_group = 0;     // bit c / nibble c
+    for (int c = 0; c < n_chunks; ++c) {
+      const int owner = splittable ? (c / chunks_per_group) % kEpiSubs : 0;
+      if (owner == sub) owned_chunks |= 1u << c;
+      if (sigmoid_gate && gs % 32 == 0) {
+        if ((c * 32 + 32) % gs == 0) group_end_chunks |= 1u << c;
+        chunk_group |= static_cast<uint32_t>((c * 32) / gs) << (4 * c);   // at most 8 groups here
+      }
+    }
     // While the main loop runs, stage the placement for the planner (any block may turn
     // out to be the last one).
     if (p.mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
@@ -328,8 +340,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       // ---------------- pass 1
       float m1 = -INFINITY, m2 = -INFINITY;
       for (int c = 0; c < n_chunks; ++c) {
-        const int owner = splittable ? (c / chunks_per_group) % kEpiSubs : 0;
-        if (owner != sub) continue;
+        if (((owned_chunks >> c) & 1u) == 0) continue;
         const int c0 = c * 32;
         uint32_t r[32];
         float q[32];
@@ -411,8 +422,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           }
           m2 = fmaxf(fminf(m1, a1[0]), fmaxf(m2, a2[0]));
           m1 = fmaxf(m1, a1[0]);
-          if ((c0 + 32) % gs == 0) {                          // last chunk of the group
-            const int g = c0 / gs;
+          if ((group_end_chunks >> c) & 1u) {                 // last chunk of the group
+            const int g = static_cast<int>((chunk_group >> (4 * c)) & 15u);
             gscore_s[g * kTileM + row_in_tile] = m1 + m2;
             glow_s[g * kTileM + row_in_tile] = m2;
             m1 = -INFINITY; m2 = -INFINITY;
@@ -597,8 +608,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
       // ---------------- pass 2
       for (int c = 0; c < n_chunks; ++c) {
-        const int owner = splittable ? (c / chunks_per_group) % kEpiSubs : 0;
-        if (owner != sub) continue;
+        if (((owned_chunks >> c) & 1u) == 0) continue;
         const int c0 = c * 32;
         int g = sigmoid_gate ? c0 / gs : 0, pos = sigmoid_gate ? c0 % gs : 0;
         const int g_start = g, pos_start = pos;

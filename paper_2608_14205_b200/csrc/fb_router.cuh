@@ -460,8 +460,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       for (int g = 0; g < 8; ++g) {
         int rank = 0;
 #pragma unroll
-        for (int h = 0; h < 8; ++h)
-          if (h != g) rank += (sc[h] > sc[g] || (sc[h] == sc[g] && h < g)) ? 1 : 0;
+        for (int h = 0; h < 8; ++h)          // a lower-numbered group wins ties
+          if (h != g) rank += (h < g ? sc[h] >= sc[g] : sc[h] > sc[g]) ? 1 : 0;
         if (g < p.n_group && rank < p.topk_group) {
           floor_key = fminf(floor_key, glow_s[g * kTileM + row_in_tile]);
           if (rank == sub) my_group = g;
@@ -571,7 +571,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             int rank = 0;
 #pragma unroll
             for (int h = 0; h < 8; ++h)
-              if (h != g) rank += (sc[h] > sc[g] || (sc[h] == sc[g] && h < g)) ? 1 : 0;
+              if (h != g) rank += (h < g ? sc[h] >= sc[g] : sc[h] > sc[g]) ? 1 : 0;
             if (g < p.n_group && rank < p.topk_group) {
               for (int j = 0; j < 32; ++j) {
                 const float x = key_s[(g * 32 + j) * kTileM + row_in_tile];
@@ -738,9 +738,11 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const uint32_t c = sh.hist[e];
         if (c) atomicAdd(&p.counts_scratch[e], c);
       }
-      __threadfence();
       named_bar_sync(kPlanBarrierId, kEpilogueThreads);
       if (et == 0) {
+        // The barrier orders every thread's histogram atomics before this fence, and the
+        // fence (cumulative) publishes them device-wide before the ticket is taken.
+        __threadfence();
         const uint32_t prev = atomicAdd(p.ticket, 1u);
         sh.is_last = (prev == gridDim.x - 1) ? 1 : 0;
       }

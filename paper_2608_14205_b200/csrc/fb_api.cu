@@ -44,6 +44,7 @@ struct fb_ctx {
   uint32_t* ticket = nullptr;           // [1],   zero between calls
   int32_t* status = nullptr;            // [1]
   uint32_t* tile_counts = nullptr;      // [max_tiles][E]
+  uint32_t* super_counts = nullptr;     // [ceil(max_tiles / 32)][E]
   // descriptor cache
   MapEntry x_maps[kMapCache];
   MapEntry w_maps[kMapCache];
@@ -306,7 +307,9 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
                                     static_cast<int>(ctx->smem_bytes[1])) == cudaSuccess;
   ok = ok && dev_alloc(&ctx->counts_scratch, FB_MAX_EXPERTS) && dev_alloc(&ctx->ticket, 1) &&
        dev_alloc(&ctx->status, 1) &&
-       dev_alloc(&ctx->tile_counts, static_cast<size_t>(ctx->max_tiles) * cfg->E);
+       dev_alloc(&ctx->tile_counts, static_cast<size_t>(ctx->max_tiles) * cfg->E) &&
+       dev_alloc(&ctx->super_counts,
+                 static_cast<size_t>((ctx->max_tiles + fb::kSuperTiles - 1) / fb::kSuperTiles) * cfg->E);
   ok = ok && cudaMemset(ctx->counts_scratch, 0, FB_MAX_EXPERTS * sizeof(uint32_t)) == cudaSuccess &&
        cudaMemset(ctx->ticket, 0, sizeof(uint32_t)) == cudaSuccess &&
        cudaMemset(ctx->status, 0, sizeof(int32_t)) == cudaSuccess;
@@ -319,7 +322,7 @@ fb_status fb_destroy(fb_ctx* ctx) {
   if (!ctx) return FB_OK;
   DeviceGuard guard(ctx->device);
   cudaDeviceSynchronize();
-  void* ptrs[] = {ctx->counts_scratch, ctx->ticket, ctx->status, ctx->tile_counts, ctx->st_hprev, ctx->st_H,
+  void* ptrs[] = {ctx->counts_scratch, ctx->ticket, ctx->status, ctx->tile_counts, ctx->super_counts, ctx->st_hprev, ctx->st_H,
                   ctx->st_pi, ctx->st_pi_out, ctx->st_counts, ctx->st_swaps, ctx->st_nswaps, ctx->st_load_before,
                   ctx->st_load_after, ctx->st_ids, ctx->st_w, ctx->st_slot_offsets, ctx->st_rank_offsets,
                   ctx->st_perm, ctx->st_inv_perm, ctx->st_rank_load};
@@ -407,6 +410,15 @@ fb_status fb_route_dispatch(fb_ctx* ctx, const fb_router* router, const void* x,
   dp.num_tiles = (T + fb::kDispatchTile - 1) / fb::kDispatchTile;
   dp.topk_ids = topk_ids;
   dp.tile_counts = ctx->tile_counts;
+  dp.super_counts = nullptr;
+  if (dp.num_tiles > 4 * fb::kSuperTiles) {                 // beyond 16k tokens the two-level sums pay off
+    const int n_super = (dp.num_tiles + fb::kSuperTiles - 1) / fb::kSuperTiles;
+    fb::fb_tile_sums_kernel<<<n_super, FB_MAX_EXPERTS, 0, stream>>>(ctx->tile_counts, ctx->super_counts,
+                                                                     dp.num_tiles, c.E);
+    ++ctx->launches;
+    if (cudaGetLastError() != cudaSuccess) return FB_ERR_CUDA;
+    dp.super_counts = ctx->super_counts;
+  }
   dp.expert_to_slot = expert_to_slot;
   dp.slot_offsets = slot_offsets;
   dp.rank_offsets = rank_offsets;

@@ -15,11 +15,13 @@ namespace fb {
 
 constexpr int kDispatchThreads = 1024;   // 4 threads per expert column for the tile sums
 constexpr int kDispatchTile = 128;     // must equal the router kernel's tile height
+constexpr int kSuperTiles = 32;        // tiles per super-block of the two-level tile sums
 
 struct DispatchParams {
   int32_t T, k, E, R, num_tiles;
   const int32_t* topk_ids;         // [T][k]
   const uint32_t* tile_counts;     // [num_tiles][E]
+  const uint32_t* super_counts;    // [ceil(num_tiles / 32)][E] sums over 32 tiles, or nullptr (few tiles)
   const int32_t* expert_to_slot;   // [E]
   uint32_t* slot_offsets;          // [E+1]
   uint32_t* rank_offsets;          // [R+1]
@@ -69,7 +71,19 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
     constexpr int kParts = kDispatchThreads / FB_MAX_EXPERTS;
     const int e = t % FB_MAX_EXPERTS, part = t / FB_MAX_EXPERTS;
     uint32_t bef = 0, tot = 0;
-    if (e < E) {
+    if (e < E && p.super_counts != nullptr) {
+      // many tiles: whole super-blocks come pre-summed, only this tile's own super-block is walked
+      const int n_super = (p.num_tiles + kSuperTiles - 1) / kSuperTiles;
+      const int my_super = tile / kSuperTiles;
+      for (int sb = part; sb < n_super; sb += kParts) {
+        const uint32_t c = __ldg(p.super_counts + static_cast<size_t>(sb) * E + e);
+        tot += c;
+        if (sb < my_super) bef += c;
+      }
+      const uint32_t* col = p.tile_counts + e;
+      for (int tt = my_super * kSuperTiles + part; tt < tile; tt += kParts)
+        bef += __ldg(col + static_cast<size_t>(tt) * E);
+    } else if (e < E) {
       const int per = (p.num_tiles + kParts - 1) / kParts;
       const int t0 = part * per, t1 = min(p.num_tiles, t0 + per);
       const uint32_t* col = p.tile_counts + e;
@@ -146,6 +160,23 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
       p.inv_perm[flat] = static_cast<int32_t>(pos);
     }
   }
+}
+
+// Sums of the per-tile histograms over super-blocks of 32 tiles (only launched when there
+// are many tiles, so that the dispatch kernel's blocks need not each walk all of them).
+__global__ void __launch_bounds__(FB_MAX_EXPERTS)
+fb_tile_sums_kernel(const uint32_t* __restrict__ tile_counts, uint32_t* __restrict__ super_counts,
+                    int num_tiles, int E) {
+  const int e = threadIdx.x, sb = blockIdx.x;
+  if (e >= E) return;
+  const int t0 = sb * kSuperTiles, t1 = min(num_tiles, t0 + kSuperTiles);
+  uint32_t c[kSuperTiles];
+#pragma unroll
+  for (int u = 0; u < kSuperTiles; ++u) c[u] = (t0 + u < t1) ? tile_counts[static_cast<size_t>(t0 + u) * E + e] : 0u;
+  uint32_t s = 0;
+#pragma unroll
+  for (int u = 0; u < kSuperTiles; ++u) s += c[u];
+  super_counts[static_cast<size_t>(sb) * E + e] = s;
 }
 
 }  // namespace fb

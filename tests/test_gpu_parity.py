@@ -286,3 +286,36 @@ def test_long_prefill_sweep_sampled(name):
 def test_mid_configs_full_size(name):
     wl = I.WORKLOADS[name]
     _run(wl, wl.T, layer=0, want_logits=False)
+
+
+# ------------------------------------------------------------------ more layers, drifts and budgets
+@pytest.mark.parametrize("layer", [19, 38, 57])
+def test_dsv3_spread_layers(layer):
+    rep, gpu = _run(I.WORKLOADS["dsv3"], 4096, layer=layer, want_logits=False)
+    assert rep["n_swaps"] <= 5
+
+
+@pytest.mark.parametrize("rho,cap", [(0.05, 0), (0.2, 2), (0.4, 10)])
+def test_sweep_shape_drift_and_budget(rho, cap):
+    wl = dataclasses.replace(I.WORKLOADS["sweep32k"], rho=rho, max_swaps=cap)
+    rep, gpu = _run(wl, 3000, layer=1, want_logits=False)
+    assert rep["n_swaps"] <= cap
+    if cap == 0:
+        assert gpu["pi_out"] == list(range(wl.E))          # empty plan keeps the placement
+
+
+def test_planner_is_identical_on_every_replay():
+    # every rank replays the planner on the same counts: R runs must give one plan
+    wl = I.WORKLOADS["dsv3"]
+    counts = I.random_counts(wl.E, 100_000, seed=11, zipf_s=1.1).to(torch.int32)
+    ctx = B.Context(128, 64, wl.E, 1, wl.R)
+    dev = torch.device("cuda")
+    bud = B.make_budget(**P.budget_kwargs(wl, 12_500))
+    seen = set()
+    for _ in range(wl.R):
+        z = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
+        out_pi, swaps, n, lb, la = z(wl.E), z(4 * 128), z(1), z(wl.R), z(wl.R)
+        ctx.fb_plan_swaps(counts.to(dev), torch.arange(wl.E, dtype=torch.int32, device=dev), bud, 3, out_pi, swaps, n,
+                          lb, la)
+        seen.add((tuple(out_pi.cpu().tolist()), tuple(swaps.cpu().tolist()[:4 * int(n.item())]), tuple(la.cpu().tolist())))
+    assert len(seen) == 1

@@ -113,10 +113,18 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
   const uint32_t gden = p.gamma_den ? p.gamma_den : 1u;
   const uint32_t gnum2 = p.gamma_den ? 2u * p.gamma_num : 0u;   // <= 2^21
   const int rpn = p.ranks_per_node;
+  // loop invariants in registers (no run-time indexing of the parameter block inside the loop)
+  const unsigned long long cost0 = p.uniform_cost_ns[0], cost1 = p.uniform_cost_ns[1];
+  const unsigned long long global_ns = p.global_ns, rank_ns = p.rank_ns, link_ns = p.link_ns;
+  const bool global_on = global_ns != FB_BUDGET_OFF, rank_on = rank_ns != FB_BUDGET_OFF, link_on = link_ns != FB_BUDGET_OFF;
+  // A link is only ever charged one cost (its class's), so its budget is a swap count.
+  const unsigned long long link_cap0 = link_ns / cost0, link_cap1 = link_ns / cost1;
+  const uint32_t max_swaps = p.max_swaps, tau = p.tau_tokens;
+  uint32_t my_links[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};   // lane i keeps the links of swaps i, i+32, ...
   unsigned long long global_spent = 0;
   uint32_t n = 0;
   __syncwarp();
-  while (n < p.max_swaps) {
+  while (n < max_swaps) {
     // frontier (lowest index on ties): max of load<<6 | (63 - rank), min of load<<6 | rank
     const uint32_t h0 = L0 >= 0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(63 - lane)) : 0u;
     const uint32_t h1 = L1 >= 0 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(31 - lane)) : 0u;
@@ -127,28 +135,28 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
     const int a = 63 - static_cast<int>(hi_key & 63u), b = static_cast<int>(lo_key & 63u);
     const int La = static_cast<int>(hi_key >> 6), Lb = static_cast<int>(lo_key >> 6);
     const int D = La - Lb;
-    if (static_cast<uint32_t>(D) <= p.tau_tokens) break;
+    if (static_cast<uint32_t>(D) <= tau) break;
     int m2l = 0;
     if (lane != a && lane != b && L0 > m2l) m2l = L0;
     if (lane + 32 != a && lane + 32 != b && L1 > m2l) m2l = L1;
     const int M2 = static_cast<int>(__reduce_max_sync(full, static_cast<uint32_t>(m2l)));
     // budgets: the cost is the same for every pair of this iteration
     const int cls = (rpn <= 0 || a / rpn == b / rpn) ? 0 : 1;
-    const unsigned long long c_ns = p.uniform_cost_ns[cls];
+    const unsigned long long c_ns = cls ? cost1 : cost0;
     const int lo = a < b ? a : b, hi = a < b ? b : a;
     const uint32_t lkey = cls == 0 ? (static_cast<uint32_t>(lo) << 8 | static_cast<uint32_t>(hi))
                                    : (0x10000u | static_cast<uint32_t>(lo / rpn) << 8 | static_cast<uint32_t>(hi / rpn));
     const unsigned long long rs_a = sh.rank_spent[a], rs_b = sh.rank_spent[b];
-    if (p.global_ns != FB_BUDGET_OFF && (c_ns > p.global_ns || global_spent > p.global_ns - c_ns)) break;
-    if (p.rank_ns != FB_BUDGET_OFF) {
+    if (global_on && (c_ns > global_ns || global_spent > global_ns - c_ns)) break;
+    if (rank_on) {
       const unsigned long long rs = rs_a > rs_b ? rs_a : rs_b;
-      if (c_ns > p.rank_ns || rs > p.rank_ns - c_ns) break;
+      if (c_ns > rank_ns || rs > rank_ns - c_ns) break;
     }
-    if (p.link_ns != FB_BUDGET_OFF) {
-      unsigned long long link_spent = 0;
-      for (uint32_t i = 0; i < n; ++i)
-        if (sh.link_key[i] == lkey) link_spent += sh.link_cost[i];
-      if (c_ns > p.link_ns || link_spent > p.link_ns - c_ns) break;
+    if (link_on) {
+      uint32_t used = 0;                                         // swaps already charged to this link
+#pragma unroll
+      for (int q = 0; q < 4; ++q) used += __popc(__ballot_sync(full, my_links[q] == lkey));
+      if (used >= (cls ? link_cap1 : link_cap0)) break;
     }
     // candidates of this lane
     long long best_ben = 0;
@@ -189,7 +197,6 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
       sh.slot_of[ea] = sb; sh.slot_of[eb] = sa;
       sh.expert_at[sa] = eb; sh.expert_at[sb] = ea;
       sh.rank_spent[a] = rs_a + c_ns; sh.rank_spent[b] = rs_b + c_ns;
-      sh.link_key[n] = lkey; sh.link_cost[n] = c_ns;
       fb_swap sw; sw.src_rank = a; sw.dst_rank = b; sw.expert_src = ea; sw.expert_dst = eb;
       p.swaps[n] = sw;
     }
@@ -197,6 +204,10 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
     if (lane + 32 == a) L1 -= dlt;
     if (lane == b) L0 += dlt;
     if (lane + 32 == b) L1 += dlt;
+    if (static_cast<int>(n & 31u) == lane) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) if (static_cast<int>(n >> 5) == q) my_links[q] = lkey;
+    }
     global_spent += c_ns;
     ++n;
     __syncwarp();

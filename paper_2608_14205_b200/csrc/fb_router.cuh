@@ -129,20 +129,6 @@ __host__ __device__ constexpr size_t epilogue_scratch_bytes(int N) {
 
 static_assert(2 * kCandCap >= 2 * (kEpiSubs - 1) * FB_MAX_TOPK + kEpiSubs * 2, "merge area must fit in the candidate area");
 
-// Same value with the reciprocal computed on the FMA pipe: a bit-trick first guess
-// (12% off) refined by three Newton steps to ~1e-7 relative error.  The argument of the
-// reciprocal is 1 + 2^x in [1, 2^116] thanks to the clamp, far from overflow.
-__device__ __forceinline__ float fb_sigmoid_fma(float z) {
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaxf(z, -80.0f) * -1.4426950408889634f));
-  const float y = 1.0f + e;
-  float r = __int_as_float(0x7EF311C7 - __float_as_int(y));
-  r = r * (2.0f - y * r);
-  r = r * (2.0f - y * r);
-  r = r * (2.0f - y * r);
-  return r;
-}
-
 struct RouterShared {
   uint64_t full_bar[kMaxStages];
   uint64_t empty_bar[kMaxStages];
@@ -299,10 +285,14 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int n_chunks = (N + 31) >> 5;
     const int chunks_per_group = (sigmoid_gate && gs % 32 == 0) ? gs / 32 : 1;
     const bool splittable = !sigmoid_gate || gs % 32 == 0 || 32 % gs == 0;
-    // DeepSeek-V3-like gate (groups of exactly one chunk, few groups kept): selection by
-    // ranking a short candidate list instead of insertion.
-    const bool fast_select = sigmoid_gate && gs == 32 && p.n_group <= 8 && p.topk_group <= kEpiSubs &&
-                             p.topk_group * 2 >= k;
+    const bool want_sum = p.topk_w != nullptr && !p.renorm && !sigmoid_gate;
+    // Selection by ranking a short candidate list instead of insertion.  Applies to
+    // DeepSeek-V3-like gates (groups of exactly one chunk, few groups kept) and to softmax
+    // gates over whole chunks, where every chunk counts as a kept group; needs at least k
+    // known keys (two per kept group) for the lower bound of the k-th key.
+    const bool fast_select =
+        sigmoid_gate ? (gs == 32 && p.n_group <= 8 && p.topk_group <= kEpiSubs && p.topk_group * 2 >= k)
+                     : (E % 32 == 0 && n_chunks <= 8 && n_chunks * 2 >= k && !want_sum);
 
     // Chunk bookkeeping, worked out while the main loop runs (integer divisions by run-time
     // values are slow and would otherwise sit between the chunks of the epilogue):
@@ -335,7 +325,6 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     top.init();
     float sm_max = -INFINITY, sm_sum = 0.0f;               // softmax denominator (weights without renorm)
     const bool has_lb = p.logit_bias != nullptr;
-    const bool want_sum = p.topk_w != nullptr && !p.renorm && !sigmoid_gate;
     if (got) {
       // ---------------- pass 1
       float m1 = -INFINITY, m2 = -INFINITY;
@@ -367,17 +356,17 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
               p.logits[row * E + c0 + j] = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
         }
         if (sigmoid_gate && c0 + 32 <= E && !has_lb) {
-          // whole chunk valid, no logit bias (the common case).  The sigmoid needs two
-          // special-function results per key and that unit is the bottleneck here, so
-          // every other key gets its reciprocal from Newton steps on the FMA pipe instead.
+          // whole chunk valid, no logit bias (the common case).  Every key goes through the
+          // same two hardware approximations, so equal logits give equal keys in every column
+          // (an FMA-pipe reciprocal on alternate columns was no faster and broke exact ties).
           const float4* sb4 = reinterpret_cast<const float4*>(&sh.select_bias[c0]);
 #pragma unroll
           for (int j4 = 0; j4 < 8; ++j4) {
             const float4 b = sb4[j4];
             q[4 * j4 + 0] = fb_sigmoid(__uint_as_float(r[4 * j4 + 0])) + b.x;
-            q[4 * j4 + 1] = fb_sigmoid_fma(__uint_as_float(r[4 * j4 + 1])) + b.y;
+            q[4 * j4 + 1] = fb_sigmoid(__uint_as_float(r[4 * j4 + 1])) + b.y;
             q[4 * j4 + 2] = fb_sigmoid(__uint_as_float(r[4 * j4 + 2])) + b.z;
-            q[4 * j4 + 3] = fb_sigmoid_fma(__uint_as_float(r[4 * j4 + 3])) + b.w;
+            q[4 * j4 + 3] = fb_sigmoid(__uint_as_float(r[4 * j4 + 3])) + b.w;
           }
         } else if (sigmoid_gate) {
 #pragma unroll
@@ -428,6 +417,21 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             glow_s[g * kTileM + row_in_tile] = m2;
             m1 = -INFINITY; m2 = -INFINITY;
           }
+        } else if (!sigmoid_gate && fast_select) {
+          // softmax gate, fast selection: the chunk's second-best key is what the bound needs
+          float a1[16], a2[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) { a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); }
+#pragma unroll
+          for (int w = 8; w >= 1; w >>= 1) {
+#pragma unroll
+            for (int j = 0; j < w; ++j) {
+              const float hi = fmaxf(a1[j], a1[j + w]);
+              a2[j] = fmaxf(fminf(a1[j], a1[j + w]), fmaxf(a2[j], a2[j + w]));
+              a1[j] = hi;
+            }
+          }
+          glow_s[c * kTileM + row_in_tile] = a2[0];
         } else if (sigmoid_gate) {
           int g = c0 / gs, pos = c0 % gs;
 #pragma unroll
@@ -451,26 +455,34 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       // ---------------- choose: rank the (at most 8) group scores of this row
       uint32_t* cand_hi = reinterpret_cast<uint32_t*>(merge_v);             // [kCandCap][128] ordered key bits
       uint32_t* cand_lo = cand_hi + kCandCap * kTileM;                       // [kCandCap][128] ~expert id
-      float sc[8];
-#pragma unroll
-      for (int g = 0; g < 8; ++g) sc[g] = g < p.n_group ? gscore_s[g * kTileM + row_in_tile] : -INFINITY;
-      int my_group = -1;
+      int my_groups[2] = {-1, -1};                        // the 32-column groups this sub scans
       float floor_key = INFINITY;
+      if (sigmoid_gate) {
+        float sc[8];
 #pragma unroll
-      for (int g = 0; g < 8; ++g) {
-        int rank = 0;
+        for (int g = 0; g < 8; ++g) sc[g] = g < p.n_group ? gscore_s[g * kTileM + row_in_tile] : -INFINITY;
 #pragma unroll
-        for (int h = 0; h < 8; ++h)          // a lower-numbered group wins ties
-          if (h != g) rank += (h < g ? sc[h] >= sc[g] : sc[h] > sc[g]) ? 1 : 0;
-        if (g < p.n_group && rank < p.topk_group) {
-          floor_key = fminf(floor_key, glow_s[g * kTileM + row_in_tile]);
-          if (rank == sub) my_group = g;
+        for (int g = 0; g < 8; ++g) {
+          int rank = 0;
+#pragma unroll
+          for (int h = 0; h < 8; ++h)          // a lower-numbered group wins ties
+            if (h != g) rank += (h < g ? sc[h] >= sc[g] : sc[h] > sc[g]) ? 1 : 0;
+          if (g < p.n_group && rank < p.topk_group) {
+            floor_key = fminf(floor_key, glow_s[g * kTileM + row_in_tile]);
+            if (rank == sub) my_groups[0] = g;   // sub s scans the row's s-th best group
+          }
         }
+      } else {
+        for (int c = 0; c < n_chunks; ++c) floor_key = fminf(floor_key, glow_s[c * kTileM + row_in_tile]);
+        if (sub < n_chunks) my_groups[0] = sub;
+        if (sub + kEpiSubs < n_chunks) my_groups[1] = sub + kEpiSubs;
       }
-      // ---------------- collect: sub s scans the row's s-th best group for keys >= floor
-      // (the kept groups' two best keys are >= floor, so at least k keys qualify)
-      if (sub < p.topk_group) {
-        const int base = my_group * 32;
+      // ---------------- collect the keys >= floor (the kept groups' two best keys are >= floor,
+      // so at least k keys qualify)
+#pragma unroll 1
+      for (int gi = 0; gi < 2; ++gi) {
+        if (my_groups[gi] < 0) continue;                  // no such group: true for the whole warp at once
+        const int base = my_groups[gi] * 32;              // (which group may differ from row to row)
         uint32_t mask = 0;
 #pragma unroll
         for (int j = 0; j < 32; ++j)
@@ -550,7 +562,13 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       if (__any_sync(0xffffffffu, overflow)) {
         // More than kCandCap keys reached the floor (many equal keys): plain scan of the
         // kept groups for the rows concerned.
-        if (overflow) {
+        if (overflow && !sigmoid_gate) {
+          top.init();
+          for (int e = 0; e < E; ++e) {
+            const float x = key_s[e * kTileM + row_in_tile];
+            if (x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+          }
+        } else if (overflow) {
           float sc[8];
 #pragma unroll
           for (int g = 0; g < 8; ++g) sc[g] = -INFINITY;

@@ -319,3 +319,22 @@ def test_planner_is_identical_on_every_replay():
                           lb, la)
         seen.add((tuple(out_pi.cpu().tolist()), tuple(swaps.cpu().tolist()[:4 * int(n.item())]), tuple(la.cpu().tolist())))
     assert len(seen) == 1
+
+
+@pytest.mark.parametrize("name", ["qwen3", "dsv3"])
+def test_all_equal_keys_take_the_overflow_path(name):
+    # all logits equal: every key reaches the selection bound, the short candidate list
+    # overflows and the plain scan must still pick the lowest ids (lowest groups first)
+    wl = I.WORKLOADS[name]
+    T = 300
+    li = I.make_layer(wl, 0, 0, T=T)
+    li.W = torch.zeros_like(li.W)
+    if li.select_bias is not None:
+        li.select_bias = torch.zeros(wl.E)
+    ctx = P.make_context(wl, T)
+    bkw = P.budget_kwargs(wl, T)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw)
+    assert gpu["status"] == 0
+    assert (gpu["ids"] == np.arange(wl.k)).all() and (gpu["ids_early"] == np.arange(wl.k)).all()
+    assert gpu["counts"].tolist() == [T] * wl.k + [0] * (wl.E - wl.k)
+    P.compare_layer(wl, li, bkw, gpu)

@@ -338,3 +338,29 @@ def test_all_equal_keys_take_the_overflow_path(name):
     assert (gpu["ids"] == np.arange(wl.k)).all() and (gpu["ids_early"] == np.arange(wl.k)).all()
     assert gpu["counts"].tolist() == [T] * wl.k + [0] * (wl.E - wl.k)
     P.compare_layer(wl, li, bkw, gpu)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_shapes(seed):
+    rng = np.random.default_rng(1000 + seed)
+    gate = int(rng.integers(0, 2))
+    if gate:
+        n_group = int(rng.choice([1, 2, 4, 8]))
+        gs = int(rng.choice([1, 2, 4, 8, 16, 32]))
+        E = n_group * gs
+        if E > 256 or E < 2:
+            E, n_group, gs = 64, 8, 8
+        topk_group = int(rng.integers(1, min(n_group, 8) + 1))
+        k = int(rng.integers(1, min(8, topk_group * gs) + 1))
+    else:
+        E = int(rng.choice([2, 8, 24, 32, 64, 96, 128, 160, 256]))
+        n_group = topk_group = 1
+        k = int(rng.integers(1, min(8, E) + 1))
+    divisors = [r for r in (1, 2, 4, 8, 16, 32, 64) if E % r == 0]
+    R = int(rng.choice(divisors))
+    d = int(rng.choice([8, 64, 200, 512, 1096]))
+    T = int(rng.choice([1, 77, 128, 129, 300, 640]))
+    wl = I.Workload(name="fuzz", T=T, d=d, E=E, k=k, R=R, layers=1, gate=gate, n_group=n_group,
+                    topk_group=topk_group, renorm=int(rng.integers(0, 2)), route_scale=float(rng.choice([1.0, 2.5])),
+                    rho=0.2, skew="zipf", zipf_s=1.0, max_swaps=int(rng.integers(0, E // 2 + 1)))
+    _run(wl, T, layer=seed, with_logit_bias=bool(rng.integers(0, 2)))

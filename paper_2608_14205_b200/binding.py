@@ -48,7 +48,7 @@ FB_ERR_RANGE = 6
 
 EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_predict_load",
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
-           "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static"]
+           "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step"]
 
 _lib = None
 
@@ -83,6 +83,9 @@ def lib() -> ctypes.CDLL:
     L.fb_predict_and_plan.argtypes = [vp, ctypes.POINTER(FbRouter), vp, i32, vp, ctypes.POINTER(FbBudget), i32,
                                       vp, vp, vp, vp, vp, vp, vp]
     L.fb_route_dispatch.argtypes = [vp, ctypes.POINTER(FbRouter), vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.fb_layer_step.argtypes = [vp, ctypes.POINTER(FbRouter), vp, vp, i32, vp, ctypes.POINTER(FbBudget), i32] \
+        + [vp] * 14
+    L.fb_layer_step.restype = ctypes.c_int
     L.fb_layer_step_host.argtypes = [vp, ctypes.POINTER(FbRouter), vp, vp, i32, vp, ctypes.POINTER(FbBudget), i32] \
         + [vp] * 14
     L.fb_predict_load_static.argtypes = [ctypes.POINTER(FbConfig), ctypes.c_int, ctypes.POINTER(FbRouter), vp, i32,
@@ -202,6 +205,15 @@ class Context:
                                        _ptr(topk_ids), _ptr(topk_w), _ptr(slot_offsets), _ptr(rank_offsets),
                                        _ptr(perm), _ptr(inv_perm), _ptr(rank_load), _ptr(logits),
                                        _stream(stream)), "fb_route_dispatch")
+
+    def fb_layer_step(self, router, h_prev, H, T, expert_to_slot, budget, layer_id, counts, expert_to_slot_out,
+                      swaps, n_swaps, load_before, load_after, topk_ids, topk_w, slot_offsets, rank_offsets, perm,
+                      inv_perm, rank_load, stream=None):
+        outs = [counts, expert_to_slot_out, swaps, n_swaps, load_before, load_after, topk_ids, topk_w,
+                slot_offsets, rank_offsets, perm, inv_perm, rank_load]
+        _check(lib().fb_layer_step(self._h, ctypes.byref(router), _ptr(h_prev), _ptr(H), T, _ptr(expert_to_slot),
+                                   ctypes.byref(budget), layer_id, *[_ptr(o) for o in outs], _stream(stream)),
+               "fb_layer_step")
 
     def fb_layer_step_host(self, router, h_prev_host, H_host, T, expert_to_slot_host, budget, layer_id,
                            counts=None, expert_to_slot_out=None, swaps=None, n_swaps=None, load_before=None,

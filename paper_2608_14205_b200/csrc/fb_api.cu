@@ -162,12 +162,20 @@ fb_status fill_plan(const fb_ctx* ctx, const fb_budget* b, const int32_t* pi, in
 }
 
 // Launch the router kernel in one of its three modes.
+// x2 is the second input of kModeLayer (the normal router input), nullptr otherwise.
 fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T, int mode,
                         uint32_t* counts_out, int32_t* topk_ids, float* topk_w, float* logits,
-                        const fb::PlanParams* plan, cudaStream_t stream) {
-  const CUtensorMap *mx = nullptr, *mw = nullptr;
+                        const fb::PlanParams* plan, cudaStream_t stream, const void* x2 = nullptr) {
+  const CUtensorMap *mx = nullptr, *mx2 = nullptr, *mw = nullptr;
   fb_status st = make_map(ctx, ctx->x_maps, &ctx->x_next, x, T, fb::kTileM, &mx);
   if (st != FB_OK) return st;
+  const CUtensorMap map_x = *mx;     // by value: the second lookup may evict the cache slot mx points to
+  mx = &map_x;
+  mx2 = mx;
+  if (mode == fb::kModeLayer) {
+    st = make_map(ctx, ctx->x_maps, &ctx->x_next, x2, T, fb::kTileM, &mx2);
+    if (st != FB_OK) return st;
+  }
   const int tiles = (T + fb::kTileM - 1) / fb::kTileM;
   const int pair = (tiles > 1 && ctx->stages[1] >= 2) ? 1 : 0;   // a single tile gains nothing from a partner
   st = make_map(ctx, ctx->w_maps, &ctx->w_next, router->W, ctx->cfg.E,
@@ -195,6 +203,10 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.logits = logits;
   p.tile_counts = ctx->tile_counts;
   if (plan) p.plan = *plan;
+  const int tiles_pad = pair ? (tiles + 1) / 2 * 2 : tiles;       // a pair never straddles the two passes
+  const int blocks = mode == fb::kModeLayer ? 2 * tiles_pad : tiles_pad;
+  p.tiles_first = tiles_pad;
+  p.ticket_target = tiles_pad;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.blockDim = dim3(fb::kRouterThreads, 1, 1);
@@ -203,20 +215,51 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   cudaLaunchAttribute attr[1];
   cudaError_t err;
   if (pair) {
-    cfg.gridDim = dim3(static_cast<unsigned>((tiles + 1) / 2 * 2), 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mw, p);
+    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mx2, *mw, p);
   } else {
-    cfg.gridDim = dim3(static_cast<unsigned>(tiles), 1, 1);
-    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1>, *mx, *mw, p);
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1>, *mx, *mx2, *mw, p);
   }
   ++ctx->launches;
   return err == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+// Dispatch index from the router kernel's top-k ids and per-tile histograms.
+fb_status launch_dispatch_index(fb_ctx* ctx, int32_t T, const int32_t* expert_to_slot, const int32_t* topk_ids,
+                                uint32_t* slot_offsets, uint32_t* rank_offsets, int32_t* perm, int32_t* inv_perm,
+                                uint32_t* rank_load, cudaStream_t stream) {
+  const fb_config& c = ctx->cfg;
+  fb::DispatchParams dp;
+  dp.T = T; dp.k = c.k; dp.E = c.E; dp.R = c.R;
+  dp.num_tiles = (T + fb::kDispatchTile - 1) / fb::kDispatchTile;
+  dp.topk_ids = topk_ids;
+  dp.tile_counts = ctx->tile_counts;
+  dp.super_counts = nullptr;
+  if (dp.num_tiles > 4 * fb::kSuperTiles) {                 // beyond 16k tokens the two-level sums pay off
+    const int n_super = (dp.num_tiles + fb::kSuperTiles - 1) / fb::kSuperTiles;
+    fb::fb_tile_sums_kernel<<<n_super, FB_MAX_EXPERTS, 0, stream>>>(ctx->tile_counts, ctx->super_counts,
+                                                                     dp.num_tiles, c.E);
+    ++ctx->launches;
+    if (cudaGetLastError() != cudaSuccess) return FB_ERR_CUDA;
+    dp.super_counts = ctx->super_counts;
+  }
+  dp.expert_to_slot = expert_to_slot;
+  dp.slot_offsets = slot_offsets;
+  dp.rank_offsets = rank_offsets;
+  dp.perm = perm;
+  dp.inv_perm = inv_perm;
+  dp.rank_load = rank_load;
+  dp.status = ctx->status;
+  fb::fb_dispatch_kernel<<<dp.num_tiles, fb::kDispatchThreads, 0, stream>>>(dp);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
 }
 
 fb_status launch_plan(fb_ctx* ctx, const fb::PlanParams& pp, const uint32_t* counts, cudaStream_t stream) {
@@ -405,30 +448,41 @@ fb_status fb_route_dispatch(fb_ctx* ctx, const fb_router* router, const void* x,
   const fb_status st = launch_router(ctx, router, x, T, fb::kModeDispatch, nullptr, topk_ids, topk_w, logits,
                                      nullptr, stream);
   if (st != FB_OK) return st;
-  fb::DispatchParams dp;
-  dp.T = T; dp.k = c.k; dp.E = c.E; dp.R = c.R;
-  dp.num_tiles = (T + fb::kDispatchTile - 1) / fb::kDispatchTile;
-  dp.topk_ids = topk_ids;
-  dp.tile_counts = ctx->tile_counts;
-  dp.super_counts = nullptr;
-  if (dp.num_tiles > 4 * fb::kSuperTiles) {                 // beyond 16k tokens the two-level sums pay off
-    const int n_super = (dp.num_tiles + fb::kSuperTiles - 1) / fb::kSuperTiles;
-    fb::fb_tile_sums_kernel<<<n_super, FB_MAX_EXPERTS, 0, stream>>>(ctx->tile_counts, ctx->super_counts,
-                                                                     dp.num_tiles, c.E);
-    ++ctx->launches;
-    if (cudaGetLastError() != cudaSuccess) return FB_ERR_CUDA;
-    dp.super_counts = ctx->super_counts;
+  return launch_dispatch_index(ctx, T, expert_to_slot, topk_ids, slot_offsets, rank_offsets, perm, inv_perm,
+                               rank_load, stream);
+}
+
+fb_status fb_layer_step(fb_ctx* ctx, const fb_router* router, const void* h_prev, const void* H, int32_t T,
+                        const int32_t* expert_to_slot, const fb_budget* budget, int32_t layer_id,
+                        uint32_t* counts, int32_t* expert_to_slot_out, fb_swap* swaps, int32_t* n_swaps,
+                        uint32_t* load_before, uint32_t* load_after, int32_t* topk_ids, float* topk_w,
+                        uint32_t* slot_offsets, uint32_t* rank_offsets, int32_t* perm, int32_t* inv_perm,
+                        uint32_t* rank_load, fb_stream stream_) {
+  (void)layer_id;
+  if (!ctx || !router || !router->W || !counts || !slot_offsets || !rank_offsets || !rank_load || T < 0)
+    return FB_ERR_INVALID_ARG;
+  if (T > ctx->cfg.T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (T > 0 && (!h_prev || !H || !topk_ids || !topk_w || !perm || !inv_perm)) return FB_ERR_INVALID_ARG;
+  if (T == 0) {
+    const fb_status st0 = fb_predict_and_plan(ctx, router, h_prev, 0, expert_to_slot, budget, layer_id, counts,
+                                              expert_to_slot_out, swaps, n_swaps, load_before, load_after, stream_);
+    if (st0 != FB_OK) return st0;
+    return fb_route_dispatch(ctx, router, H, 0, expert_to_slot_out, topk_ids, topk_w, slot_offsets, rank_offsets,
+                             perm, inv_perm, rank_load, nullptr, stream_);
   }
-  dp.expert_to_slot = expert_to_slot;
-  dp.slot_offsets = slot_offsets;
-  dp.rank_offsets = rank_offsets;
-  dp.perm = perm;
-  dp.inv_perm = inv_perm;
-  dp.rank_load = rank_load;
-  dp.status = ctx->status;
-  fb::fb_dispatch_kernel<<<dp.num_tiles, fb::kDispatchThreads, 0, stream>>>(dp);
-  ++ctx->launches;
-  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+  fb::PlanParams pp;
+  memset(&pp, 0, sizeof(pp));
+  fb_status st = fill_plan(ctx, budget, expert_to_slot, expert_to_slot_out, swaps, n_swaps, load_before, load_after,
+                           &pp);
+  if (st != FB_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  // one launch for both router passes; the dispatch index needs the new placement and follows
+  st = launch_router(ctx, router, h_prev, T, fb::kModeLayer, counts, topk_ids, topk_w, nullptr, &pp, stream, H);
+  if (st != FB_OK) return st;
+  return launch_dispatch_index(ctx, T, expert_to_slot_out, topk_ids, slot_offsets, rank_offsets, perm, inv_perm,
+                               rank_load, stream);
 }
 
 fb_status fb_layer_step_host(fb_ctx* ctx, const fb_router* router, const void* h_prev_host, const void* H_host,
@@ -469,12 +523,11 @@ fb_status fb_layer_step_host(fb_ctx* ctx, const fb_router* router, const void* h
   ok = ok && cudaMemcpyAsync(ctx->st_pi, expert_to_slot_host, E * sizeof(int32_t), cudaMemcpyHostToDevice, stream) ==
                  cudaSuccess;
   if (!ok) return FB_ERR_CUDA;
-  fb_status st = fb_predict_and_plan(ctx, router, ctx->st_hprev, T, ctx->st_pi, budget, layer_id, ctx->st_counts,
-                                     ctx->st_pi_out, ctx->st_swaps, ctx->st_nswaps, ctx->st_load_before,
-                                     ctx->st_load_after, stream);
-  if (st != FB_OK) return st;
-  st = fb_route_dispatch(ctx, router, ctx->st_H, T, ctx->st_pi_out, ctx->st_ids, ctx->st_w, ctx->st_slot_offsets,
-                         ctx->st_rank_offsets, ctx->st_perm, ctx->st_inv_perm, ctx->st_rank_load, nullptr, stream);
+  const fb_status st = fb_layer_step(ctx, router, ctx->st_hprev, ctx->st_H, T, ctx->st_pi, budget, layer_id,
+                                     ctx->st_counts, ctx->st_pi_out, ctx->st_swaps, ctx->st_nswaps,
+                                     ctx->st_load_before, ctx->st_load_after, ctx->st_ids, ctx->st_w,
+                                     ctx->st_slot_offsets, ctx->st_rank_offsets, ctx->st_perm, ctx->st_inv_perm,
+                                     ctx->st_rank_load, stream);
   if (st != FB_OK) return st;
   auto back = [&](void* dst, const void* src, size_t bytes) {
     if (dst && bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;

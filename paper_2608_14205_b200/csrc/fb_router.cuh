@@ -49,7 +49,10 @@ constexpr uint32_t kAccumBarrierId = 2;      // named barrier: accumulator finis
 enum RouterMode : int {
   kModePredict = 0,        // histogram -> counts
   kModePredictPlan = 1,    // histogram -> counts -> planner in the last block
-  kModeDispatch = 2        // ids, weights, per-tile histogram for the dispatch index
+  kModeDispatch = 2,       // ids, weights, per-tile histogram for the dispatch index
+  kModeLayer = 3           // one launch for a whole layer: blocks [0, tiles_first) run the early pass
+                           // (mode 1) on the first input, the others the normal pass (mode 2) on
+                           // the second; the second wave of blocks fills the SMs the first frees
 };
 
 struct RouterParams {
@@ -60,6 +63,8 @@ struct RouterParams {
   int32_t stages;
   int32_t tmem_cols;                 // power of two >= max(32, 2 N): two accumulators
   int32_t mode;
+  int32_t tiles_first;               // kModeLayer: blocks below this index (even) belong to the early pass
+  int32_t ticket_target;             // number of blocks that take a ticket (those that publish counts)
   const float* logit_bias;           // [E] or nullptr
   const float* select_bias;          // [E] or nullptr
   uint32_t* counts_scratch;          // [E] zero on entry, zero again on exit
@@ -159,14 +164,21 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32
 // both blocks get their stage-free and accumulator-ready signals from its commits.
 template <int kCtas>
 __global__ void __launch_bounds__(kRouterThreads, 1)
-fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                 const __grid_constant__ RouterParams p) {
+fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x2,
+                 const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ RouterParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ RouterShared sh;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int tile = blockIdx.x;
+  // kModeLayer: which pass this block belongs to, its tile there and its input
+  const bool second_pass = p.mode == kModeLayer && static_cast<int>(blockIdx.x) >= p.tiles_first;
+  const int mode = p.mode == kModeLayer ? (second_pass ? kModeDispatch : kModePredictPlan) : p.mode;
+  const int tile = second_pass ? static_cast<int>(blockIdx.x) - p.tiles_first : static_cast<int>(blockIdx.x);
+  const CUtensorMap* xmap = second_pass ? &tmap_x2 : &tmap_x;
+  // outputs of the normal pass are not written by blocks of the early pass
+  int32_t* const out_ids = (p.mode == kModeLayer && !second_pass) ? nullptr : p.topk_ids;
+  float* const out_w = (p.mode == kModeLayer && !second_pass) ? nullptr : p.topk_w;
   const uint32_t cta_rank = kCtas == 2 ? cluster_ctarank() : 0u;
   const uint32_t b_tile_bytes = static_cast<uint32_t>(p.N / kCtas) * kBlockK * 2;
   const uint32_t stage_bytes = kATileBytes + b_tile_bytes;
@@ -182,7 +194,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
     mbar_init(smem_u32(&sh.accum_bar), 2);                 // one commit per MMA issuer
     fence_mbar_init();
-    prefetch_tensormap(&tmap_x);
+    prefetch_tensormap(xmap);
     prefetch_tensormap(&tmap_w);
   }
   if (warp == 1) {
@@ -197,7 +209,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
       sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
     }
-    if (p.mode == kModePredictPlan) plan_clear(sh.plan, et, kEpilogueThreads);
+    if (mode == kModePredictPlan) plan_clear(sh.plan, et, kEpilogueThreads);
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -218,14 +230,14 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (kCtas == 1) {
           const uint32_t full = smem_u32(&sh.full_bar[s]);
           mbar_arrive_expect_tx(full, stage_bytes);
-          tma_load_2d(a_dst, &tmap_x, full, kb * kBlockK, tile * kTileM, pol_x);
+          tma_load_2d(a_dst, xmap, full, kb * kBlockK, tile * kTileM, pol_x);
           tma_load_2d(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK, 0, pol_w);
         } else {
           // both blocks report their bytes to the even block's barrier, which expects
           // the bytes of the whole pair
           const uint32_t full = map_to_cta(smem_u32(&sh.full_bar[s]), 0u);
           if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&sh.full_bar[s]), 2u * stage_bytes);
-          tma_load_2d_pair(a_dst, &tmap_x, full, kb * kBlockK, tile * kTileM, pol_x);
+          tma_load_2d_pair(a_dst, xmap, full, kb * kBlockK, tile * kTileM, pol_x);
           tma_load_2d_pair(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK,
                            static_cast<int32_t>(cta_rank) * (p.N / 2), pol_w);
         }
@@ -285,7 +297,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int n_chunks = (N + 31) >> 5;
     const int chunks_per_group = (sigmoid_gate && gs % 32 == 0) ? gs / 32 : 1;
     const bool splittable = !sigmoid_gate || gs % 32 == 0 || 32 % gs == 0;
-    const bool want_sum = p.topk_w != nullptr && !p.renorm && !sigmoid_gate;
+    const bool want_sum = out_w != nullptr && !p.renorm && !sigmoid_gate;
     // Selection by ranking a short candidate list instead of insertion.  Applies to
     // DeepSeek-V3-like gates (groups of exactly one chunk, few groups kept) and to softmax
     // gates over whole chunks, where every chunk counts as a kept group; needs at least k
@@ -308,7 +320,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
     // While the main loop runs, stage the placement for the planner (any block may turn
     // out to be the last one).
-    if (p.mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
+    if (mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
     named_bar_sync(kAccumBarrierId, kEpilogueThreads + 32);
     const bool got = sh.accum_ok != 0;
     tcgen05_fence_after();
@@ -704,12 +716,12 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 
     // ---- outputs per row
     if (writer) {
-      if (p.topk_ids != nullptr) {
+      if (out_ids != nullptr) {
 #pragma unroll
         for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j < k) p.topk_ids[row * k + j] = top.i[j];
+          if (j < k) out_ids[row * k + j] = top.i[j];
       }
-      if (p.topk_w != nullptr) {
+      if (out_w != nullptr) {
         float w[FB_MAX_TOPK];
         float wsum = 0.0f;
         const float ref = top.v[0];                         // row maximum of the keys
@@ -724,7 +736,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         else scale = p.renorm ? p.route_scale / wsum : p.route_scale;
 #pragma unroll
         for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j < k) p.topk_w[row * k + j] = w[j] * scale;
+          if (j < k) out_w[row * k + j] = w[j] * scale;
       }
     }
     // ---- histogram: one shared-memory atomic per distinct expert per warp (Eq. 5)
@@ -747,7 +759,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
     }
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-    if (p.mode == kModeDispatch) {
+    if (mode == kModeDispatch) {
       if (static_cast<long long>(tile) * kTileM < p.T)       // the padding block of an odd pair owns no tile
         for (int e = et; e < E; e += kEpilogueThreads)
           p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
@@ -762,7 +774,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // fence (cumulative) publishes them device-wide before the ticket is taken.
         __threadfence();
         const uint32_t prev = atomicAdd(p.ticket, 1u);
-        sh.is_last = (prev == gridDim.x - 1) ? 1 : 0;
+        sh.is_last = (prev == static_cast<uint32_t>(p.ticket_target) - 1) ? 1 : 0;
       }
       named_bar_sync(kPlanBarrierId, kEpilogueThreads);
       if (sh.is_last) {
@@ -777,7 +789,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (et == 0) *p.ticket = 0;
         if (sh.abort_flag) { if (et == 0) atomicCAS(p.status, 0, FB_ERR_TIMEOUT); }
         named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-        if (p.mode == kModePredictPlan && warp == 2) plan_swaps_warp(p.plan, sh.plan, lane, p.status);
+        if (mode == kModePredictPlan && warp == 2) plan_swaps_warp(p.plan, sh.plan, lane, p.status);
       }
     }
   }

@@ -85,10 +85,18 @@ def run_gpu_layer(ctx: B.Context, wl: I.Workload, li: I.LayerInputs, bkw: dict, 
     logits = torch.full((max(1, T * E),), float("nan"), device=dev) if want_logits else None
     ctx.fb_route_dispatch(router, H, T, f_pi_out, ids, w, slot_offsets, rank_offsets, perm, inv_perm, rank_load,
                           logits)
+    # the whole layer in one call, into buffers of its own
+    l_counts, l_pi_out, l_swaps, l_n, l_lb, l_la = u32(E), u32(E), u32(4 * ms), u32(1), u32(R), u32(R)
+    l_ids, l_w = u32(max(1, T * k)), torch.full((max(1, T * k),), float("nan"), device=dev)
+    l_so, l_ro, l_rl = u32(E + 1), u32(R + 1), u32(R)
+    l_perm, l_inv = u32(max(1, T * k)), u32(max(1, T * k))
+    ctx.fb_layer_step(router, h_prev, H, T, pi, budget, 0, l_counts, l_pi_out, l_swaps, l_n, l_lb, l_la,
+                      l_ids, l_w, l_so, l_ro, l_perm, l_inv, l_rl)
     status = ctx.fb_device_status()
     torch.cuda.synchronize(dev)
     n = int(n_swaps.item())
     fn = int(f_n.item())
+    ln = int(l_n.item())
     out = dict(
         status=status,
         counts=counts.cpu().numpy().astype(np.int64),
@@ -107,6 +115,17 @@ def run_gpu_layer(ctx: B.Context, wl: I.Workload, li: I.LayerInputs, bkw: dict, 
         rank_offsets=rank_offsets.cpu().numpy().astype(np.int64),
         perm=perm.cpu().numpy()[:T * k].astype(np.int64), inv_perm=inv_perm.cpu().numpy()[:T * k].astype(np.int64),
         rank_load=rank_load.cpu().numpy().astype(np.int64),
+        layer=dict(counts=l_counts.cpu().numpy().astype(np.int64),
+                   swaps=[tuple(r) for r in l_swaps.cpu().numpy().reshape(-1, 4)[:ln].tolist()],
+                   pi_out=l_pi_out.cpu().numpy().tolist(), load_before=l_lb.cpu().numpy().tolist(),
+                   load_after=l_la.cpu().numpy().tolist(),
+                   ids=l_ids.cpu().numpy()[:T * k].reshape(T, k),
+                   w=l_w.cpu().numpy()[:T * k].reshape(T, k).astype(np.float64),
+                   slot_offsets=l_so.cpu().numpy().astype(np.int64),
+                   rank_offsets=l_ro.cpu().numpy().astype(np.int64),
+                   perm=l_perm.cpu().numpy()[:T * k].astype(np.int64),
+                   inv_perm=l_inv.cpu().numpy()[:T * k].astype(np.int64),
+                   rank_load=l_rl.cpu().numpy().astype(np.int64)),
     )
     return out
 
@@ -204,6 +223,17 @@ def compare_layer(wl: I.Workload, li: I.LayerInputs, bkw: dict, gpu: dict, place
     assert gpu["rank_load"].tolist() == rl.tolist()
     assert np.array_equal(gpu["perm"], perm), "perm differs"
     assert np.array_equal(gpu["inv_perm"], inv), "inv_perm differs"
+    # ---- the one-call layer step: the same kernels on the same inputs, so every output is
+    # bit-identical to the separate entry points (which the oracle has just checked)
+    ly = gpu["layer"]
+    assert ly["counts"].tolist() == gpu["counts"].tolist(), "layer step: counts differ"
+    assert ly["swaps"] == swaps and ly["pi_out"] == pi_new, "layer step: plan differs"
+    assert ly["load_before"] == before and ly["load_after"] == after
+    assert np.array_equal(ly["ids"], gpu["ids"]), "layer step: top-k ids differ"
+    assert np.array_equal(ly["w"], gpu["w"]), "layer step: routing weights differ"
+    assert ly["slot_offsets"].tolist() == so.tolist() and ly["rank_offsets"].tolist() == ro.tolist()
+    assert ly["rank_load"].tolist() == rl.tolist()
+    assert np.array_equal(ly["perm"], perm) and np.array_equal(ly["inv_perm"], inv), "layer step: dispatch index"
     realized = O.expert_histogram(gpu["ids"], E)
     report["real_max_over_mean_before"] = O.max_over_mean(O.rank_loads(realized, pi0, R))
     report["real_max_over_mean_after"] = O.max_over_mean(O.rank_loads(realized, pi_new, R))

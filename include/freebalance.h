@@ -254,6 +254,27 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream);
 /* Kernels this library has launched through `ctx` so far (for benchmarks). */
 uint64_t fb_launch_count(const fb_ctx* ctx);
 
+/* Limit on the SM pairs the router kernel may occupy (0 = no limit, the default).  The
+ * prediction pass is meant to run beside the previous layer's attention (stage 1 of the
+ * method is hidden behind it), so a caller may want to leave SMs free.  A call with more
+ * 256-row tile pairs than the limit (or than fit on the GPU at once, fb_max_pairs) runs
+ * the persistent kernel, where each block pair walks several tiles; results do not depend
+ * on the limit.  Honoured for the gate shapes that kernel supports (E a multiple of 32 up
+ * to 256; sigmoid gates with 32-expert groups and topk_group <= 4, or softmax gates whose
+ * weights are renormalised); other shapes ignore it.  Returns FB_ERR_INVALID_ARG for a
+ * negative limit. */
+fb_status fb_set_pair_limit(fb_ctx* ctx, int32_t pairs);
+/* Measurement aid: the next router-kernel launch made through ctx records the two CUDA
+ * events (cudaEvent_t handles owned by the caller, either may be NULL) on its stream,
+ * one directly before and one directly after the launch, and then forgets them.  Lets a
+ * caller time that kernel alone inside a call that launches several kernels. */
+fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
+/* Block pairs of the persistent router kernel that fit on the GPU at once (0 when the
+ * configuration does not support that kernel). */
+int32_t fb_max_pairs(const fb_ctx* ctx);
+/* How many of the launches counted by fb_launch_count were the persistent router kernel. */
+uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
+
 /* Text for a status code; never NULL. */
 const char* fb_status_string(fb_status s);
 

@@ -48,7 +48,9 @@ FB_ERR_RANGE = 6
 
 EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_predict_load",
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
-           "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step"]
+           "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
+           "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
+           "fb_time_next_router_launch"]
 
 _lib = None
 
@@ -92,6 +94,14 @@ def lib() -> ctypes.CDLL:
                                          vp, vp, vp, vp]
     L.fb_predict_load_static.restype = ctypes.c_int
     L.fb_device_status.argtypes = [vp, ctypes.POINTER(i32), vp]
+    L.fb_set_pair_limit.argtypes = [vp, i32]
+    L.fb_set_pair_limit.restype = ctypes.c_int
+    L.fb_max_pairs.argtypes = [vp]
+    L.fb_max_pairs.restype = i32
+    L.fb_time_next_router_launch.argtypes = [vp, vp, vp]
+    L.fb_time_next_router_launch.restype = ctypes.c_int
+    L.fb_persistent_launch_count.argtypes = [vp]
+    L.fb_persistent_launch_count.restype = u64
     L.fb_launch_count.argtypes = [vp]
     L.fb_launch_count.restype = u64
     L.fb_status_string.argtypes = [ctypes.c_int]
@@ -229,6 +239,26 @@ class Context:
         word = ctypes.c_int32(0)
         _check(lib().fb_device_status(self._h, ctypes.byref(word), _stream(stream)), "fb_device_status")
         return int(word.value)
+
+    def fb_set_pair_limit(self, pairs: int) -> None:
+        _check(lib().fb_set_pair_limit(self._h, pairs), "fb_set_pair_limit")
+
+    def fb_max_pairs(self) -> int:
+        return int(lib().fb_max_pairs(self._h))
+
+    def fb_time_next_router_launch(self, event_before, event_after) -> None:
+        """torch.cuda.Event objects (created with enable_timing=True); either may be None."""
+        def handle(ev):
+            if ev is None:
+                return None
+            if not ev.cuda_event:          # torch creates the CUDA event lazily, on the first record
+                ev.record()
+            return ctypes.c_void_p(ev.cuda_event)
+        _check(lib().fb_time_next_router_launch(self._h, handle(event_before), handle(event_after)),
+               "fb_time_next_router_launch")
+
+    def fb_persistent_launch_count(self) -> int:
+        return int(lib().fb_persistent_launch_count(self._h))
 
     def fb_launch_count(self) -> int:
         return int(lib().fb_launch_count(self._h))

@@ -12,6 +12,7 @@
 #include "fb_dispatch.cuh"
 #include "fb_planner.cuh"
 #include "fb_router.cuh"
+#include "fb_router_persistent.cuh"
 
 namespace {
 
@@ -38,6 +39,13 @@ struct fb_ctx {
   int tmem_cols = 0;
   size_t smem_bytes[2] = {0, 0};
   int max_tiles = 0;
+  // persistent router kernel (several tiles per block pair): pipeline depth (0 = not usable
+  // for this shape), dynamic shared memory, block pairs that fit on the GPU at once, and
+  // the caller's limit on the pairs to use (0 = none)
+  int persist_stages = 0;
+  size_t persist_smem = 0;
+  int max_pairs = 0;
+  int pair_limit = 0;
   EncodeTiledFn encode = nullptr;
   // device scratch
   uint32_t* counts_scratch = nullptr;   // [256], zero between calls
@@ -59,6 +67,8 @@ struct fb_ctx {
   uint32_t* st_slot_offsets = nullptr; uint32_t* st_rank_offsets = nullptr;
   int32_t* st_perm = nullptr; int32_t* st_inv_perm = nullptr; uint32_t* st_rank_load = nullptr;
   uint64_t launches = 0;
+  uint64_t persistent_launches = 0;
+  cudaEvent_t ev_before = nullptr, ev_after = nullptr;   // one-shot: recorded around the next router launch     // of those, launches of the persistent router kernel
 };
 
 namespace {
@@ -204,9 +214,21 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.tile_counts = ctx->tile_counts;
   if (plan) p.plan = *plan;
   const int tiles_pad = pair ? (tiles + 1) / 2 * 2 : tiles;       // a pair never straddles the two passes
-  const int blocks = mode == fb::kModeLayer ? 2 * tiles_pad : tiles_pad;
+  int blocks = mode == fb::kModeLayer ? 2 * tiles_pad : tiles_pad;
   p.tiles_first = tiles_pad;
   p.ticket_target = tiles_pad;
+  // More tile pairs than block pairs fit on the GPU (or than the caller allows): the
+  // persistent kernel walks several tiles per block pair and overlaps their epilogues.
+  bool persistent = false;
+  if (pair && ctx->persist_stages >= 2 && logits == nullptr) {
+    const bool want_sum = topk_w != nullptr && !c.renorm && c.gate == FB_GATE_SOFTMAX_TOPK;
+    const int pairs_avail = ctx->pair_limit > 0 && ctx->pair_limit < ctx->max_pairs ? ctx->pair_limit : ctx->max_pairs;
+    if (fb::persistent_gate_ok(c.E, c.k, c.gate, p.n_group, p.topk_group, want_sum) && blocks / 2 > pairs_avail) {
+      persistent = true;
+      blocks = 2 * pairs_avail;
+      p.stages = ctx->persist_stages;
+    }
+  }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.blockDim = dim3(fb::kRouterThreads, 1, 1);
@@ -214,6 +236,8 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   cudaError_t err;
+  if (persistent) cfg.dynamicSmemBytes = ctx->persist_smem;
+  if (ctx->ev_before) cudaEventRecord(ctx->ev_before, stream);
   if (pair) {
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -222,12 +246,16 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mx2, *mw, p);
+    err = persistent ? cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel, *mx, *mx2, *mw, p)
+                     : cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mx2, *mw, p);
   } else {
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
     err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1>, *mx, *mx2, *mw, p);
   }
+  if (ctx->ev_after) cudaEventRecord(ctx->ev_after, stream);
+  ctx->ev_before = ctx->ev_after = nullptr;
   ++ctx->launches;
+  if (persistent) ++ctx->persistent_launches;
   return err == cudaSuccess ? FB_OK : FB_ERR_CUDA;
 }
 
@@ -334,6 +362,16 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
     ctx->smem_bytes[pair] = dyn + 1024;
   }
   ctx->max_tiles = (cfg->T_max + fb::kTileM - 1) / fb::kTileM;
+  if (ctx->stages[1] >= 2 && ctx->N % 32 == 0 && ctx->N == cfg->E) {
+    const size_t budget_p = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::PersistShared) - 2048;
+    const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N / 2) * fb::kBlockK * 2;
+    if (budget_p > 1024 + fb::kPersistScratchBytes + 2 * stage_bytes) {
+      int stages = static_cast<int>((budget_p - 1024 - fb::kPersistScratchBytes) / stage_bytes);
+      if (stages > fb::kMaxStages) stages = fb::kMaxStages;
+      ctx->persist_stages = stages;
+      ctx->persist_smem = stages * stage_bytes + fb::kPersistScratchBytes + 1024;
+    }
+  }
 
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -348,6 +386,28 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   if (ctx->stages[1] >= 2)
     ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(ctx->smem_bytes[1])) == cudaSuccess;
+  if (ok && ctx->persist_stages >= 2) {
+    ok = cudaFuncSetAttribute(fb::fb_router_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(ctx->persist_smem)) == cudaSuccess;
+    // how many block pairs the GPU holds at once (the grid of the persistent kernel)
+    cudaLaunchConfig_t occ;
+    memset(&occ, 0, sizeof(occ));
+    occ.gridDim = dim3(2 * static_cast<unsigned>(prop.multiProcessorCount), 1, 1);
+    occ.blockDim = dim3(fb::kRouterThreads, 1, 1);
+    occ.dynamicSmemBytes = ctx->persist_smem;
+    cudaLaunchAttribute cl[1];
+    cl[0].id = cudaLaunchAttributeClusterDimension;
+    cl[0].val.clusterDim.x = 2; cl[0].val.clusterDim.y = 1; cl[0].val.clusterDim.z = 1;
+    occ.attrs = cl;
+    occ.numAttrs = 1;
+    int n_clusters = 0;
+    if (ok && cudaOccupancyMaxActiveClusters(&n_clusters, fb::fb_router_persistent_kernel, &occ) == cudaSuccess &&
+        n_clusters >= 1)
+      ctx->max_pairs = n_clusters;
+    else
+      ctx->persist_stages = 0;                           // not usable here: the one-tile kernel serves every call
+    cudaGetLastError();
+  }
   ok = ok && dev_alloc(&ctx->counts_scratch, FB_MAX_EXPERTS) && dev_alloc(&ctx->ticket, 1) &&
        dev_alloc(&ctx->status, 1) &&
        dev_alloc(&ctx->tile_counts, static_cast<size_t>(ctx->max_tiles) * cfg->E) &&
@@ -561,6 +621,23 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream_) {
 }
 
 uint64_t fb_launch_count(const fb_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+fb_status fb_set_pair_limit(fb_ctx* ctx, int32_t pairs) {
+  if (!ctx || pairs < 0) return FB_ERR_INVALID_ARG;
+  ctx->pair_limit = pairs;
+  return FB_OK;
+}
+
+fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after) {
+  if (!ctx) return FB_ERR_INVALID_ARG;
+  ctx->ev_before = static_cast<cudaEvent_t>(event_before);
+  ctx->ev_after = static_cast<cudaEvent_t>(event_after);
+  return FB_OK;
+}
+
+int32_t fb_max_pairs(const fb_ctx* ctx) { return ctx ? ctx->max_pairs : 0; }
+
+uint64_t fb_persistent_launch_count(const fb_ctx* ctx) { return ctx ? ctx->persistent_launches : 0; }
 
 }  // extern "C"
 

@@ -50,8 +50,12 @@ def make_context(wl: I.Workload, T_max: int) -> B.Context:
 
 
 def run_gpu_layer(ctx: B.Context, wl: I.Workload, li: I.LayerInputs, bkw: dict, want_logits=True,
-                  placement=None):
-    """All entry points on one layer; returns numpy copies of every output."""
+                  placement=None, pair_limit=0):
+    """All entry points on one layer; returns numpy copies of every output.
+
+    ``pair_limit`` > 0 caps the SM pairs of the router kernel for these calls, which sends
+    calls with more tile pairs than that through the persistent kernel."""
+    ctx.fb_set_pair_limit(pair_limit)
     dev = torch.device("cuda", ctx.device)
     T = li.h_prev.shape[0]
     E, R, k = wl.E, wl.R, wl.k
@@ -94,6 +98,7 @@ def run_gpu_layer(ctx: B.Context, wl: I.Workload, li: I.LayerInputs, bkw: dict, 
                       l_ids, l_w, l_so, l_ro, l_perm, l_inv, l_rl)
     status = ctx.fb_device_status()
     torch.cuda.synchronize(dev)
+    ctx.fb_set_pair_limit(0)
     n = int(n_swaps.item())
     fn = int(f_n.item())
     ln = int(l_n.item())

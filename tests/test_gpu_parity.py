@@ -14,11 +14,13 @@ from tests import parity_util as P
 pytestmark = pytest.mark.gpu
 
 
-def _run(wl, T, layer=0, seed=0, with_logit_bias=False, placement=None, want_logits=True, sample=None, **bud):
+def _run(wl, T, layer=0, seed=0, with_logit_bias=False, placement=None, want_logits=True, sample=None,
+         pair_limit=0, **bud):
     li = I.make_layer(wl, layer, seed, T=T, with_logit_bias=with_logit_bias)
     ctx = P.make_context(wl, max(T, 1))
     bkw = P.budget_kwargs(wl, max(T, 1), **bud)
-    gpu = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=want_logits, placement=placement)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=want_logits, placement=placement, pair_limit=pair_limit)
+    gpu["persistent_launches"] = ctx.fb_persistent_launch_count()
     rep = P.compare_layer(wl, li, bkw, gpu, placement=placement, sample_rows=sample)
     ctx.close()
     return rep, gpu
@@ -364,3 +366,72 @@ def test_random_shapes(seed):
                     topk_group=topk_group, renorm=int(rng.integers(0, 2)), route_scale=float(rng.choice([1.0, 2.5])),
                     rho=0.2, skew="zipf", zipf_s=1.0, max_swaps=int(rng.integers(0, E // 2 + 1)))
     _run(wl, T, layer=seed, with_logit_bias=bool(rng.integers(0, 2)))
+
+
+# ------------------------------------------------------------------ persistent router kernel (several tiles per block pair)
+@pytest.mark.parametrize("name,T,limit,d,lb", [
+    ("dsv3", 777, 1, None, False), ("dsv3", 1500, 2, None, False), ("dsv3", 2049, 3, None, True),
+    ("dsv3", 1000, 1, 448, False),      # 7 k-blocks: the two issuers' shares differ in length
+    ("dsv3", 600, 1, 64, True),         # a single k-block: only one accumulator is written
+    ("qwen3", 1000, 1, None, False), ("qwen3", 2500, 2, None, True), ("sweep32k", 900, 1, None, False),
+])
+def test_persistent_kernel_small(name, T, limit, d, lb):
+    wl = I.WORKLOADS[name]
+    if d is not None:
+        wl = dataclasses.replace(wl, d=d)
+    rep, gpu = _run(wl, T, layer=1, with_logit_bias=lb, want_logits=False, pair_limit=limit)
+    # predict, predict+plan, route+dispatch and the one-call layer step all took that kernel
+    assert gpu["persistent_launches"] == 4
+
+
+@pytest.mark.parametrize("name", ["qwen3", "dsv3"])
+def test_persistent_kernel_overflow_path(name):
+    wl = I.WORKLOADS[name]
+    T = 700
+    li = I.make_layer(wl, 0, 0, T=T)
+    li.W = torch.zeros_like(li.W)
+    li.W[:, 0] = 0.02                     # rows differ in their common logit only: all keys of a row stay equal
+    if li.select_bias is not None:
+        li.select_bias = torch.zeros(wl.E)
+    ctx = P.make_context(wl, T)
+    bkw = P.budget_kwargs(wl, T)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False, pair_limit=1)
+    assert ctx.fb_persistent_launch_count() == 4
+    assert (gpu["ids"] == np.arange(wl.k)).all() and (gpu["ids_early"] == np.arange(wl.k)).all()
+    P.compare_layer(wl, li, bkw, gpu)
+    ctx.close()
+
+
+def test_persistent_kernel_mixed_rows_overflow_and_not():
+    # half of the rows have all keys equal (overflow path), the others are ordinary
+    wl = I.WORKLOADS["dsv3"]
+    T = 900
+    li = I.make_layer(wl, 2, 0, T=T)
+    li.h_prev[::2] = 0
+    li.H[::2] = 0
+    li.select_bias = torch.zeros(wl.E)
+    ctx = P.make_context(wl, T)
+    bkw = P.budget_kwargs(wl, T)
+    gpu = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False, pair_limit=2)
+    assert ctx.fb_persistent_launch_count() == 4
+    assert (gpu["ids"][::2] == np.arange(wl.k)).all()
+    P.compare_layer(wl, li, bkw, gpu)
+    ctx.close()
+
+
+def test_pair_limit_does_not_change_results():
+    wl = I.WORKLOADS["dsv3"]
+    T = 3000
+    li = I.make_layer(wl, 5, 0, T=T)
+    ctx = P.make_context(wl, T)
+    bkw = P.budget_kwargs(wl, T)
+    ref = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False)
+    assert ctx.fb_persistent_launch_count() == 0
+    for limit in (1, 5, 11):
+        got = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False, pair_limit=limit)
+        for key in ("counts", "ids_early", "ids", "w", "perm", "inv_perm", "slot_offsets", "rank_load"):
+            assert np.array_equal(ref[key], got[key]), (limit, key)
+        assert ref["swaps"] == got["swaps"] and ref["layer"]["swaps"] == got["layer"]["swaps"]
+        assert np.array_equal(ref["layer"]["ids"], got["layer"]["ids"]) and np.array_equal(ref["layer"]["w"], got["layer"]["w"])
+    assert ctx.fb_persistent_launch_count() == 12
+    ctx.close()

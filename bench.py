@@ -1,10 +1,11 @@
 #!/usr/bin/env python
 """Benchmark of the FreeBalance per-layer hot path on B200.
 
-One "step" = the whole hot path for one MoE layer on one prefill batch:
-fb_predict_and_plan on h_{l-1} (early router pass, gating, top-k, histogram, rank
-loads, swap planner - one kernel launch) followed by fb_route_dispatch on H_l under
-the new placement (normal router pass, routing weights, dispatch index - two
+One "step" = the whole hot path for one MoE layer on one prefill batch, through
+fb_layer_step: the early router pass on h_{l-1} (gating, top-k, histogram, rank loads,
+swap planner) and the normal router pass on H_l (top-k ids, routing weights) in ONE
+kernel launch, then the dispatch index under the new placement in a second launch.
+`--api separate` times the same work as fb_predict_and_plan + fb_route_dispatch (three
 launches).  The metric is tokens per second through that path, per layer.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload dsv3] [--impl reference]
@@ -192,6 +193,8 @@ def main():
     ap.add_argument("--workload", default="dsv3", choices=sorted(I.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ring", type=int, default=2, help="distinct layers cycled through")
+    ap.add_argument("--api", default="layer", choices=["layer", "separate"],
+                    help="layer: fb_layer_step (default); separate: fb_predict_and_plan + fb_route_dispatch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     args = ap.parse_args()
@@ -237,11 +240,22 @@ def main():
                slot_offsets=i32(E + 1), rank_offsets=i32(R + 1), perm=i32(T * k), inv_perm=i32(T * k),
                rank_load=i32(R))
 
-    def step(L):
+    layer_api = args.api == "layer"
+
+    def predict_and_plan(L):
         ctx.fb_predict_and_plan(L["router"], L["h_prev"], T, L["pi"], budget, 0, out["counts"], out["pi_out"],
                                 out["swaps"], out["n_swaps"], out["load_before"], out["load_after"])
-        ctx.fb_route_dispatch(L["router"], L["H"], T, out["pi_out"], out["ids"], out["w"], out["slot_offsets"],
-                              out["rank_offsets"], out["perm"], out["inv_perm"], out["rank_load"])
+
+    def step(L):
+        if layer_api:
+            ctx.fb_layer_step(L["router"], L["h_prev"], L["H"], T, L["pi"], budget, 0, out["counts"], out["pi_out"],
+                              out["swaps"], out["n_swaps"], out["load_before"], out["load_after"], out["ids"],
+                              out["w"], out["slot_offsets"], out["rank_offsets"], out["perm"], out["inv_perm"],
+                              out["rank_load"])
+        else:
+            predict_and_plan(L)
+            ctx.fb_route_dispatch(L["router"], L["H"], T, out["pi_out"], out["ids"], out["w"], out["slot_offsets"],
+                                  out["rank_offsets"], out["perm"], out["inv_perm"], out["rank_load"])
 
     def barrier():
         if distributed:
@@ -256,41 +270,49 @@ def main():
 
     # ---- timed region: exactly K steps; events on the launching (current) stream
     K = args.steps
-    # The whole region is bracketed by two events.  Per-launch times (for the roofline of the
-    # dominant kernel) come from extra events on every `sample_every`-th step only: an event
+    # The whole region is bracketed by two events.  The duration of the dominant kernel (the
+    # router kernel: the first launch of the step) comes from a pair of events that the library
+    # records directly around that launch, on every `sample_every`-th step only: an event
     # between two launches keeps the GPU from starting the next kernel's launch early and
     # costs about 2 us per record, which would otherwise be charged to every step.
     sample_every = 8 if K >= 16 else 1
     sampled = [i for i in range(K) if i % sample_every == 0]
-    ev = {i: [torch.cuda.Event(enable_timing=True) for _ in range(3)] for i in sampled}
+    ev = {i: [torch.cuda.Event(enable_timing=True) for _ in range(2)] for i in sampled}
+    for pair in ev.values():                 # torch creates the CUDA event on its first record
+        for e in pair:
+            e.record()
     ev_begin, ev_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(physical_gpu_index(local_rank))
     launches0 = ctx.fb_launch_count()
+    persistent0 = ctx.fb_persistent_launch_count()
     barrier()
     sampler.start()
     ev_begin.record()
     for i in range(K):
-        L = layers[i % ring]
-        e3 = ev.get(i)
-        if e3:
-            e3[0].record()
-        ctx.fb_predict_and_plan(L["router"], L["h_prev"], T, L["pi"], budget, 0, out["counts"], out["pi_out"],
-                                out["swaps"], out["n_swaps"], out["load_before"], out["load_after"])
-        if e3:
-            e3[1].record()
-        ctx.fb_route_dispatch(L["router"], L["H"], T, out["pi_out"], out["ids"], out["w"], out["slot_offsets"],
-                              out["rank_offsets"], out["perm"], out["inv_perm"], out["rank_load"])
-        if e3:
-            e3[2].record()
+        e2 = ev.get(i)
+        if e2:
+            ctx.fb_time_next_router_launch(e2[0], e2[1])
+        step(layers[i % ring])
     ev_end.record()
     barrier()
     clocks = sampler.stop()
     launches = ctx.fb_launch_count() - launches0
+    persistent_launches = ctx.fb_persistent_launch_count() - persistent0
     total_ms = ev_begin.elapsed_time(ev_end)
-    predict_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in sampled]
-    dispatch_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in sampled]
+    router_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in sampled]
     total_ms = max_over_ranks(total_ms, dev)
     status = ctx.fb_device_status()
+
+    # ---- the fused predictor + planner alone (fb_predict_and_plan), outside the timed region:
+    # per-launch events, for the roofline fraction of that call by itself
+    pp_n = 0 if args.no_e2e else 24
+    pp_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(pp_n)]
+    for i in range(pp_n):
+        pp_ev[i][0].record()
+        predict_and_plan(layers[i % ring])
+        pp_ev[i][1].record()
+    barrier()
+    pp_ms = [a.elapsed_time(b) for a, b in pp_ev]
 
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
     L0 = layers_cpu[0]
@@ -320,30 +342,42 @@ def main():
         peaks = measured_peaks()
         ms_per_step = total_ms / K
         value = whole_job_throughput(world, T, K, total_ms)
-        # roofline of the dominant kernel (the fused router kernel of fb_predict_and_plan)
-        alg_bytes = 2 * T * d + 2 * d * E + 4 * E
-        alg_flops = 2 * T * d * E
-        k1_ms = statistics.mean(predict_ms)
-        achieved_gbs = alg_bytes / (k1_ms * 1e-3) / 1e9
-        achieved_tf = alg_flops / (k1_ms * 1e-3) / 1e12
-        t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
-        t_tensor = alg_flops / (peaks["bf16_tflops"] * 1e12)
-        roof = {"kernel": "fb_router_kernel (fb_predict_and_plan)", "bound": "hbm" if t_hbm >= t_tensor else "tensor",
-                "achieved": achieved_gbs if t_hbm >= t_tensor else achieved_tf,
-                "peak": peaks["hbm_gbs"] if t_hbm >= t_tensor else peaks["bf16_tflops"],
-                "unit": "GB/s" if t_hbm >= t_tensor else "TFLOP/s",
-                "frac": (achieved_gbs / peaks["hbm_gbs"]) if t_hbm >= t_tensor else (achieved_tf / peaks["bf16_tflops"]),
-                "peak_source": peaks["source"], "traffic": None, "kernel_us": k1_ms * 1e3,
-                "kernel_us_median": statistics.median(predict_ms) * 1e3,
-                "t_roof_us": max(t_hbm, t_tensor) * 1e6, "tensor_tflops": achieved_tf,
-                "tensor_frac_of_burst": achieved_tf / peaks["bf16_tflops"],
-                "dispatch_us": statistics.mean(dispatch_ms) * 1e3, "launches_timed": len(predict_ms)}
+        # Roofline of the dominant kernel: the router kernel of the step.  Algorithmic work per
+        # launch: read each input matrix once (2 T d bytes per pass), W once, write the counts and,
+        # in the normal pass, ids and weights (8 T k); 2 T d E flops per pass.
+        passes = 2 if layer_api else 1
+        alg_bytes = passes * 2 * T * d + 2 * d * E + 4 * E + (8 * T * k if layer_api else 0)
+        alg_flops = passes * 2 * T * d * E
+        k1_ms = statistics.mean(router_ms)
+
+        def roofline(ms, nbytes, nflops, kernel):
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            tf = nflops / (ms * 1e-3) / 1e12
+            t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+            t_tensor = nflops / (peaks["bf16_tflops"] * 1e12)
+            hbm = t_hbm >= t_tensor
+            return {"kernel": kernel, "bound": "hbm" if hbm else "tensor", "achieved": gbs if hbm else tf,
+                    "peak": peaks["hbm_gbs"] if hbm else peaks["bf16_tflops"], "unit": "GB/s" if hbm else "TFLOP/s",
+                    "frac": (gbs / peaks["hbm_gbs"]) if hbm else (tf / peaks["bf16_tflops"]),
+                    "peak_source": peaks["source"], "traffic": None, "kernel_us": ms * 1e3,
+                    "t_roof_us": max(t_hbm, t_tensor) * 1e6, "algorithmic_bytes": nbytes, "algorithmic_flops": nflops,
+                    "tensor_tflops": tf, "tensor_frac_of_burst": tf / peaks["bf16_tflops"],
+                    "tensor_frac_of_sustained": tf / peaks["bf16_tflops_sustained"]}
+
+        persistent = persistent_launches > 0
+        kname = ("fb_router_persistent_kernel" if persistent else "fb_router_kernel") + \
+                (" (fb_layer_step: both router passes in one launch)" if layer_api else " (fb_predict_and_plan)")
+        roof = roofline(k1_ms, alg_bytes, alg_flops, kname)
+        roof["kernel_us_median"] = statistics.median(router_ms) * 1e3
+        roof["launches_timed"] = len(router_ms)
+        roof["rest_of_step_us"] = ms_per_step * 1e3 - k1_ms * 1e3
+        traffic_key = wl.name + ("/layer" if layer_api else "")
         traffic_file = os.path.join(ROOT, "profiles", "router_kernel_traffic.json")
         if os.path.exists(traffic_file):
             with open(traffic_file) as f:
                 tr = json.load(f)
-            if wl.name in tr:
-                roof["traffic"] = tr[wl.name]
+            if traffic_key in tr:
+                roof["traffic"] = tr[traffic_key]
 
         lb, la = out["load_before"].cpu().tolist(), out["load_after"].cpu().tolist()
         pi_new = out["pi_out"].cpu().tolist()
@@ -362,6 +396,7 @@ def main():
                 "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": wl.name, "T": T, "d": d, "E": E, "k": k, "R": R,
                            "gate": "sigmoid_group_topk" if wl.gate else "softmax_topk",
+                           "api": "fb_layer_step" if layer_api else "fb_predict_and_plan + fb_route_dispatch",
                            "layers_in_ring": ring, "parallelism": f"replicas x{world}",
                            "l2": "each input matrix (%.0f MB) exceeds L2 (126 MB); consecutive launches read different matrices"
                                  % (T * d * 2 / 1e6) if T * d * 2 > L2_BYTES else
@@ -372,6 +407,10 @@ def main():
                         "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
                 "gpu_launches": int(launches), "device_status": status,
                 "roofline": roof,
+                "predict_and_plan": None if not pp_ms else dict(
+                    roofline(statistics.mean(pp_ms), 2 * T * d + 2 * d * E + 4 * E, 2 * T * d * E,
+                             "fb_router_kernel (fb_predict_and_plan alone, one event pair per launch)"),
+                    tokens_per_s=T / (statistics.mean(pp_ms) * 1e-3), launches_timed=len(pp_ms)),
                 "load_balance": {"predicted_max_over_mean": [mom(lb), mom(la)],
                                  "realized_max_over_mean": [mom(real_before), mom(real_after)],
                                  "n_swaps": int(out["n_swaps"].item())}}

@@ -238,6 +238,13 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)
       : "r"(taddr)
       : "memory");
 }
+// Both 32-bit words to shared memory when pred != 0; a predicated store, not a branch.
+__device__ __forceinline__ void st_shared_v2_if(uint32_t pred, uint32_t addr, uint32_t lo, uint32_t hi) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.u32 p, %0, 0;\n@p st.shared.v2.u32 [%1], {%2, %3};\n}\n" ::"r"(pred), "r"(addr),
+      "r"(lo), "r"(hi)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }

@@ -202,11 +202,11 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     float* gscore_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) +
                                                static_cast<size_t>(p.stages) * stage_bytes);   // [8][128]
     float* glow_s = gscore_s + kPersistGroups * kTileM;                                         // [8][128]
-    uint32_t* cand_hi = reinterpret_cast<uint32_t*>(glow_s + kPersistGroups * kTileM);          // [32][128]
-    uint32_t* cand_lo = cand_hi + kCandCap * kTileM;                                             // [32][128]
+    // candidates [32][128]: ordered key bits in the high word, ~expert id in the low word
+    unsigned long long* cand = reinterpret_cast<unsigned long long*>(glow_s + kPersistGroups * kTileM);
     uint32_t* out_hi = reinterpret_cast<uint32_t*>(gscore_s);   // [8][128]: group scores are dead by then
     uint32_t* out_lo = reinterpret_cast<uint32_t*>(glow_s);
-    float* merge_v = reinterpret_cast<float*>(cand_hi);         // [3][8][128]: candidates are dead by then
+    float* merge_v = reinterpret_cast<float*>(cand);            // [3][8][128]: candidates are dead by then
     int32_t* merge_i = reinterpret_cast<int32_t*>(merge_v + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);
 
     // any block may turn out to take the last ticket of the early pass
@@ -337,16 +337,18 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
           uint32_t mine = 0;
 #pragma unroll
           for (int j = 0; j < 32; ++j) mine += key[ci][j] >= floor_key ? 1u : 0u;
-          uint32_t pos = atomicAdd(&sh.cand_count[row_in_tile], mine);
+          const uint32_t first = atomicAdd(&sh.cand_count[row_in_tile], mine);
+          // predicated stores, no branches: slot address advances past every hit, a hit is stored
+          // while the slot is inside the list
+          const uint32_t list = smem_u32(cand) + static_cast<uint32_t>(row_in_tile) * 8u;
+          const uint32_t list_end = list + kCandCap * kTileM * 8u;
+          uint32_t slot = list + first * (kTileM * 8u);
+          const uint32_t id0 = ~static_cast<uint32_t>(c * 32);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            if (key[ci][j] >= floor_key) {
-              if (pos < kCandCap) {
-                cand_hi[pos * kTileM + row_in_tile] = ordered_bits(key[ci][j]);
-                cand_lo[pos * kTileM + row_in_tile] = ~static_cast<uint32_t>(c * 32 + j);
-              }
-              ++pos;
-            }
+            const uint32_t hit = key[ci][j] >= floor_key ? 1u : 0u;
+            st_shared_v2_if(hit & (slot < list_end ? 1u : 0u), slot, id0 - j, ordered_bits(key[ci][j]));
+            slot += hit * (kTileM * 8u);
           }
         }
       }
@@ -368,16 +370,13 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
           for (int t = 0; t < 4; ++t) {
             const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
             const uint32_t cc = c < n ? c : 0;
-            mykey[t] = (static_cast<unsigned long long>(cand_hi[cc * kTileM + row_in_tile]) << 32) |
-                       cand_lo[cc * kTileM + row_in_tile];
+            mykey[t] = cand[cc * kTileM + row_in_tile];
             rank[t] = 0;
           }
 #pragma unroll 2
           for (uint32_t d = 0; d < n_most; ++d) {
             const uint32_t dd = d < n ? d : 0;
-            const unsigned long long other = d < n
-                ? (static_cast<unsigned long long>(cand_hi[dd * kTileM + row_in_tile]) << 32) | cand_lo[dd * kTileM + row_in_tile]
-                : 0ull;
+            const unsigned long long other = d < n ? cand[dd * kTileM + row_in_tile] : 0ull;
 #pragma unroll
             for (int t = 0; t < 4; ++t) rank[t] += other > mykey[t] ? 1u : 0u;
           }

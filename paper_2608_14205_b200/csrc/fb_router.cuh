@@ -149,6 +149,135 @@ struct RouterShared {
   PlanShared plan;
 };
 
+// Order-preserving map of a float onto unsigned integers, and back.
+__device__ __forceinline__ uint32_t ordered_bits(float x) {
+  const uint32_t b = __float_as_uint(x);
+  return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t u) {
+  return __uint_as_float(u ^ ((u >> 31) ? 0x80000000u : 0xffffffffu));
+}
+
+// Ranking selection, shared by both router kernels.  cand[c * 128 + row] holds candidate c of
+// the row as one 64-bit word: ordered key bits in the high half, ~expert id in the low half,
+// so that "larger word" means "larger key, then lower id".  The kEpiSubs threads of a row
+// share the candidates (candidate c belongs to thread c % kEpiSubs); a candidate with fewer
+// than FB_MAX_TOPK larger ones is written to out_hi/out_lo[rank][row].  Returns true when
+// the row had more candidates than the list holds (nothing is written for it then).
+__device__ __forceinline__ bool rank_candidates(const unsigned long long* cand, uint32_t n_all, int sub,
+                                                int row_in_tile, uint32_t* out_hi, uint32_t* out_lo) {
+  const bool overflow = n_all > kCandCap;
+  const uint32_t n = overflow ? 0u : n_all;
+  const uint32_t n_most = __reduce_max_sync(0xffffffffu, n);
+#pragma unroll 1
+  for (uint32_t tier = 0; tier * 4 * kEpiSubs < n_most; ++tier) {
+    unsigned long long mykey[4];
+    uint32_t rank[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
+      mykey[t] = cand[(c < n ? c : 0) * kTileM + row_in_tile];
+      rank[t] = 0;
+    }
+#pragma unroll 2
+    for (uint32_t d = 0; d < n_most; ++d) {
+      const unsigned long long other = d < n ? cand[d * kTileM + row_in_tile] : 0ull;
+#pragma unroll
+      for (int t = 0; t < 4; ++t) rank[t] += other > mykey[t] ? 1u : 0u;
+    }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
+      if (c < n && rank[t] < static_cast<uint32_t>(FB_MAX_TOPK)) {
+        out_hi[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t] >> 32);
+        out_lo[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t]);
+      }
+    }
+  }
+  return overflow;
+}
+
+// The row's top-k list as rank_candidates left it.
+__device__ __forceinline__ void read_ranked(TopK& top, int k, const uint32_t* out_hi, const uint32_t* out_lo,
+                                            int row_in_tile) {
+#pragma unroll
+  for (int j = 0; j < FB_MAX_TOPK; ++j) {
+    if (j < k) {
+      top.v[j] = from_ordered_bits(out_hi[j * kTileM + row_in_tile]);
+      top.i[j] = static_cast<int32_t>(~out_lo[j * kTileM + row_in_tile]);
+    }
+  }
+}
+
+// Expert ids and routing weights of one token (Eq. 3's top-k with the model's weight rule).
+// select_bias_s: the selection bias in shared memory; sm_max / sm_sum: the row's softmax
+// denominator in the form sum * exp(max), used only by softmax gates without renormalisation.
+__device__ __forceinline__ void write_row_outputs(const TopK& top, const RouterParams& p, long long row,
+                                                  int32_t* out_ids, float* out_w, const float* select_bias_s,
+                                                  float sm_max, float sm_sum) {
+  const int k = p.k;
+  const bool sigmoid_gate = p.gate != FB_GATE_SOFTMAX_TOPK;
+  if (out_ids != nullptr) {
+#pragma unroll
+    for (int j = 0; j < FB_MAX_TOPK; ++j)
+      if (j < k) out_ids[row * k + j] = top.i[j];
+  }
+  if (out_w != nullptr) {
+    float w[FB_MAX_TOPK];
+    float wsum = 0.0f;
+    const float ref = top.v[0];                         // row maximum of the keys
+#pragma unroll
+    for (int j = 0; j < FB_MAX_TOPK; ++j) {
+      if (!sigmoid_gate) w[j] = (j < k) ? __expf(top.v[j] - ref) : 0.0f;
+      else w[j] = (j < k) ? top.v[j] - select_bias_s[top.i[j]] : 0.0f;   // unbiased sigmoid score
+      wsum += w[j];
+    }
+    float scale;
+    if (!sigmoid_gate) scale = p.renorm ? 1.0f / wsum : 1.0f / (sm_sum * __expf(sm_max - ref));
+    else scale = p.renorm ? p.route_scale / wsum : p.route_scale;
+#pragma unroll
+    for (int j = 0; j < FB_MAX_TOPK; ++j)
+      if (j < k) out_w[row * k + j] = w[j] * scale;
+  }
+}
+
+// End of a tile in the prediction modes: add the tile's histogram (shared memory, cleared
+// here) to the cross-block counts, take a ticket, and in the block that takes the last one
+// publish the count vector (Eq. 5), re-arm the scratch for the next call and run the planner
+// (Algorithm 1) when asked.  Called by all epilogue threads; et = thread index among them.
+template <class Shared>
+__device__ __forceinline__ void publish_counts(Shared& sh, const RouterParams& p, int et, int warp, int lane,
+                                               bool run_planner) {
+  for (int e = et; e < p.E; e += kEpilogueThreads) {
+    const uint32_t c = sh.hist[e];
+    if (c) atomicAdd(&p.counts_scratch[e], c);
+    sh.hist[e] = 0;
+  }
+  named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+  if (et == 0) {
+    // The barrier orders every thread's histogram atomics before this fence, and the
+    // fence (cumulative) publishes them device-wide before the ticket is taken.
+    __threadfence();
+    const uint32_t prev = atomicAdd(p.ticket, 1u);
+    sh.is_last = (prev == static_cast<uint32_t>(p.ticket_target) - 1) ? 1 : 0;
+  }
+  named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+  if (sh.is_last) {
+    // Every other tile has published its counts: this block finishes the pass.
+    __threadfence();
+    for (int e = et; e < p.E; e += kEpilogueThreads) {
+      const uint32_t c = __ldcg(&p.counts_scratch[e]);
+      p.counts_out[e] = c;
+      sh.plan.cnt[e] = c;
+      p.counts_scratch[e] = 0;           // ready for the next call
+    }
+    if (et == 0) *p.ticket = 0;
+    if (sh.abort_flag) { if (et == 0) atomicCAS(p.status, 0, FB_ERR_TIMEOUT); }
+    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    if (run_planner && warp == 2) plan_swaps_warp(p.plan, sh.plan, lane, p.status);
+  }
+}
+
 // Load columns [c0, c0 + 32) (or 16 when fewer remain) of this warp's 32 rows.
 __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32_t (&r)[32]) {
   if (N - c0 >= 32) tmem_ld_32x32b_x32(taddr + c0, r);
@@ -465,8 +594,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
     if (got && fast_select) {
       // ---------------- choose: rank the (at most 8) group scores of this row
-      uint32_t* cand_hi = reinterpret_cast<uint32_t*>(merge_v);             // [kCandCap][128] ordered key bits
-      uint32_t* cand_lo = cand_hi + kCandCap * kTileM;                       // [kCandCap][128] ~expert id
+      unsigned long long* cand = reinterpret_cast<unsigned long long*>(merge_v);   // [kCandCap][128], see rank_candidates
       int my_groups[2] = {-1, -1};                        // the 32-column groups this sub scans
       float floor_key = INFINITY;
       if (sigmoid_gate) {
@@ -507,10 +635,9 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           if (mask != 0 && first + i < kCandCap) {
             const int j = __ffs(mask) - 1;
             mask &= mask - 1;
-            const uint32_t bits = __float_as_uint(key_s[(base + j) * kTileM + row_in_tile]);
-            // order-preserving map of the float onto unsigned integers
-            cand_hi[(first + i) * kTileM + row_in_tile] = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
-            cand_lo[(first + i) * kTileM + row_in_tile] = ~static_cast<uint32_t>(base + j);
+            cand[(first + i) * kTileM + row_in_tile] =
+                (static_cast<unsigned long long>(ordered_bits(key_s[(base + j) * kTileM + row_in_tile])) << 32) |
+                ~static_cast<uint32_t>(base + j);
           }
         }
       }
@@ -520,57 +647,12 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     uint32_t* out_lo = out_hi + FB_MAX_TOPK * kTileM;
     bool overflow = false;
     if (got && fast_select) {
-      // ---------------- rank: candidate c beats d if its key is larger, or equal with a
-      // lower expert id; a candidate with fewer than k better ones is the rank-th choice
-      const uint32_t* cand_hi = reinterpret_cast<const uint32_t*>(merge_v);
-      const uint32_t* cand_lo = cand_hi + kCandCap * kTileM;
-      const uint32_t n_all = sh.cand_count[row_in_tile];
-      overflow = n_all > kCandCap;
-      const uint32_t n = overflow ? 0u : n_all;
-      const uint32_t n_most = __reduce_max_sync(0xffffffffu, n);
-#pragma unroll 1
-      for (uint32_t tier = 0; tier * 4 * kEpiSubs < n_most; ++tier) {
-        unsigned long long mykey[4];
-        uint32_t rank[4];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
-          const uint32_t cc = c < n ? c : 0;
-          mykey[t] = (static_cast<unsigned long long>(cand_hi[cc * kTileM + row_in_tile]) << 32) |
-                     cand_lo[cc * kTileM + row_in_tile];
-          rank[t] = 0;
-        }
-#pragma unroll 2
-        for (uint32_t d = 0; d < n_most; ++d) {
-          const uint32_t dd = d < n ? d : 0;
-          const unsigned long long other = d < n
-              ? (static_cast<unsigned long long>(cand_hi[dd * kTileM + row_in_tile]) << 32) | cand_lo[dd * kTileM + row_in_tile]
-              : 0ull;
-#pragma unroll
-          for (int t = 0; t < 4; ++t) rank[t] += other > mykey[t] ? 1u : 0u;
-        }
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
-          if (c < n && rank[t] < static_cast<uint32_t>(FB_MAX_TOPK)) {
-            out_hi[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t] >> 32);
-            out_lo[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t]);
-          }
-        }
-      }
+      overflow = rank_candidates(reinterpret_cast<const unsigned long long*>(merge_v), sh.cand_count[row_in_tile], sub,
+                                 row_in_tile, out_hi, out_lo);
     }
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
     if (got && fast_select && sub == 0) {
-      if (!overflow) {
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j) {
-          if (j < k) {
-            const uint32_t u = out_hi[j * kTileM + row_in_tile];
-            top.v[j] = __uint_as_float(u ^ ((u >> 31) ? 0x80000000u : 0xffffffffu));
-            top.i[j] = static_cast<int32_t>(~out_lo[j * kTileM + row_in_tile]);
-          }
-        }
-      }
+      if (!overflow) read_ranked(top, k, out_hi, out_lo, row_in_tile);
       if (__any_sync(0xffffffffu, overflow)) {
         // More than kCandCap keys reached the floor (many equal keys): plain scan of the
         // kept groups for the rows concerned.
@@ -715,30 +797,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
 
     // ---- outputs per row
-    if (writer) {
-      if (out_ids != nullptr) {
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j < k) out_ids[row * k + j] = top.i[j];
-      }
-      if (out_w != nullptr) {
-        float w[FB_MAX_TOPK];
-        float wsum = 0.0f;
-        const float ref = top.v[0];                         // row maximum of the keys
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j) {
-          if (!sigmoid_gate) w[j] = (j < k) ? __expf(top.v[j] - ref) : 0.0f;
-          else w[j] = (j < k) ? top.v[j] - sh.select_bias[top.i[j]] : 0.0f;   // unbiased sigmoid score
-          wsum += w[j];
-        }
-        float scale;
-        if (!sigmoid_gate) scale = p.renorm ? 1.0f / wsum : 1.0f / (sm_sum * __expf(sm_max - ref));
-        else scale = p.renorm ? p.route_scale / wsum : p.route_scale;
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j < k) out_w[row * k + j] = w[j] * scale;
-      }
-    }
+    if (writer) write_row_outputs(top, p, row, out_ids, out_w, sh.select_bias, sm_max, sm_sum);
     // ---- histogram: one shared-memory atomic per distinct expert per warp (Eq. 5)
     if (sub == 0) {
       if (E > 32) {
@@ -764,33 +823,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         for (int e = et; e < E; e += kEpilogueThreads)
           p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
     } else {
-      for (int e = et; e < E; e += kEpilogueThreads) {
-        const uint32_t c = sh.hist[e];
-        if (c) atomicAdd(&p.counts_scratch[e], c);
-      }
-      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-      if (et == 0) {
-        // The barrier orders every thread's histogram atomics before this fence, and the
-        // fence (cumulative) publishes them device-wide before the ticket is taken.
-        __threadfence();
-        const uint32_t prev = atomicAdd(p.ticket, 1u);
-        sh.is_last = (prev == static_cast<uint32_t>(p.ticket_target) - 1) ? 1 : 0;
-      }
-      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-      if (sh.is_last) {
-        // Every other block has published its counts: this one finishes the call.
-        __threadfence();
-        for (int e = et; e < E; e += kEpilogueThreads) {
-          const uint32_t c = __ldcg(&p.counts_scratch[e]);
-          p.counts_out[e] = c;
-          sh.plan.cnt[e] = c;
-          p.counts_scratch[e] = 0;           // ready for the next call
-        }
-        if (et == 0) *p.ticket = 0;
-        if (sh.abort_flag) { if (et == 0) atomicCAS(p.status, 0, FB_ERR_TIMEOUT); }
-        named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-        if (mode == kModePredictPlan && warp == 2) plan_swaps_warp(p.plan, sh.plan, lane, p.status);
-      }
+      publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
     }
   }
 

@@ -55,15 +55,6 @@ __host__ __device__ inline bool persistent_gate_ok(int E, int k, int gate, int n
   return (E / 32) * 2 >= k && !want_sum;
 }
 
-// Order-preserving map of a float onto unsigned integers, and back.
-__device__ __forceinline__ uint32_t ordered_bits(float x) {
-  const uint32_t b = __float_as_uint(x);
-  return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
-}
-__device__ __forceinline__ float from_ordered_bits(uint32_t u) {
-  return __uint_as_float(u ^ ((u >> 31) ? 0x80000000u : 0xffffffffu));
-}
-
 __device__ __forceinline__ void ring_advance(int& s, uint32_t& phase, int stages) {
   if (++s == stages) { s = 0; phase ^= 1u; }
 }
@@ -354,56 +345,15 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
       }
       named_bar_sync(kPlanBarrierId, kEpilogueThreads);
 
-      // ---------------- rank: candidate c beats d if its key is larger, or equal with a lower
-      // expert id; a candidate with fewer than k better ones is the rank-th choice
-      const uint32_t n_all = sh.cand_count[row_in_tile];
-      const bool overflow = n_all > kCandCap;                // many equal keys: handled below
+      // ---------------- rank the candidates (many equal keys can overflow the list: handled below)
+      const bool overflow = rank_candidates(cand, sh.cand_count[row_in_tile], sub, row_in_tile, out_hi, out_lo);
       if (overflow) sh.any_overflow = 1;
-      {
-        const uint32_t n = overflow ? 0u : n_all;
-        const uint32_t n_most = __reduce_max_sync(0xffffffffu, n);
-#pragma unroll 1
-        for (uint32_t tier = 0; tier * 4 * kEpiSubs < n_most; ++tier) {
-          unsigned long long mykey[4];
-          uint32_t rank[4];
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
-            const uint32_t cc = c < n ? c : 0;
-            mykey[t] = cand[cc * kTileM + row_in_tile];
-            rank[t] = 0;
-          }
-#pragma unroll 2
-          for (uint32_t d = 0; d < n_most; ++d) {
-            const uint32_t dd = d < n ? d : 0;
-            const unsigned long long other = d < n ? cand[dd * kTileM + row_in_tile] : 0ull;
-#pragma unroll
-            for (int t = 0; t < 4; ++t) rank[t] += other > mykey[t] ? 1u : 0u;
-          }
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const uint32_t c = (tier * 4 + t) * kEpiSubs + sub;
-            if (c < n && rank[t] < static_cast<uint32_t>(FB_MAX_TOPK)) {
-              out_hi[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t] >> 32);
-              out_lo[rank[t] * kTileM + row_in_tile] = static_cast<uint32_t>(mykey[t]);
-            }
-          }
-        }
-      }
       named_bar_sync(kPlanBarrierId, kEpilogueThreads);
       TopK top;
       top.init();
       if (sub == 0) {
         sh.cand_count[row_in_tile] = 0;                      // ready for the next tile
-        if (!overflow) {
-#pragma unroll
-          for (int j = 0; j < FB_MAX_TOPK; ++j) {
-            if (j < k) {
-              top.v[j] = from_ordered_bits(out_hi[j * kTileM + row_in_tile]);
-              top.i[j] = static_cast<int32_t>(~out_lo[j * kTileM + row_in_tile]);
-            }
-          }
-        }
+        if (!overflow) read_ranked(top, k, out_hi, out_lo, row_in_tile);
       }
       if (sh.any_overflow != 0) {
         // Some row of the tile had more than kCandCap keys at or above its floor (many equal
@@ -443,27 +393,8 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
       // ---------------- outputs per row
       const bool writer = valid && sub == 0;
       if (writer) {
-        if (out_ids != nullptr) {
-#pragma unroll
-          for (int j = 0; j < FB_MAX_TOPK; ++j)
-            if (j < k) out_ids[row * k + j] = top.i[j];
-        }
-        if (out_w != nullptr) {
-          float w[FB_MAX_TOPK];
-          float wsum = 0.0f;
-          const float ref = top.v[0];                         // row maximum of the keys
-#pragma unroll
-          for (int j = 0; j < FB_MAX_TOPK; ++j) {
-            if (!sigmoid_gate) w[j] = (j < k) ? __expf(top.v[j] - ref) : 0.0f;
-            else w[j] = (j < k) ? top.v[j] - sh.select_bias[top.i[j]] : 0.0f;   // unbiased sigmoid score
-            wsum += w[j];
-          }
-          // softmax gates reach this kernel only with renormalised weights
-          const float scale = !sigmoid_gate ? 1.0f / wsum : (p.renorm ? p.route_scale / wsum : p.route_scale);
-#pragma unroll
-          for (int j = 0; j < FB_MAX_TOPK; ++j)
-            if (j < k) out_w[row * k + j] = w[j] * scale;
-        }
+        // softmax gates reach this kernel only with renormalised weights: no denominator needed
+        write_row_outputs(top, p, row, out_ids, out_w, sh.select_bias, 0.0f, 1.0f);
         // ---------------- histogram (Eq. 5)
 #pragma unroll
         for (int j = 0; j < FB_MAX_TOPK; ++j)
@@ -478,33 +409,7 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
           sh.hist[e] = 0;
         }
       } else {
-        for (int e = et; e < E; e += kEpilogueThreads) {
-          const uint32_t c = sh.hist[e];
-          if (c) atomicAdd(&p.counts_scratch[e], c);
-          sh.hist[e] = 0;
-        }
-        named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-        if (et == 0) {
-          // The barrier orders every thread's histogram atomics before this fence, and the
-          // fence (cumulative) publishes them device-wide before the ticket is taken.
-          __threadfence();
-          const uint32_t prev = atomicAdd(p.ticket, 1u);
-          sh.is_last = (prev == static_cast<uint32_t>(p.ticket_target) - 1) ? 1 : 0;
-        }
-        named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-        if (sh.is_last) {
-          // Every other tile of the pass has published its counts: this block finishes the pass.
-          __threadfence();
-          for (int e = et; e < E; e += kEpilogueThreads) {
-            const uint32_t c = __ldcg(&p.counts_scratch[e]);
-            p.counts_out[e] = c;
-            sh.plan.cnt[e] = c;
-            p.counts_scratch[e] = 0;           // ready for the next call
-          }
-          if (et == 0) *p.ticket = 0;
-          named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-          if (mode == kModePredictPlan && warp == 2) plan_swaps_warp(p.plan, sh.plan, lane, p.status);
-        }
+        publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
       }
     }
   }

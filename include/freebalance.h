@@ -258,8 +258,9 @@ uint64_t fb_launch_count(const fb_ctx* ctx);
  * prediction pass is meant to run beside the previous layer's attention (stage 1 of the
  * method is hidden behind it), so a caller may want to leave SMs free.  A call with more
  * 256-row tile pairs than the limit (or than fit on the GPU at once, fb_max_pairs) runs
- * the persistent kernel, where each block pair walks several tiles; results do not depend
- * on the limit.  Honoured for the gate shapes that kernel supports (E a multiple of 32 up
+ * the persistent kernel, where each block pair walks several tiles (on as few block pairs as
+ * the resulting number of rounds needs: 128 tile pairs run on 64 block pairs, not on all 74);
+ * results do not depend on the limit.  Honoured for the gate shapes that kernel supports (E a multiple of 32 up
  * to 256; sigmoid gates with 32-expert groups and topk_group <= 4, or softmax gates whose
  * weights are renormalised); other shapes ignore it.  Returns FB_ERR_INVALID_ARG for a
  * negative limit. */

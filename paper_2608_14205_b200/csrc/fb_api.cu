@@ -237,18 +237,24 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   cfg.blockDim = dim3(fb::kRouterThreads, 1, 1);
   cfg.dynamicSmemBytes = ctx->smem_bytes[pair];
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   cudaError_t err;
   if (persistent) cfg.dynamicSmemBytes = ctx->persist_smem;
   if (ctx->ev_before) cudaEventRecord(ctx->ev_before, stream);
+  // Programmatic dependent launch: when the previous kernel of the stream allows it (the
+  // dispatch-index kernel does), this kernel's set-up overlaps that kernel's execution; the
+  // kernel waits for its completion (griddepcontrol.wait) before it reads any global memory.
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (pair) {
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
     err = persistent ? cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel, *mx, *mx2, *mw, p)
                      : cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mx2, *mw, p);
   } else {

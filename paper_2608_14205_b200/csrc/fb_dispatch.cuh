@@ -10,6 +10,7 @@
 #include <stdint.h>
 
 #include "../../include/freebalance.h"
+#include "fb_ptx.cuh"
 
 namespace fb {
 
@@ -47,6 +48,9 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
   const int t = threadIdx.x;
   const int tile = blockIdx.x;
   const int E = p.E, k = p.k;
+  // The next router kernel of the stream may set itself up while this grid runs (it waits for
+  // this grid's completion before it reads anything).
+  pdl_launch_dependents();
   if (t == 0) bad = 0;
   for (int s = t; s < FB_MAX_EXPERTS; s += kDispatchThreads) {
     owner[s] = -1; before[s] = 0; total[s] = 0;

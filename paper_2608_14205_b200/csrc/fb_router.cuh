@@ -335,8 +335,6 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     for (int e = et; e < FB_MAX_EXPERTS + 32; e += kEpilogueThreads) {
       if (e < FB_MAX_EXPERTS) sh.hist[e] = 0;
       if (e < kTileM) sh.cand_count[e] = 0;
-      sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
-      sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
     }
     if (mode == kModePredictPlan) plan_clear(sh.plan, et, kEpilogueThreads);
   }
@@ -344,6 +342,9 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   __syncthreads();
   if (kCtas == 2) { cluster_arrive(); cluster_wait(); }   // the partner's barriers and TMEM are ready too
   tcgen05_fence_after();
+  // Everything above touched only this block's own state and the call's parameters; from here on
+  // the kernel reads memory that earlier work of the stream may have written.
+  pdl_wait();
   const uint32_t tmem_base = sh.tmem_base;
 
   if (warp == 0) {
@@ -447,8 +448,12 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         chunk_group |= static_cast<uint32_t>((c * 32) / gs) << (4 * c);   // at most 8 groups here
       }
     }
-    // While the main loop runs, stage the placement for the planner (any block may turn
-    // out to be the last one).
+    // While the main loop runs, stage the biases (read by these warps only, after the barrier
+    // below) and the placement for the planner (any block may turn out to be the last one).
+    for (int e = et; e < FB_MAX_EXPERTS + 32; e += kEpilogueThreads) {
+      sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
+      sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
+    }
     if (mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
     named_bar_sync(kAccumBarrierId, kEpilogueThreads + 32);
     const bool got = sh.accum_ok != 0;

@@ -104,8 +104,6 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     for (int e = et; e < FB_MAX_EXPERTS; e += kEpilogueThreads) {
       sh.hist[e] = 0;
       if (e < kTileM) sh.cand_count[e] = 0;
-      sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
-      sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
     }
     if (p.mode == kModePredictPlan || p.mode == kModeLayer) plan_clear(sh.plan, et, kEpilogueThreads);
   }
@@ -113,6 +111,9 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
   __syncthreads();
   cluster_arrive(); cluster_wait();          // the partner's barriers and tensor memory are ready too
   tcgen05_fence_after();
+  // Everything above touched only this block's own state and the call's parameters; from here on
+  // the kernel reads memory that earlier work of the stream may have written.
+  pdl_wait();
   const uint32_t tmem_base = sh.tmem_base;
 
   if (warp == 0) {
@@ -200,6 +201,11 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     float* merge_v = reinterpret_cast<float*>(cand);            // [3][8][128]: candidates are dead by then
     int32_t* merge_i = reinterpret_cast<int32_t*>(merge_v + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);
 
+    // biases (read by these warps only, after the first barrier below)
+    for (int e = et; e < FB_MAX_EXPERTS; e += kEpilogueThreads) {
+      sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
+      sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
+    }
     // any block may turn out to take the last ticket of the early pass
     if (p.mode == kModePredictPlan || p.mode == kModeLayer) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
     uint32_t tiles_done = 0;

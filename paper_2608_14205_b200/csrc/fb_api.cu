@@ -312,6 +312,36 @@ bool dev_alloc(Tp** p, size_t count) {
 
 }  // namespace
 
+// Shape-dependent launch parameters of the one-tile router kernel (host arithmetic and
+// function attributes only): padded width, TMEM columns, pipeline depth and dynamic shared
+// memory of the single-block and the pair variant.
+static fb_status setup_router_shape(fb_ctx* ctx, const cudaDeviceProp& prop) {
+  const fb_config& cfg = ctx->cfg;
+  ctx->N = (cfg.E + 15) / 16 * 16;
+  ctx->tmem_cols = next_pow2_at_least_32(2 * ctx->N)   /* two accumulators */;
+  const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
+  for (int pair = 0; pair < 2; ++pair) {
+    const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N / (pair + 1)) * fb::kBlockK * 2;
+    int stages = static_cast<int>((budget - 1024) / stage_bytes);
+    if (stages > fb::kMaxStages) stages = fb::kMaxStages;
+    size_t dyn = stages * stage_bytes;
+    if (dyn < fb::epilogue_scratch_bytes(ctx->N)) dyn = fb::epilogue_scratch_bytes(ctx->N);
+    if (stages < 2 || dyn + 1024 > budget) {
+      if (pair == 0) return FB_ERR_UNSUPPORTED_SHAPE;
+      stages = 0;                                      // pair kernel not usable for this shape
+    }
+    ctx->stages[pair] = stages;
+    ctx->smem_bytes[pair] = dyn + 1024;
+  }
+  ctx->max_tiles = (cfg.T_max + fb::kTileM - 1) / fb::kTileM;
+  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(ctx->smem_bytes[0])) == cudaSuccess;
+  if (ctx->stages[1] >= 2)
+    ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(ctx->smem_bytes[1])) == cudaSuccess;
+  return ok ? FB_OK : FB_ERR_CUDA;
+}
+
 extern "C" {
 
 const char* fb_status_string(fb_status s) {
@@ -354,23 +384,10 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   if (!ctx) return FB_ERR_CUDA;
   ctx->cfg = *cfg;
   ctx->device = device;
-  ctx->N = (cfg->E + 15) / 16 * 16;
-  ctx->tmem_cols = next_pow2_at_least_32(2 * ctx->N)   /* two accumulators */;
-  const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
-  for (int pair = 0; pair < 2; ++pair) {
-    const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N / (pair + 1)) * fb::kBlockK * 2;
-    int stages = static_cast<int>((budget - 1024) / stage_bytes);
-    if (stages > fb::kMaxStages) stages = fb::kMaxStages;
-    size_t dyn = stages * stage_bytes;
-    if (dyn < fb::epilogue_scratch_bytes(ctx->N)) dyn = fb::epilogue_scratch_bytes(ctx->N);
-    if (stages < 2 || dyn + 1024 > budget) {
-      if (pair == 0) { delete ctx; return FB_ERR_UNSUPPORTED_SHAPE; }
-      stages = 0;                                      // pair kernel not usable for this shape
-    }
-    ctx->stages[pair] = stages;
-    ctx->smem_bytes[pair] = dyn + 1024;
+  {
+    const fb_status ss = setup_router_shape(ctx, prop);
+    if (ss != FB_OK) { delete ctx; return ss; }
   }
-  ctx->max_tiles = (cfg->T_max + fb::kTileM - 1) / fb::kTileM;
   if (ctx->stages[1] >= 2 && ctx->N % 32 == 0 && ctx->N == cfg->E) {
     const size_t budget_p = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::PersistShared) - 2048;
     const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx->N / 2) * fb::kBlockK * 2;
@@ -390,12 +407,8 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
     return FB_ERR_CUDA;
   }
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(ctx->smem_bytes[0])) == cudaSuccess;
-  if (ctx->stages[1] >= 2)
-    ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    static_cast<int>(ctx->smem_bytes[1])) == cudaSuccess;
-  if (ok && ctx->persist_stages >= 2) {
+  bool ok = true;
+  if (ctx->persist_stages >= 2) {
     ok = cudaFuncSetAttribute(fb::fb_router_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(ctx->persist_smem)) == cudaSuccess;
     // how many block pairs the GPU holds at once (the grid of the persistent kernel)
@@ -711,30 +724,9 @@ extern "C" fb_status fb_predict_load_static(const fb_config* cfg, int device, co
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FB_ERR_CUDA;
     ctx.cfg = *cfg;
-    ctx.N = (cfg->E + 15) / 16 * 16;
-    ctx.tmem_cols = next_pow2_at_least_32(2 * ctx.N);
-    const size_t budget = static_cast<size_t>(prop.sharedMemPerBlockOptin) - sizeof(fb::RouterShared) - 2048;
-    for (int pair = 0; pair < 2; ++pair) {
-      const size_t stage_bytes = fb::kATileBytes + static_cast<size_t>(ctx.N / (pair + 1)) * fb::kBlockK * 2;
-      int stages = static_cast<int>((budget - 1024) / stage_bytes);
-      if (stages > fb::kMaxStages) stages = fb::kMaxStages;
-      size_t dyn = stages * stage_bytes;
-      if (dyn < fb::epilogue_scratch_bytes(ctx.N)) dyn = fb::epilogue_scratch_bytes(ctx.N);
-      if (stages < 2 || dyn + 1024 > budget) {
-        if (pair == 0) { ctx.cfg.E = -1; return FB_ERR_UNSUPPORTED_SHAPE; }
-        stages = 0;
-      }
-      ctx.stages[pair] = stages;
-      ctx.smem_bytes[pair] = dyn + 1024;
-    }
-    bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   static_cast<int>(ctx.smem_bytes[0])) == cudaSuccess;
-    if (ctx.stages[1] >= 2)
-      ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      static_cast<int>(ctx.smem_bytes[1])) == cudaSuccess;
-    if (!ok) { ctx.cfg.E = -1; return FB_ERR_CUDA; }
+    const fb_status ss = setup_router_shape(&ctx, prop);
+    if (ss != FB_OK) { ctx.cfg.E = -1; return ss; }
     for (int i = 0; i < kMapCache; ++i) { ctx.x_maps[i] = MapEntry(); ctx.w_maps[i] = MapEntry(); }
-    ctx.max_tiles = (cfg->T_max + fb::kTileM - 1) / fb::kTileM;
   }
   ctx.counts_scratch = st.scratch;
   ctx.ticket = st.scratch + FB_STATIC_MAX_EXPERTS;

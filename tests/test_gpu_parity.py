@@ -435,3 +435,30 @@ def test_pair_limit_does_not_change_results():
         assert np.array_equal(ref["layer"]["ids"], got["layer"]["ids"]) and np.array_equal(ref["layer"]["w"], got["layer"]["w"])
     assert ctx.fb_persistent_launch_count() == 12
     ctx.close()
+
+
+def test_router_launch_events_and_pair_queries():
+    wl = I.WORKLOADS["dsv3"]
+    T = 1024
+    li = I.make_layer(wl, 0, 0, T=T)
+    ctx = P.make_context(wl, T)
+    assert 1 <= ctx.fb_max_pairs() <= 74                 # one block pair per two SMs at most
+    dev = torch.device("cuda", ctx.device)
+    router = B.make_router(li.W.to(dev), None, li.select_bias.to(dev))
+    counts = torch.zeros(wl.E, dtype=torch.int32, device=dev)
+    before, after = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    x = li.h_prev.to(dev)
+    ctx.fb_predict_load(router, x, T, counts)            # warm-up
+    ctx.fb_time_next_router_launch(before, after)
+    ctx.fb_predict_load(router, x, T, counts)
+    ctx.fb_predict_load(router, x, T, counts)            # not timed: the request was for one launch
+    torch.cuda.synchronize(dev)
+    us = before.elapsed_time(after) * 1e3
+    assert 1.0 < us < 500.0, us
+    assert int(counts.sum().item()) == T * wl.k
+    ctx.close()
+    tiny = P.make_context(I.WORKLOADS["tiny"], 512)
+    assert tiny.fb_max_pairs() == 0                      # E = 8: the persistent kernel does not apply
+    with pytest.raises(Exception):
+        tiny.fb_set_pair_limit(-1)
+    tiny.close()

@@ -29,10 +29,17 @@ itself live in ``tests/test_oracle_*.py``):
 * ``dispatch_index``     pinned: brute-force ``sorted`` on tiny inputs, a
                           hand-worked example, permutation/offset invariants.
 * ``budget_ns``          pinned: Eq. 10 special cases.
+* ``row_cosine_mean``    pinned: closed forms (equal, opposite, orthogonal rows,
+                          a 45-degree pair, scale invariance, the zero-row rule).
+* ``serving_loop``       pinned: placement carry-over checked step by step against
+                          ``layer_step`` started from the carried placement, a
+                          hand-worked two-step example of the realised-load
+                          figures, and the empty-budget case (nothing ever moves).
 """
 from __future__ import annotations
 
 import dataclasses
+import math
 from fractions import Fraction
 from typing import List, Optional, Sequence, Tuple
 
@@ -398,3 +405,69 @@ def layer_step(h_prev_bits, H_bits, W_bits, gate: Gate, R: int, expert_to_slot, 
     disp = dispatch_index(ids, pi_new, R)
     return dict(z_early=z_early, ids_early=ids_early, counts=counts, swaps=swaps, pi_new=pi_new,
                 load_before=load_before, load_after=load_after, z=z, ids=ids, w=w, dispatch=disp)
+
+
+# ----------------------------------------------------------------------------
+# Prediction / planning quality over a sequence of prefill steps
+# (Evaluation, "Metrics" and "Prediction and Planning Quality")
+# ----------------------------------------------------------------------------
+def row_cosine_mean(a: np.ndarray, b: np.ndarray) -> float:
+    """Cosine similarity between corresponding rows (tokens) of a and b, averaged over
+    the rows; a row with a zero vector on either side contributes 0."""
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    if a.shape[0] == 0:
+        return 0.0
+    total = 0.0
+    for i in range(a.shape[0]):
+        na = math.sqrt(float(np.dot(a[i], a[i])))
+        nb = math.sqrt(float(np.dot(b[i], b[i])))
+        if na > 0.0 and nb > 0.0:
+            total += float(np.dot(a[i], b[i])) / (na * nb)
+    return total / a.shape[0]
+
+
+def serving_loop(trace, gate: Gate, R: int, bud: Budget, with_cosines: bool = True):
+    """Run layer_step over a sequence of prefill steps with the placement of every layer
+    carried from one step to the next (a committed swap plan stays in force until a later
+    plan changes it), and record the paper's quality metrics per (step, layer).
+
+    ``trace`` yields ``(step, layer, h_prev_bits, H_bits, W_bits, select_bias, logit_bias)``
+    in execution order.  Returns ``(records, summary, placements)``.
+    """
+    placements = {}
+    records = []
+    for step, layer, h_prev_bits, H_bits, W_bits, select_bias, logit_bias in trace:
+        pi_old = placements.get(layer, list(range(gate.E)))
+        out = layer_step(h_prev_bits, H_bits, W_bits, gate, R, pi_old, bud, select_bias, logit_bias, layer)
+        realized = expert_histogram(out["ids"], gate.E)
+        real_before = rank_loads(realized, pi_old, R)
+        real_after = rank_loads(realized, out["pi_new"], R)
+        real_vanilla = rank_loads(realized, list(range(gate.E)), R)      # the fixed initial placement
+        rec = dict(step=step, layer=layer, pi_old=list(pi_old), pi_new=list(out["pi_new"]), swaps=out["swaps"],
+                   counts=out["counts"], realized=realized,
+                   pred_before=max_over_mean(out["load_before"]), pred_after=max_over_mean(out["load_after"]),
+                   real_before=max_over_mean(real_before), real_after=max_over_mean(real_after),
+                   real_vanilla=max_over_mean(real_vanilla),
+                   hit_rate=topk_hit_rate(out["ids_early"], out["ids"]),
+                   improved=max_over_mean(real_after) < max_over_mean(real_before))
+        if with_cosines:
+            rec["cos_hidden"] = row_cosine_mean(bf16_bits_to_f64(h_prev_bits), bf16_bits_to_f64(H_bits))
+            rec["cos_logits"] = row_cosine_mean(out["z_early"], out["z"])
+        records.append(rec)
+        placements[layer] = list(out["pi_new"])
+    moved = [r for r in records if len(r["swaps"]) > 0]
+    n = max(1, len(records))
+    summary = dict(
+        layers_run=len(records),
+        swaps_per_layer=sum(len(r["swaps"]) for r in records) / n,
+        hit_rate=sum(r["hit_rate"] for r in records) / n,
+        real_max_over_mean_vanilla=max((r["real_vanilla"] for r in records), default=1.0),
+        real_max_over_mean_balanced=max((r["real_after"] for r in records), default=1.0),
+        layers_with_migration=len(moved),
+        improved_fraction=(sum(1 for r in moved if r["improved"]) / len(moved)) if moved else None,
+    )
+    if with_cosines and records:
+        summary["cos_hidden"] = sum(r["cos_hidden"] for r in records) / n
+        summary["cos_logits"] = sum(r["cos_logits"] for r in records) / n
+    return records, summary, placements

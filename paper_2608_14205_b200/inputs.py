@@ -178,6 +178,57 @@ def make_layer(wl: Workload, layer: int = 0, seed: int = 0, T: Optional[int] = N
                        expert_to_slot=torch.arange(wl.E, dtype=torch.int32))
 
 
+def make_step_layer(wl: Workload, layer: int, step: int, seed: int = 0, T: Optional[int] = None,
+                    rho: Optional[float] = None, sys_drift: float = 0.0) -> LayerInputs:
+    """One layer of one prefill step of a changing-task serving sequence.
+
+    Stands in for the paper's "Mixed Tasks" workload, where every prefill step draws all of
+    its requests from one task and the task changes from step to step: the router weights
+    of a layer are those of ``make_layer`` (fixed across steps), every token of step
+    ``step`` belongs to the single task cluster ``c(step)`` (a seeded sequence over the
+    workload's clusters; shapes without clusters just get fresh noise per step), and the
+    normal router input adds, on top of the per-token drift of relative norm ``rho``, a
+    systematic component ``sys_drift * ||h_i|| * u`` along a fixed unit direction ``u`` of
+    the layer that raises a seeded Zipf-ordered set of experts, so that the early pass
+    mispredicts the aggregate counts and not only single tokens.
+    """
+    T = wl.T if T is None else T
+    rho = wl.rho if rho is None else rho
+    W = make_router(wl, layer, seed)
+    Wf = W.float()
+    row_norm2 = (Wf * Wf).sum(dim=1).clamp_min(1e-12)
+
+    g = _gen(seed, layer, 1000 + 10 * step + 3)
+    h = torch.randn(T, wl.d, generator=g, dtype=torch.float32)
+    if wl.skew == "clusters" and T > 0:
+        gc = _gen(seed, layer, 4)                     # the same cluster means as make_layer
+        mus = []
+        for _ in range(wl.n_clusters):
+            o = wl.kappa * _zipf_log_weights(wl.E, wl.zipf_s, gc).float()
+            mus.append(((o / row_norm2)[:, None] * Wf).sum(dim=0))
+        task = int(torch.randint(0, wl.n_clusters, (1,), generator=_gen(seed, 0, 2000 + step)).item())
+        h += mus[task]
+    h_prev = h.to(torch.bfloat16)
+
+    g = _gen(seed, layer, 1000 + 10 * step + 5)
+    u = torch.randn(T, wl.d, generator=g, dtype=torch.float32)
+    hf = h_prev.float()
+    hn = hf.norm(dim=1, keepdim=True)
+    Hf = hf + u * (rho * hn / u.norm(dim=1, keepdim=True).clamp_min(1e-20))
+    if sys_drift != 0.0 and T > 0:
+        o = _zipf_log_weights(wl.E, max(wl.zipf_s, 1.0), _gen(seed, layer, 9)).float()
+        direction = ((o / row_norm2)[:, None] * Wf).sum(dim=0)
+        direction = direction / direction.norm().clamp_min(1e-20)
+        Hf = Hf + sys_drift * hn * direction[None, :]
+    H = Hf.to(torch.bfloat16)
+
+    select_bias = None
+    if wl.gate == GATE_SIGMOID_GROUP_TOPK:
+        select_bias = 0.02 * torch.randn(wl.E, generator=_gen(seed, layer, 6), dtype=torch.float32)
+    return LayerInputs(h_prev=h_prev, H=H, W=W, select_bias=select_bias, logit_bias=None,
+                       expert_to_slot=torch.arange(wl.E, dtype=torch.int32))
+
+
 def random_counts(E: int, total: int, seed: int, zipf_s: float = 1.0) -> torch.Tensor:
     """A skewed expert count vector with a given sum, for planner-only tests."""
     g = _gen(seed, 0, 8)

@@ -254,6 +254,24 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream);
 /* Kernels this library has launched through `ctx` so far (for benchmarks). */
 uint64_t fb_launch_count(const fb_ctx* ctx);
 
+/* ---- prediction-quality metrics (Evaluation, "Metrics"); not part of the per-layer hot path ---- */
+#define FB_DTYPE_BF16 0
+#define FB_DTYPE_F32 1
+/* Mean over the rows (tokens) of the cosine similarity between row i of a and row i of b:
+ * the paper's hidden-state cosine (a = h_prev, b = H, bf16 [rows][n]) and logit cosine
+ * (a, b = the two router invocations' logits, f32 [rows][n], as dumped by fb_predict_load
+ * and fb_route_dispatch).  A row that is zero on either side contributes 0.  All pointers
+ * are device pointers; row_scratch (double[rows]) receives the per-row cosines, mean_out
+ * (one double) their mean; sums are formed in double precision in a fixed order.  rows = 0
+ * gives 0.  Errors: FB_ERR_INVALID_ARG for a bad size, dtype or NULL pointer. */
+fb_status fb_row_cosine_mean(const void* a, const void* b, int64_t rows, int32_t n, int32_t dtype,
+                             double* row_scratch, double* mean_out, fb_stream stream);
+/* Numerator of the top-k hit rate: the number of (token, expert) assignments of ids_b
+ * ([T][k], the normal pass) that also appear in ids_a ([T][k], the early pass); the hit
+ * rate is that number / (T k).  Device pointers; hits_out is one uint32. */
+fb_status fb_topk_hits(const int32_t* ids_a, const int32_t* ids_b, int32_t T, int32_t k, uint32_t* hits_out,
+                       fb_stream stream);
+
 /* Limit on the SM pairs the router kernel may occupy (0 = no limit, the default).  The
  * prediction pass is meant to run beside the previous layer's attention (stage 1 of the
  * method is hidden behind it), so a caller may want to leave SMs free.  A call with more

@@ -50,7 +50,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
-           "fb_time_next_router_launch"]
+           "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits"]
 
 _lib = None
 
@@ -98,6 +98,10 @@ def lib() -> ctypes.CDLL:
     L.fb_set_pair_limit.restype = ctypes.c_int
     L.fb_max_pairs.argtypes = [vp]
     L.fb_max_pairs.restype = i32
+    L.fb_row_cosine_mean.argtypes = [vp, vp, ctypes.c_int64, i32, i32, vp, vp, vp]
+    L.fb_row_cosine_mean.restype = ctypes.c_int
+    L.fb_topk_hits.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.fb_topk_hits.restype = ctypes.c_int
     L.fb_time_next_router_launch.argtypes = [vp, vp, vp]
     L.fb_time_next_router_launch.restype = ctypes.c_int
     L.fb_persistent_launch_count.argtypes = [vp]
@@ -161,6 +165,24 @@ def fb_budget_ns(t_attn_ns: int, delta_ns: int) -> int:
 
 def fb_swap_cost_ns(budget: FbBudget, rank_a: int, rank_b: int) -> int:
     return int(lib().fb_swap_cost_ns(ctypes.byref(budget), rank_a, rank_b))
+
+
+FB_DTYPE_BF16, FB_DTYPE_F32 = 0, 1
+
+
+def fb_row_cosine_mean(a: torch.Tensor, b: torch.Tensor, row_scratch: torch.Tensor, mean_out: torch.Tensor,
+                       stream=None) -> None:
+    """a, b: [rows, n] bf16 or f32 device tensors; row_scratch: float64 [rows]; mean_out: float64 [1]."""
+    assert a.shape == b.shape and a.dtype == b.dtype and a.dim() == 2
+    assert row_scratch.dtype == torch.float64 and mean_out.dtype == torch.float64
+    dtype = {torch.bfloat16: FB_DTYPE_BF16, torch.float32: FB_DTYPE_F32}[a.dtype]
+    _check(lib().fb_row_cosine_mean(_ptr(a), _ptr(b), a.shape[0], a.shape[1], dtype, _ptr(row_scratch),
+                                    _ptr(mean_out), _stream(stream)), "fb_row_cosine_mean")
+
+
+def fb_topk_hits(ids_a: torch.Tensor, ids_b: torch.Tensor, T: int, k: int, hits_out: torch.Tensor,
+                 stream=None) -> None:
+    _check(lib().fb_topk_hits(_ptr(ids_a), _ptr(ids_b), T, k, _ptr(hits_out), _stream(stream)), "fb_topk_hits")
 
 
 def fb_predict_load_static(cfg: FbConfig, device: int, router: FbRouter, x, T: int, counts, topk_ids=None,

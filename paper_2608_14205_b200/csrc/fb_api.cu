@@ -11,6 +11,7 @@
 #include "../../include/freebalance.h"
 #include "fb_dispatch.cuh"
 #include "fb_planner.cuh"
+#include "fb_quality.cuh"
 #include "fb_router.cuh"
 #include "fb_router_persistent.cuh"
 
@@ -643,6 +644,33 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream_) {
 }
 
 uint64_t fb_launch_count(const fb_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+fb_status fb_row_cosine_mean(const void* a, const void* b, int64_t rows, int32_t n, int32_t dtype,
+                             double* row_scratch, double* mean_out, fb_stream stream_) {
+  if (rows < 0 || n <= 0 || (dtype != FB_DTYPE_BF16 && dtype != FB_DTYPE_F32) || !mean_out) return FB_ERR_INVALID_ARG;
+  if (rows > 0 && (!a || !b || !row_scratch)) return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (rows > 0) {
+    const unsigned blocks = static_cast<unsigned>((rows + fb::kCosineWarpsPerBlock - 1) / fb::kCosineWarpsPerBlock);
+    if (dtype == FB_DTYPE_BF16)
+      fb::fb_row_cosine_kernel<__nv_bfloat16><<<blocks, 32 * fb::kCosineWarpsPerBlock, 0, stream>>>(
+          static_cast<const __nv_bfloat16*>(a), static_cast<const __nv_bfloat16*>(b), rows, n, row_scratch);
+    else
+      fb::fb_row_cosine_kernel<float><<<blocks, 32 * fb::kCosineWarpsPerBlock, 0, stream>>>(
+          static_cast<const float*>(a), static_cast<const float*>(b), rows, n, row_scratch);
+  }
+  fb::fb_mean_kernel<<<1, fb::kMeanThreads, 0, stream>>>(row_scratch, rows, mean_out);
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status fb_topk_hits(const int32_t* ids_a, const int32_t* ids_b, int32_t T, int32_t k, uint32_t* hits_out,
+                       fb_stream stream_) {
+  if (T < 0 || k < 1 || k > FB_MAX_TOPK || !hits_out || (T > 0 && (!ids_a || !ids_b))) return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (cudaMemsetAsync(hits_out, 0, sizeof(uint32_t), stream) != cudaSuccess) return FB_ERR_CUDA;
+  if (T > 0) fb::fb_topk_hits_kernel<<<(T + 255) / 256, 256, 0, stream>>>(ids_a, ids_b, T, k, hits_out);
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
 
 fb_status fb_set_pair_limit(fb_ctx* ctx, int32_t pairs) {
   if (!ctx || pairs < 0) return FB_ERR_INVALID_ARG;

@@ -1,0 +1,76 @@
+// Prediction-quality metrics of the evaluation (not part of the per-layer hot path):
+// the mean over tokens of the cosine similarity between two row-major matrices (hidden
+// states before / after the residual update, or the two router invocations' logits), and
+// the number of final top-k assignments the early pass recovered (hit rate numerator).
+// Sums are formed in a fixed order, in double precision, so results are reproducible.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fb {
+
+constexpr int kCosineWarpsPerBlock = 8;
+constexpr int kMeanThreads = 1024;
+
+__device__ __forceinline__ double load_as_double(const __nv_bfloat16* p, long long i) {
+  return static_cast<double>(__bfloat162float(p[i]));
+}
+__device__ __forceinline__ double load_as_double(const float* p, long long i) { return static_cast<double>(p[i]); }
+
+// One warp per row: lane l takes elements l, l + 32, ...; the three partial sums are
+// combined by a butterfly, which gives every lane the same total.
+template <class Tin>
+__global__ void __launch_bounds__(32 * kCosineWarpsPerBlock)
+fb_row_cosine_kernel(const Tin* __restrict__ a, const Tin* __restrict__ b, long long rows, int n,
+                     double* __restrict__ row_cos) {
+  const long long row = static_cast<long long>(blockIdx.x) * kCosineWarpsPerBlock + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const long long base = row * n;
+  double dot = 0.0, na = 0.0, nb = 0.0;
+  for (int j = lane; j < n; j += 32) {
+    const double x = load_as_double(a, base + j), y = load_as_double(b, base + j);
+    dot += x * y; na += x * x; nb += y * y;
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    na += __shfl_xor_sync(0xffffffffu, na, off);
+    nb += __shfl_xor_sync(0xffffffffu, nb, off);
+  }
+  if (lane == 0) row_cos[row] = (na > 0.0 && nb > 0.0) ? dot / (sqrt(na) * sqrt(nb)) : 0.0;
+}
+
+// Mean of v[0 .. count) by one block: strided partial sums, then a shared-memory tree.
+__global__ void __launch_bounds__(kMeanThreads)
+fb_mean_kernel(const double* __restrict__ v, long long count, double* __restrict__ out) {
+  __shared__ double part[kMeanThreads];
+  double s = 0.0;
+  for (long long i = threadIdx.x; i < count; i += kMeanThreads) s += v[i];
+  part[threadIdx.x] = s;
+  __syncthreads();
+  for (int w = kMeanThreads / 2; w >= 1; w >>= 1) {
+    if (threadIdx.x < w) part[threadIdx.x] += part[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = count > 0 ? part[0] / static_cast<double>(count) : 0.0;
+}
+
+// hits += |ids_a[i, :] intersect ids_b[i, :]| over tokens i (ids within a token are distinct).
+__global__ void __launch_bounds__(256)
+fb_topk_hits_kernel(const int32_t* __restrict__ ids_a, const int32_t* __restrict__ ids_b, int T, int k,
+                    uint32_t* __restrict__ hits) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  uint32_t mine = 0;
+  if (i < T) {
+    for (int x = 0; x < k; ++x) {
+      const int32_t e = ids_b[static_cast<long long>(i) * k + x];
+      for (int y = 0; y < k; ++y) mine += ids_a[static_cast<long long>(i) * k + y] == e ? 1u : 0u;
+    }
+  }
+  mine = __reduce_add_sync(0xffffffffu, mine);
+  if ((threadIdx.x & 31) == 0 && mine) atomicAdd(hits, mine);      // integer sum: order does not matter
+}
+
+}  // namespace fb

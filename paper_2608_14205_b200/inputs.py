@@ -187,10 +187,12 @@ def make_step_layer(wl: Workload, layer: int, step: int, seed: int = 0, T: Optio
     of a layer are those of ``make_layer`` (fixed across steps), every token of step
     ``step`` belongs to the single task cluster ``c(step)`` (a seeded sequence over the
     workload's clusters; shapes without clusters just get fresh noise per step), and the
-    normal router input adds, on top of the per-token drift of relative norm ``rho``, a
-    systematic component ``sys_drift * ||h_i|| * u`` along a fixed unit direction ``u`` of
-    the layer that raises a seeded Zipf-ordered set of experts, so that the early pass
-    mispredicts the aggregate counts and not only single tokens.
+    normal router input adds, on top of the per-token drift of relative norm ``rho``, the
+    same systematic vector to every token: the combination of router rows that moves the
+    logit of expert e by about ``sys_drift * o_e``, where ``o`` is a seeded, zero-mean Zipf
+    log-weight vector of the layer (logits have a standard deviation of about
+    ``0.02 * sqrt(d)``).  The early pass then mispredicts the aggregate counts and not only
+    single tokens.
     """
     T = wl.T if T is None else T
     rho = wl.rho if rho is None else rho
@@ -218,8 +220,7 @@ def make_step_layer(wl: Workload, layer: int, step: int, seed: int = 0, T: Optio
     if sys_drift != 0.0 and T > 0:
         o = _zipf_log_weights(wl.E, max(wl.zipf_s, 1.0), _gen(seed, layer, 9)).float()
         direction = ((o / row_norm2)[:, None] * Wf).sum(dim=0)
-        direction = direction / direction.norm().clamp_min(1e-20)
-        Hf = Hf + sys_drift * hn * direction[None, :]
+        Hf = Hf + sys_drift * direction[None, :]
     H = Hf.to(torch.bfloat16)
 
     select_bias = None

@@ -31,6 +31,10 @@ itself live in ``tests/test_oracle_*.py``):
 * ``budget_ns``          pinned: Eq. 10 special cases.
 * ``row_cosine_mean``    pinned: closed forms (equal, opposite, orthogonal rows,
                           a 45-degree pair, scale invariance, the zero-row rule).
+* ``apply_swaps``        pinned: the placement definition (the slot the new placement
+                          names holds the expert's original bytes, for every expert),
+                          a hand-worked exchange, identity on the empty plan, twice =
+                          identity, agreement with ``plan_swaps``' own new placement.
 * ``serving_loop``       pinned: placement carry-over checked step by step against
                           ``layer_step`` started from the carried placement, a
                           hand-worked two-step example of the realised-load
@@ -471,3 +475,22 @@ def serving_loop(trace, gate: Gate, R: int, bud: Budget, with_cosines: bool = Tr
         summary["cos_hidden"] = sum(r["cos_hidden"] for r in records) / n
         summary["cos_logits"] = sum(r["cos_logits"] for r in records) / n
     return records, summary, placements
+
+
+# ----------------------------------------------------------------------------
+# Stage 3 on one device: the accepted swaps applied to the expert weights
+# (Method overview, "Weight Transfer"; "Budgeted Expert-Swap Planning", pairwise exchange)
+# ----------------------------------------------------------------------------
+def apply_swaps(slot_weights: np.ndarray, expert_to_slot: Sequence[int], swaps):
+    """Exchange, swap by swap, the weights of the two experts of each accepted swap between
+    the physical slots that hold them.  ``slot_weights[p]`` is the byte image of the expert
+    in slot p.  Returns ``(new_slot_weights, expert_to_slot_after)``."""
+    w = np.array(slot_weights, copy=True)
+    pi = [int(p) for p in expert_to_slot]
+    for _, _, e_a, e_b in swaps:
+        pa, pb = pi[e_a], pi[e_b]
+        tmp = w[pa].copy()
+        w[pa] = w[pb]
+        w[pb] = tmp
+        pi[e_a], pi[e_b] = pb, pa
+    return w, pi

@@ -254,6 +254,24 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream);
 /* Kernels this library has launched through `ctx` so far (for benchmarks). */
 uint64_t fb_launch_count(const fb_ctx* ctx);
 
+/* ---- stage 3 on one device (Method overview, "Weight Transfer"): apply a plan to the weights ----
+ * slot_weights is a device buffer of E slot images of expert_bytes each (slot p at byte
+ * offset p * expert_bytes; 16-byte aligned, expert_bytes a multiple of 16); slot p holds the
+ * weights of the expert placed there.  For each of the *n_swaps accepted swaps (device
+ * scalar and device array as written by fb_plan_swaps / fb_predict_and_plan / fb_layer_step;
+ * max_swaps = capacity of the array) the images of the two experts' slots UNDER
+ * expert_to_slot - the placement BEFORE the plan, i.e. the planner's input - are exchanged
+ * in place, so that afterwards every expert's weights sit in the slot the planner's output
+ * placement names.  One launch for the whole plan (swaps of one plan touch disjoint slots);
+ * no staging memory; nothing is read on the host, so the call can follow the planner on the
+ * same stream, or run on another stream behind an event, beside the attention kernels.
+ * The caller keeps the weights unused by other work on the device until the call completes.
+ * status_word (device, optional) receives FB_ERR_RANGE / FB_ERR_BAD_PLACEMENT if a swap or
+ * the placement is out of range (that swap is skipped).  Traffic: 4 * expert_bytes per swap. */
+fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, const int32_t* expert_to_slot,
+                         const fb_swap* swaps, const int32_t* n_swaps, int32_t max_swaps, int32_t* status_word,
+                         fb_stream stream);
+
 /* ---- prediction-quality metrics (Evaluation, "Metrics"); not part of the per-layer hot path ---- */
 #define FB_DTYPE_BF16 0
 #define FB_DTYPE_F32 1

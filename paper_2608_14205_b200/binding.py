@@ -50,7 +50,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
-           "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits"]
+           "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps"]
 
 _lib = None
 
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
     L.fb_row_cosine_mean.argtypes = [vp, vp, ctypes.c_int64, i32, i32, vp, vp, vp]
     L.fb_row_cosine_mean.restype = ctypes.c_int
     L.fb_topk_hits.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.fb_apply_swaps.argtypes = [vp, u64, i32, vp, vp, vp, i32, vp, vp]
+    L.fb_apply_swaps.restype = ctypes.c_int
     L.fb_topk_hits.restype = ctypes.c_int
     L.fb_time_next_router_launch.argtypes = [vp, vp, vp]
     L.fb_time_next_router_launch.restype = ctypes.c_int
@@ -178,6 +180,13 @@ def fb_row_cosine_mean(a: torch.Tensor, b: torch.Tensor, row_scratch: torch.Tens
     dtype = {torch.bfloat16: FB_DTYPE_BF16, torch.float32: FB_DTYPE_F32}[a.dtype]
     _check(lib().fb_row_cosine_mean(_ptr(a), _ptr(b), a.shape[0], a.shape[1], dtype, _ptr(row_scratch),
                                     _ptr(mean_out), _stream(stream)), "fb_row_cosine_mean")
+
+
+def fb_apply_swaps(slot_weights: torch.Tensor, expert_bytes: int, E: int, expert_to_slot: torch.Tensor,
+                   swaps: torch.Tensor, n_swaps: torch.Tensor, max_swaps: int, status_word=None, stream=None) -> None:
+    """Exchange the slot images of every accepted swap in place (stage 3 on one device)."""
+    _check(lib().fb_apply_swaps(_ptr(slot_weights), expert_bytes, E, _ptr(expert_to_slot), _ptr(swaps),
+                                _ptr(n_swaps), max_swaps, _ptr(status_word), _stream(stream)), "fb_apply_swaps")
 
 
 def fb_topk_hits(ids_a: torch.Tensor, ids_b: torch.Tensor, T: int, k: int, hits_out: torch.Tensor,

@@ -10,6 +10,7 @@
 
 #include "../../include/freebalance.h"
 #include "fb_dispatch.cuh"
+#include "fb_migrate.cuh"
 #include "fb_planner.cuh"
 #include "fb_quality.cuh"
 #include "fb_router.cuh"
@@ -644,6 +645,29 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream_) {
 }
 
 uint64_t fb_launch_count(const fb_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, const int32_t* expert_to_slot,
+                         const fb_swap* swaps, const int32_t* n_swaps, int32_t max_swaps, int32_t* status_word,
+                         fb_stream stream_) {
+  if (E < 1 || E > FB_MAX_EXPERTS || max_swaps < 0 || expert_bytes % 16 != 0) return FB_ERR_INVALID_ARG;
+  if (max_swaps == 0 || expert_bytes == 0) return FB_OK;
+  if (!slot_weights || !expert_to_slot || !swaps || !n_swaps) return FB_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(slot_weights) % 16 != 0) return FB_ERR_INVALID_ARG;
+  fb::MigrateParams mp;
+  mp.slot_weights = static_cast<uint8_t*>(slot_weights);
+  mp.expert_bytes = expert_bytes;
+  mp.E = E;
+  mp.expert_to_slot = expert_to_slot;
+  mp.swaps = swaps;
+  mp.n_swaps = n_swaps;
+  mp.status = status_word;
+  const uint64_t per_block = static_cast<uint64_t>(fb::kMigrateThreads) * fb::kMigrateUnroll * 16;
+  uint64_t bx = (expert_bytes + per_block - 1) / per_block;
+  if (bx > fb::kMigrateBlocksPerSwap) bx = fb::kMigrateBlocksPerSwap;
+  const dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(max_swaps), 1);
+  fb::fb_swap_weights_kernel<<<grid, fb::kMigrateThreads, 0, static_cast<cudaStream_t>(stream_)>>>(mp);
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
 
 fb_status fb_row_cosine_mean(const void* a, const void* b, int64_t rows, int32_t n, int32_t dtype,
                              double* row_scratch, double* mean_out, fb_stream stream_) {

@@ -314,6 +314,31 @@ def main():
     barrier()
     pp_ms = [a.elapsed_time(b) for a, b in pp_ev]
 
+    # ---- stage 3 on this device (not part of the step): the plan just produced, applied to a buffer
+    # of E slot images of the workload's expert size; HBM bound, 4 bytes of traffic per byte moved
+    mig = None
+    if not args.no_e2e and wl.expert_bytes > 0 and bkw["max_swaps"] > 0:
+        S = wl.expert_bytes // 16 * 16
+        weights = torch.empty(E * S, dtype=torch.uint8, device=dev)      # content does not matter for timing
+        cap = int(bkw["max_swaps"])
+        L0d = layers[(K - 1) % ring]
+        run_mig = lambda: B.fb_apply_swaps(weights, S, E, L0d["pi"], out["swaps"], out["n_swaps"], cap)
+        for _ in range(3):
+            run_mig()
+        barrier()
+        m_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(10)]
+        for a, b in m_ev:
+            a.record()
+            run_mig()
+            b.record()
+        barrier()
+        n_sw = int(out["n_swaps"].item())
+        m_us = statistics.mean(a.elapsed_time(b) for a, b in m_ev) * 1e3
+        mig = {"kernel": "fb_swap_weights_kernel (fb_apply_swaps)", "swaps": n_sw, "expert_bytes": S,
+               "traffic_bytes": 4 * S * n_sw, "us": m_us,
+               "achieved_GBps": 4 * S * n_sw / (m_us * 1e-6) / 1e9 if m_us > 0 else None}
+        del weights
+
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
     L0 = layers_cpu[0]
     pin = lambda t: t.contiguous().pin_memory()
@@ -411,6 +436,8 @@ def main():
                     roofline(statistics.mean(pp_ms), 2 * T * d + 2 * d * E + 4 * E, 2 * T * d * E,
                              "fb_router_kernel (fb_predict_and_plan alone, one event pair per launch)"),
                     tokens_per_s=T / (statistics.mean(pp_ms) * 1e-3), launches_timed=len(pp_ms)),
+                "migration": None if mig is None else dict(
+                    mig, frac_of_hbm_peak=(mig["achieved_GBps"] / peaks["hbm_gbs"]) if mig["achieved_GBps"] else None),
                 "load_balance": {"predicted_max_over_mean": [mom(lb), mom(la)],
                                  "realized_max_over_mean": [mom(real_before), mom(real_after)],
                                  "n_swaps": int(out["n_swaps"].item())}}

@@ -272,6 +272,21 @@ fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, c
                          const fb_swap* swaps, const int32_t* n_swaps, int32_t max_swaps, int32_t* status_word,
                          fb_stream stream);
 
+/* The same exchange issued from the host as device-to-device copies, the way a serving engine
+ * moves expert weights between ranks: the plan (n_swaps, swaps) and the placement before the
+ * plan are copied to the host on plan_stream, the call WAITS for that stream, and then
+ * enqueues, for every swap, the pairwise exchange through a staging buffer of at most
+ * staging_bytes (0 = one whole expert) on copy_stream: stage <- A, A <- B, B <- stage, piece
+ * by piece.  No kernel of the library runs, so the transfer does not compete for SMs with the
+ * attention kernels it is meant to hide behind.  Returns after the copies are enqueued; the
+ * staging buffer (owned by ctx, grown on demand) and a small pinned host buffer are allocated
+ * on first use.  Traffic: 6 * expert_bytes per swap.  Errors: FB_ERR_RANGE /
+ * FB_ERR_BAD_PLACEMENT for a swap or placement out of range (copies of earlier swaps may
+ * already be enqueued), FB_ERR_CUDA. */
+fb_status fb_apply_swaps_staged(fb_ctx* ctx, void* slot_weights, uint64_t expert_bytes, const int32_t* expert_to_slot,
+                                const fb_swap* swaps, const int32_t* n_swaps, int32_t max_swaps,
+                                uint64_t staging_bytes, fb_stream plan_stream, fb_stream copy_stream);
+
 /* ---- prediction-quality metrics (Evaluation, "Metrics"); not part of the per-layer hot path ---- */
 #define FB_DTYPE_BF16 0
 #define FB_DTYPE_F32 1

@@ -50,7 +50,8 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
-           "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps"]
+           "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
+           "fb_apply_swaps_staged"]
 
 _lib = None
 
@@ -103,6 +104,8 @@ def lib() -> ctypes.CDLL:
     L.fb_topk_hits.argtypes = [vp, vp, i32, i32, vp, vp]
     L.fb_apply_swaps.argtypes = [vp, u64, i32, vp, vp, vp, i32, vp, vp]
     L.fb_apply_swaps.restype = ctypes.c_int
+    L.fb_apply_swaps_staged.argtypes = [vp, vp, u64, vp, vp, vp, i32, u64, vp, vp]
+    L.fb_apply_swaps_staged.restype = ctypes.c_int
     L.fb_topk_hits.restype = ctypes.c_int
     L.fb_time_next_router_launch.argtypes = [vp, vp, vp]
     L.fb_time_next_router_launch.restype = ctypes.c_int
@@ -270,6 +273,12 @@ class Context:
         word = ctypes.c_int32(0)
         _check(lib().fb_device_status(self._h, ctypes.byref(word), _stream(stream)), "fb_device_status")
         return int(word.value)
+
+    def fb_apply_swaps_staged(self, slot_weights, expert_bytes, expert_to_slot, swaps, n_swaps, max_swaps,
+                              staging_bytes=0, plan_stream=None, copy_stream=None) -> None:
+        _check(lib().fb_apply_swaps_staged(self._h, _ptr(slot_weights), expert_bytes, _ptr(expert_to_slot),
+                                           _ptr(swaps), _ptr(n_swaps), max_swaps, staging_bytes,
+                                           _stream(plan_stream), _stream(copy_stream)), "fb_apply_swaps_staged")
 
     def fb_set_pair_limit(self, pairs: int) -> None:
         _check(lib().fb_set_pair_limit(self._h, pairs), "fb_set_pair_limit")

@@ -62,6 +62,9 @@ struct fb_ctx {
   // staging for fb_layer_step_host (allocated on first use)
   bool staged = false;
   void* st_hprev = nullptr; void* st_H = nullptr;
+  // staging for fb_apply_swaps_staged (allocated on first use): pinned host copy of a plan and of the
+  // placement, and one device buffer of mig_stage_bytes
+  void* mig_host = nullptr; void* mig_stage = nullptr; uint64_t mig_stage_bytes = 0;
   int32_t* st_pi = nullptr; int32_t* st_pi_out = nullptr;
   uint32_t* st_counts = nullptr; fb_swap* st_swaps = nullptr; int32_t* st_nswaps = nullptr;
   uint32_t* st_load_before = nullptr; uint32_t* st_load_after = nullptr;
@@ -455,6 +458,8 @@ fb_status fb_destroy(fb_ctx* ctx) {
                   ctx->st_perm, ctx->st_inv_perm, ctx->st_rank_load};
   for (void* p : ptrs)
     if (p) cudaFree(p);
+  if (ctx->mig_stage) cudaFree(ctx->mig_stage);
+  if (ctx->mig_host) cudaFreeHost(ctx->mig_host);
   delete ctx;
   return FB_OK;
 }
@@ -661,12 +666,64 @@ fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, c
   mp.swaps = swaps;
   mp.n_swaps = n_swaps;
   mp.status = status_word;
-  const uint64_t per_block = static_cast<uint64_t>(fb::kMigrateThreads) * fb::kMigrateUnroll * 16;
-  uint64_t bx = (expert_bytes + per_block - 1) / per_block;
-  if (bx > fb::kMigrateBlocksPerSwap) bx = fb::kMigrateBlocksPerSwap;
-  const dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(max_swaps), 1);
+  mp.max_swaps = max_swaps;
+  const uint64_t per_piece = static_cast<uint64_t>(fb::kMigrateThreads) * fb::kMigrateUnroll * 16;
+  uint64_t units = (expert_bytes + per_piece - 1) / per_piece * static_cast<uint64_t>(max_swaps);
+  if (units > fb::kMigrateBlocks) units = fb::kMigrateBlocks;
+  const dim3 grid(static_cast<unsigned>(units), 1, 1);
   fb::fb_swap_weights_kernel<<<grid, fb::kMigrateThreads, 0, static_cast<cudaStream_t>(stream_)>>>(mp);
   return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status fb_apply_swaps_staged(fb_ctx* ctx, void* slot_weights, uint64_t expert_bytes, const int32_t* expert_to_slot,
+                                const fb_swap* swaps, const int32_t* n_swaps, int32_t max_swaps,
+                                uint64_t staging_bytes, fb_stream plan_stream_, fb_stream copy_stream_) {
+  if (!ctx || max_swaps < 0 || max_swaps > FB_MAX_EXPERTS / 2) return FB_ERR_INVALID_ARG;
+  if (max_swaps == 0 || expert_bytes == 0) return FB_OK;
+  if (!slot_weights || !expert_to_slot || !swaps || !n_swaps) return FB_ERR_INVALID_ARG;
+  cudaStream_t plan_stream = static_cast<cudaStream_t>(plan_stream_);
+  cudaStream_t copy_stream = static_cast<cudaStream_t>(copy_stream_);
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  const int E = ctx->cfg.E;
+  if (staging_bytes == 0 || staging_bytes > expert_bytes) staging_bytes = expert_bytes;
+  // host copy of the plan: [n_swaps][swaps: max_swaps][placement: E]
+  const size_t host_bytes = sizeof(int32_t) * (1 + 4 * static_cast<size_t>(FB_MAX_EXPERTS / 2) + FB_MAX_EXPERTS);
+  if (!ctx->mig_host && cudaMallocHost(&ctx->mig_host, host_bytes) != cudaSuccess) return FB_ERR_CUDA;
+  if (ctx->mig_stage_bytes < staging_bytes) {
+    if (ctx->mig_stage) { cudaStreamSynchronize(copy_stream); cudaFree(ctx->mig_stage); ctx->mig_stage = nullptr; }
+    if (cudaMalloc(&ctx->mig_stage, staging_bytes) != cudaSuccess) { ctx->mig_stage_bytes = 0; return FB_ERR_CUDA; }
+    ctx->mig_stage_bytes = staging_bytes;
+  }
+  int32_t* h_n = static_cast<int32_t*>(ctx->mig_host);
+  fb_swap* h_swaps = reinterpret_cast<fb_swap*>(h_n + 1);
+  int32_t* h_pi = h_n + 1 + 4 * (FB_MAX_EXPERTS / 2);
+  bool ok = cudaMemcpyAsync(h_n, n_swaps, sizeof(int32_t), cudaMemcpyDeviceToHost, plan_stream) == cudaSuccess &&
+            cudaMemcpyAsync(h_swaps, swaps, sizeof(fb_swap) * max_swaps, cudaMemcpyDeviceToHost, plan_stream) ==
+                cudaSuccess &&
+            cudaMemcpyAsync(h_pi, expert_to_slot, sizeof(int32_t) * E, cudaMemcpyDeviceToHost, plan_stream) ==
+                cudaSuccess &&
+            cudaStreamSynchronize(plan_stream) == cudaSuccess;       // the host needs the plan to issue the copies
+  if (!ok) return FB_ERR_CUDA;
+  const int n = *h_n;
+  if (n < 0 || n > max_swaps) return FB_ERR_RANGE;
+  uint8_t* base = static_cast<uint8_t*>(slot_weights);
+  for (int i = 0; i < n; ++i) {
+    const int ea = h_swaps[i].expert_src, eb = h_swaps[i].expert_dst;
+    if (ea < 0 || ea >= E || eb < 0 || eb >= E || ea == eb) return FB_ERR_RANGE;
+    const int pa = h_pi[ea], pb = h_pi[eb];
+    if (pa < 0 || pa >= E || pb < 0 || pb >= E || pa == pb) return FB_ERR_BAD_PLACEMENT;
+    uint8_t* A = base + static_cast<uint64_t>(pa) * expert_bytes;
+    uint8_t* Bp = base + static_cast<uint64_t>(pb) * expert_bytes;
+    // pairwise exchange through the bounded staging buffer, one piece at a time
+    for (uint64_t off = 0; off < expert_bytes; off += staging_bytes) {
+      const uint64_t len = expert_bytes - off < staging_bytes ? expert_bytes - off : staging_bytes;
+      ok = ok && cudaMemcpyAsync(ctx->mig_stage, A + off, len, cudaMemcpyDeviceToDevice, copy_stream) == cudaSuccess &&
+           cudaMemcpyAsync(A + off, Bp + off, len, cudaMemcpyDeviceToDevice, copy_stream) == cudaSuccess &&
+           cudaMemcpyAsync(Bp + off, ctx->mig_stage, len, cudaMemcpyDeviceToDevice, copy_stream) == cudaSuccess;
+    }
+  }
+  return ok ? FB_OK : FB_ERR_CUDA;
 }
 
 fb_status fb_row_cosine_mean(const void* a, const void* b, int64_t rows, int32_t n, int32_t dtype,

@@ -86,3 +86,30 @@ def test_empty_plan_bad_arguments_and_bad_swaps():
     with pytest.raises(B.FbError):
         B.fb_apply_swaps(z[1:], 16, 8, i, i, i, 1)                   # misaligned buffer
     B.fb_apply_swaps(z, 64, 8, i, i, i, 0)                           # capacity 0: nothing to do
+
+
+@pytest.mark.parametrize("S,stage", [(4096, 0), (1 << 20, 1 << 18), (3 * 4096 + 16, 4096)])
+def test_staged_exchange_by_device_copies(S, stage):
+    # the host-issued variant: same result, whole-expert staging, pieces, and a ragged last piece
+    wl = I.WORKLOADS["qwen3"]
+    E, R = wl.E, wl.R
+    dev = torch.device("cuda")
+    pi0 = I.random_placement(E, 7).tolist()
+    counts = I.random_counts(E, 60000, 7, zipf_s=1.1).tolist()
+    bud = O.Budget(max_swaps=6, global_ns=2**64 - 1, rank_ns=2**64 - 1, link_ns=2**64 - 1, tau_tokens=0,
+                   gamma_num=1, gamma_den=100, alpha_ns=(0, 0), fs_per_byte=(0, 0), ranks_per_node=0, expert_bytes=0)
+    swaps, pi_new, _, _ = O.plan_swaps(counts, pi0, R, bud)
+    assert len(swaps) >= 2
+    w = np.random.default_rng(2).integers(0, 256, size=(E, S), dtype=np.uint8)
+    sw = np.zeros((8, 4), dtype=np.int32)
+    sw[:len(swaps)] = swaps
+    w_d = torch.from_numpy(w.copy()).to(dev)
+    ctx = B.Context(128, wl.d, E, wl.k, R, wl.gate, wl.n_group, wl.topk_group)
+    side = torch.cuda.Stream()
+    ctx.fb_apply_swaps_staged(w_d, S, torch.tensor(pi0, dtype=torch.int32, device=dev), torch.from_numpy(sw).to(dev),
+                              torch.tensor([len(swaps)], dtype=torch.int32, device=dev), 8, stage,
+                              plan_stream=None, copy_stream=side)
+    side.synchronize()
+    ref, _ = O.apply_swaps(w, pi0, swaps)
+    assert np.array_equal(w_d.cpu().numpy(), ref)
+    ctx.close()

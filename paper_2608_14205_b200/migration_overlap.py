@@ -50,10 +50,22 @@ def main():
     ap.add_argument("--window-us", type=float, default=500.0, help="target duration of the stand-in attention")
     ap.add_argument("--expert-bytes", type=int, default=0, help="0 = the workload's expert size")
     ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--exchange-only", type=int, default=0, metavar="SLOTS",
+                    help="only time fb_apply_swaps: 5 swaps among SLOTS (>= 10) slot images of the expert size")
     args = ap.parse_args()
     wl = I.WORKLOADS[args.workload]
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
+    if args.exchange_only:
+        slots = max(10, args.exchange_only)
+        S = (args.expert_bytes or wl.expert_bytes or 16 * 2**20) // 16 * 16
+        weights = torch.empty(slots * S, dtype=torch.uint8, device=dev)
+        pi = torch.arange(slots, dtype=torch.int32, device=dev)
+        swaps = torch.tensor([[0, 1, 2 * i, 2 * i + 1] for i in range(5)], dtype=torch.int32, device=dev)
+        n_swaps = torch.tensor([5], dtype=torch.int32, device=dev)
+        us = _timed(lambda: B.fb_apply_swaps(weights, S, slots, pi, swaps, n_swaps, 5), args.reps, dev)
+        print(json.dumps(dict(expert_bytes=S, swaps=5, traffic_bytes=20 * S, us=us, GBps=20 * S / us / 1e3)))
+        return
     T, E = wl.T, wl.E
     S = (args.expert_bytes or wl.expert_bytes or 16 * 2**20) // 16 * 16
     li = I.make_layer(wl, 0, 0)

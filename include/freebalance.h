@@ -272,6 +272,24 @@ fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, c
                          const fb_swap* swaps, const int32_t* n_swaps, int32_t max_swaps, int32_t* status_word,
                          fb_stream stream);
 
+/* Cost-model calibration ("Budgeted Expert-Swap Planning": the parameters of Eq. 9 are
+ * calibrated during runtime initialisation).  fb_fit_cost_model fits C = alpha + 2 S / beta
+ * through two timed exchanges of experts of bytes_small and bytes_large each (host
+ * arithmetic, exact): *fs_per_byte = 1/beta in femtoseconds per byte rounded up, *alpha_ns
+ * rounded down and not below zero - the units of fb_budget.  FB_ERR_INVALID_ARG unless
+ * bytes_large > bytes_small and t_large_ns > t_small_ns.
+ * fb_calibrate_exchange takes the two timings itself: it exchanges two slot images of
+ * bytes_small and of bytes_large bytes (slot_weights: device buffer of 2 * bytes_large
+ * bytes, 16-byte aligned; its contents are not preserved),
+ * reps times each after two warm-up runs, keeps the fastest, and fits.  Blocking (it waits
+ * for its own events); allocates 28 bytes of device memory for the duration of the call.
+ * t_small_ns_out / t_large_ns_out (optional) receive the two timings. */
+fb_status fb_fit_cost_model(uint64_t t_small_ns, uint64_t t_large_ns, uint64_t bytes_small, uint64_t bytes_large,
+                            uint64_t* alpha_ns, uint64_t* fs_per_byte);
+fb_status fb_calibrate_exchange(void* slot_weights, uint64_t bytes_small, uint64_t bytes_large, int32_t reps,
+                                uint64_t* alpha_ns, uint64_t* fs_per_byte, uint64_t* t_small_ns_out,
+                                uint64_t* t_large_ns_out, fb_stream stream);
+
 /* The same exchange issued from the host as device-to-device copies, the way a serving engine
  * moves expert weights between ranks: the plan (n_swaps, swaps) and the placement before the
  * plan are copied to the host on plan_stream, the call WAITS for that stream, and then

@@ -35,6 +35,9 @@ itself live in ``tests/test_oracle_*.py``):
                           names holds the expert's original bytes, for every expert),
                           a hand-worked exchange, identity on the empty plan, twice =
                           identity, agreement with ``plan_swaps``' own new placement.
+* ``fit_cost_model``     pinned: exact recovery of alpha and beta from synthetic timings that
+                          follow Eq. 9, the rounding directions, rejection of a non-increasing pair.
+* ``budgets_by_attention_type`` pinned: hand-worked homogeneous and hybrid layer lists (Eq. 10).
 * ``serving_loop``       pinned: placement carry-over checked step by step against
                           ``layer_step`` started from the carried placement, a
                           hand-worked two-step example of the realised-load
@@ -494,3 +497,32 @@ def apply_swaps(slot_weights: np.ndarray, expert_to_slot: Sequence[int], swaps):
         w[pb] = tmp
         pi[e_a], pi[e_b] = pb, pa
     return w, pi
+
+
+# ----------------------------------------------------------------------------
+# Cost-model calibration and per-attention-type budgets ("Budgeted Expert-Swap Planning")
+# ----------------------------------------------------------------------------
+def fit_cost_model(t_small_ns: int, t_large_ns: int, bytes_small: int, bytes_large: int):
+    """Eq. 9 fitted through two timed exchanges of experts of two sizes:
+    C = alpha + (S(e_a) + S(e_b)) / beta with S(e_a) = S(e_b) = bytes.  Returns
+    ``(alpha_ns, fs_per_byte)`` in the planner's integer units: 1/beta rounded up to whole
+    femtoseconds per byte, alpha rounded down to whole nanoseconds and clamped at 0."""
+    d_bytes = 2 * (bytes_large - bytes_small)
+    d_t = t_large_ns - t_small_ns
+    if d_bytes <= 0 or d_t <= 0:
+        raise ValueError("the larger exchange must move more bytes and take longer")
+    inv_beta = Fraction(d_t * 1_000_000, d_bytes)                       # femtoseconds per byte
+    fs_per_byte = -((-inv_beta.numerator) // inv_beta.denominator)      # ceiling
+    alpha = Fraction(t_small_ns) - Fraction(2 * bytes_small) * inv_beta / 1_000_000
+    return max(0, alpha.numerator // alpha.denominator), fs_per_byte
+
+
+def budgets_by_attention_type(layer_types: Sequence[str], profiled_ns: dict, delta_ns: int) -> List[int]:
+    """Eq. 10 per layer: B_l = max(0, T_attn[r(l)] - delta), where r(l) is the first layer with
+    the attention type of layer l and ``profiled_ns`` maps that first layer to its measured time."""
+    first = {}
+    out = []
+    for l, t in enumerate(layer_types):
+        first.setdefault(t, l)
+        out.append(budget_ns(profiled_ns[first[t]], delta_ns))
+    return out

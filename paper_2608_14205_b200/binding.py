@@ -51,7 +51,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
            "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
-           "fb_apply_swaps_staged"]
+           "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange"]
 
 _lib = None
 
@@ -106,6 +106,10 @@ def lib() -> ctypes.CDLL:
     L.fb_apply_swaps.restype = ctypes.c_int
     L.fb_apply_swaps_staged.argtypes = [vp, vp, u64, vp, vp, vp, i32, u64, vp, vp]
     L.fb_apply_swaps_staged.restype = ctypes.c_int
+    L.fb_fit_cost_model.argtypes = [u64, u64, u64, u64, ctypes.POINTER(u64), ctypes.POINTER(u64)]
+    L.fb_fit_cost_model.restype = ctypes.c_int
+    L.fb_calibrate_exchange.argtypes = [vp, u64, u64, i32] + [ctypes.POINTER(u64)] * 4 + [vp]
+    L.fb_calibrate_exchange.restype = ctypes.c_int
     L.fb_topk_hits.restype = ctypes.c_int
     L.fb_time_next_router_launch.argtypes = [vp, vp, vp]
     L.fb_time_next_router_launch.restype = ctypes.c_int
@@ -183,6 +187,24 @@ def fb_row_cosine_mean(a: torch.Tensor, b: torch.Tensor, row_scratch: torch.Tens
     dtype = {torch.bfloat16: FB_DTYPE_BF16, torch.float32: FB_DTYPE_F32}[a.dtype]
     _check(lib().fb_row_cosine_mean(_ptr(a), _ptr(b), a.shape[0], a.shape[1], dtype, _ptr(row_scratch),
                                     _ptr(mean_out), _stream(stream)), "fb_row_cosine_mean")
+
+
+def fb_fit_cost_model(t_small_ns: int, t_large_ns: int, bytes_small: int, bytes_large: int) -> tuple[int, int]:
+    """(alpha_ns, fs_per_byte) of Eq. 9 from two timed exchanges; host arithmetic only."""
+    a, f = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    _check(lib().fb_fit_cost_model(t_small_ns, t_large_ns, bytes_small, bytes_large, ctypes.byref(a),
+                                   ctypes.byref(f)), "fb_fit_cost_model")
+    return int(a.value), int(f.value)
+
+
+def fb_calibrate_exchange(slot_weights: torch.Tensor, bytes_small: int, bytes_large: int, reps: int = 5,
+                          stream=None) -> dict:
+    """Time two exchanges on the device and fit Eq. 9; returns alpha_ns, fs_per_byte and the timings."""
+    vals = [ctypes.c_uint64(0) for _ in range(4)]
+    _check(lib().fb_calibrate_exchange(_ptr(slot_weights), bytes_small, bytes_large, reps,
+                                       *[ctypes.byref(v) for v in vals], _stream(stream)), "fb_calibrate_exchange")
+    return dict(alpha_ns=int(vals[0].value), fs_per_byte=int(vals[1].value), t_small_ns=int(vals[2].value),
+                t_large_ns=int(vals[3].value))
 
 
 def fb_apply_swaps(slot_weights: torch.Tensor, expert_bytes: int, E: int, expert_to_slot: torch.Tensor,

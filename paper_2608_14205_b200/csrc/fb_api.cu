@@ -667,12 +667,79 @@ fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, c
   mp.n_swaps = n_swaps;
   mp.status = status_word;
   mp.max_swaps = max_swaps;
+  mp.copy_bytes = expert_bytes;
   const uint64_t per_piece = static_cast<uint64_t>(fb::kMigrateThreads) * fb::kMigrateUnroll * 16;
   uint64_t units = (expert_bytes + per_piece - 1) / per_piece * static_cast<uint64_t>(max_swaps);
   if (units > fb::kMigrateBlocks) units = fb::kMigrateBlocks;
   const dim3 grid(static_cast<unsigned>(units), 1, 1);
   fb::fb_swap_weights_kernel<<<grid, fb::kMigrateThreads, 0, static_cast<cudaStream_t>(stream_)>>>(mp);
   return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status fb_fit_cost_model(uint64_t t_small_ns, uint64_t t_large_ns, uint64_t bytes_small, uint64_t bytes_large,
+                            uint64_t* alpha_ns, uint64_t* fs_per_byte) {
+  if (!alpha_ns || !fs_per_byte || bytes_large <= bytes_small || t_large_ns <= t_small_ns) return FB_ERR_INVALID_ARG;
+  const unsigned __int128 d_bytes = static_cast<unsigned __int128>(2) * (bytes_large - bytes_small);
+  const unsigned __int128 d_t = t_large_ns - t_small_ns;
+  const unsigned __int128 fs = (d_t * 1000000u + d_bytes - 1) / d_bytes;             // 1 / beta, rounded up
+  if (fs > ~static_cast<uint64_t>(0)) return FB_ERR_RANGE;
+  // alpha = t_small - 2 S_small * d_t / d_bytes, rounded down, not below zero
+  const unsigned __int128 lhs = static_cast<unsigned __int128>(t_small_ns) * d_bytes;
+  const unsigned __int128 rhs = static_cast<unsigned __int128>(2) * bytes_small * d_t;
+  *alpha_ns = lhs > rhs ? static_cast<uint64_t>((lhs - rhs) / d_bytes) : 0;
+  *fs_per_byte = static_cast<uint64_t>(fs);
+  return FB_OK;
+}
+
+fb_status fb_calibrate_exchange(void* slot_weights, uint64_t bytes_small, uint64_t bytes_large, int32_t reps,
+                                uint64_t* alpha_ns, uint64_t* fs_per_byte, uint64_t* t_small_ns_out,
+                                uint64_t* t_large_ns_out, fb_stream stream_) {
+  if (!slot_weights || !alpha_ns || !fs_per_byte || reps < 1 || reps > 1000 || bytes_small == 0 ||
+      bytes_small % 16 != 0 || bytes_large % 16 != 0 || bytes_large <= bytes_small)
+    return FB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  // a one-swap plan over two slots, kept on the device for the duration of the call
+  int32_t* plan = nullptr;                       // [pi: 2][swap: 4][n: 1]
+  if (cudaMalloc(&plan, 7 * sizeof(int32_t)) != cudaSuccess) return FB_ERR_CUDA;
+  const int32_t h_plan[7] = {0, 1, 0, 1, 0, 1, 1};
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  bool ok = cudaMemcpyAsync(plan, h_plan, sizeof(h_plan), cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+            cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess;
+  uint64_t t_ns[2] = {0, 0};
+  const uint64_t sizes[2] = {bytes_small, bytes_large};
+  for (int which = 0; which < 2 && ok; ++which) {
+    // the two images lie bytes_large apart for both sizes: the same addresses are warm in both runs
+    float best = 0.0f;
+    for (int r = 0; r < reps + 2 && ok; ++r) {
+      ok = cudaEventRecord(e0, stream) == cudaSuccess;
+      fb::MigrateParams mp;
+      mp.slot_weights = static_cast<uint8_t*>(slot_weights);
+      mp.expert_bytes = bytes_large;             // slot stride
+      mp.E = 2;
+      mp.expert_to_slot = plan;
+      mp.swaps = reinterpret_cast<const fb_swap*>(plan + 2);
+      mp.n_swaps = plan + 6;
+      mp.max_swaps = 1;
+      mp.status = nullptr;
+      mp.copy_bytes = sizes[which];
+      const uint64_t per_piece = static_cast<uint64_t>(fb::kMigrateThreads) * fb::kMigrateUnroll * 16;
+      uint64_t units = (sizes[which] + per_piece - 1) / per_piece;
+      if (units > fb::kMigrateBlocks) units = fb::kMigrateBlocks;
+      fb::fb_swap_weights_kernel<<<static_cast<unsigned>(units), fb::kMigrateThreads, 0, stream>>>(mp);
+      ok = ok && cudaEventRecord(e1, stream) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess;
+      float ms = 0.0f;
+      ok = ok && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
+      if (r >= 2 && (best == 0.0f || ms < best)) best = ms;          // first two runs warm up; keep the fastest
+    }
+    t_ns[which] = static_cast<uint64_t>(best * 1e6f);
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  cudaFree(plan);
+  if (!ok) return FB_ERR_CUDA;
+  if (t_small_ns_out) *t_small_ns_out = t_ns[0];
+  if (t_large_ns_out) *t_large_ns_out = t_ns[1];
+  return fb_fit_cost_model(t_ns[0], t_ns[1], bytes_small, bytes_large, alpha_ns, fs_per_byte);
 }
 
 fb_status fb_apply_swaps_staged(fb_ctx* ctx, void* slot_weights, uint64_t expert_bytes, const int32_t* expert_to_slot,

@@ -23,7 +23,8 @@ constexpr int kMigrateBlocks = 148 * 8;   // fixed grid: blocks stride over (swa
 
 struct MigrateParams {
   uint8_t* slot_weights;          // [E][expert_bytes], slot major
-  uint64_t expert_bytes;          // multiple of 16
+  uint64_t expert_bytes;          // distance between slot images, multiple of 16
+  uint64_t copy_bytes;            // bytes exchanged per image (= expert_bytes except when calibrating)
   int32_t E;
   const int32_t* expert_to_slot;  // [E] placement BEFORE the plan
   const fb_swap* swaps;           // [max_swaps]
@@ -35,7 +36,7 @@ struct MigrateParams {
 __global__ void __launch_bounds__(kMigrateThreads)
 fb_swap_weights_kernel(const __grid_constant__ MigrateParams p) {
   const int n = min(*p.n_swaps, p.max_swaps);
-  const uint64_t n_vec = p.expert_bytes / 16;
+  const uint64_t n_vec = p.copy_bytes / 16;
   const uint64_t per_piece = static_cast<uint64_t>(kMigrateThreads) * kMigrateUnroll;
   const uint64_t pieces = (n_vec + per_piece - 1) / per_piece;      // per swap
   const uint64_t total = pieces * static_cast<uint64_t>(n > 0 ? n : 0);

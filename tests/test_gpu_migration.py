@@ -113,3 +113,29 @@ def test_staged_exchange_by_device_copies(S, stage):
     ref, _ = O.apply_swaps(w, pi0, swaps)
     assert np.array_equal(w_d.cpu().numpy(), ref)
     ctx.close()
+
+
+def test_calibration_predicts_the_exchange_time():
+    dev = torch.device("cuda")
+    small, large = 1 << 20, 44_040_192
+    buf = torch.empty(2 * large, dtype=torch.uint8, device=dev)
+    cal = B.fb_calibrate_exchange(buf, small, large, reps=5)
+    assert cal["t_large_ns"] > cal["t_small_ns"] > 0
+    assert (cal["alpha_ns"], cal["fs_per_byte"]) == O.fit_cost_model(cal["t_small_ns"], cal["t_large_ns"], small, large)
+    gbps = 1e6 / cal["fs_per_byte"]                                  # bytes per ns = GB/s moved per direction
+    assert 500 < gbps < 8000 and cal["alpha_ns"] < 50_000, cal
+    # the fitted model, handed to the planner's cost function, reproduces an independent measurement
+    bud = B.make_budget(max_swaps=4, alpha_ns=(cal["alpha_ns"],) * 2, fs_per_byte=(cal["fs_per_byte"],) * 2,
+                        expert_bytes=16 << 20)
+    predicted = B.fb_swap_cost_ns(bud, 0, 1)
+    w = torch.empty(2 * (16 << 20), dtype=torch.uint8, device=dev)
+    pi = torch.arange(2, dtype=torch.int32, device=dev)
+    sw = torch.tensor([[0, 1, 0, 1]], dtype=torch.int32, device=dev)
+    n = torch.tensor([1], dtype=torch.int32, device=dev)
+    best = 1e9
+    for _ in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); B.fb_apply_swaps(w, 16 << 20, 2, pi, sw, n, 1); b.record()
+        torch.cuda.synchronize()
+        best = min(best, a.elapsed_time(b) * 1e6)
+    assert 0.6 * best < predicted < 1.6 * best, (predicted, best, cal)

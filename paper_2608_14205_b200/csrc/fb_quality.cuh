@@ -18,20 +18,52 @@ __device__ __forceinline__ double load_as_double(const __nv_bfloat16* p, long lo
 }
 __device__ __forceinline__ double load_as_double(const float* p, long long i) { return static_cast<double>(p[i]); }
 
-// One warp per row: lane l takes elements l, l + 32, ...; the three partial sums are
-// combined by a butterfly, which gives every lane the same total.
+// 16 bytes of a row as doubles: 8 bf16 or 4 f32 values.
+__device__ __forceinline__ int unpack16(const __nv_bfloat16* p, long long i, double (&v)[8]) {
+  const uint4 q = *reinterpret_cast<const uint4*>(p + i);
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    v[2 * t] = static_cast<double>(__uint_as_float(w[t] << 16));              // low half = element 2t
+    v[2 * t + 1] = static_cast<double>(__uint_as_float(w[t] & 0xffff0000u));
+  }
+  return 8;
+}
+__device__ __forceinline__ int unpack16(const float* p, long long i, double (&v)[8]) {
+  const float4 q = *reinterpret_cast<const float4*>(p + i);
+  v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+  return 4;
+}
+
+// One warp per row.  Rows whose start and length allow it are read 16 bytes per lane and
+// step (kVec elements); otherwise lane l takes elements l, l + 32, ...  Either way a lane
+// adds its elements in ascending order and the three partial sums are combined by a
+// butterfly, which gives every lane the same total.
 template <class Tin>
 __global__ void __launch_bounds__(32 * kCosineWarpsPerBlock)
 fb_row_cosine_kernel(const Tin* __restrict__ a, const Tin* __restrict__ b, long long rows, int n,
                      double* __restrict__ row_cos) {
+  constexpr int kVec = 16 / static_cast<int>(sizeof(Tin));
   const long long row = static_cast<long long>(blockIdx.x) * kCosineWarpsPerBlock + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
   const long long base = row * n;
   double dot = 0.0, na = 0.0, nb = 0.0;
-  for (int j = lane; j < n; j += 32) {
-    const double x = load_as_double(a, base + j), y = load_as_double(b, base + j);
-    dot += x * y; na += x * x; nb += y * y;
+  const bool wide = n % kVec == 0 && reinterpret_cast<uintptr_t>(a) % 16 == 0 && reinterpret_cast<uintptr_t>(b) % 16 == 0;
+  if (wide) {
+    for (int j = lane * kVec; j < n; j += 32 * kVec) {
+      double x[8], y[8];
+      const int m = unpack16(a, base + j, x);
+      unpack16(b, base + j, y);
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+        if (t < m) { dot += x[t] * y[t]; na += x[t] * x[t]; nb += y[t] * y[t]; }
+    }
+  } else {
+    for (int j = lane; j < n; j += 32) {
+      const double x = load_as_double(a, base + j), y = load_as_double(b, base + j);
+      dot += x * y; na += x * x; nb += y * y;
+    }
   }
 #pragma unroll
   for (int off = 16; off >= 1; off >>= 1) {

@@ -462,3 +462,44 @@ def test_router_launch_events_and_pair_queries():
     with pytest.raises(Exception):
         tiny.fb_set_pair_limit(-1)
     tiny.close()
+
+
+def test_two_contexts_on_two_streams_do_not_interfere():
+    # each context owns its scratch: calls of different contexts may overlap on the device
+    wl = I.WORKLOADS["dsv3"]
+    T = 1500
+    dev = torch.device("cuda")
+    layers = [I.make_layer(wl, l, 0, T=T) for l in (0, 1)]
+    ctxs = [P.make_context(wl, T) for _ in layers]
+    streams = [torch.cuda.Stream() for _ in layers]
+    budget = B.make_budget(**P.budget_kwargs(wl, T))
+    i32 = lambda n: torch.zeros(n, dtype=torch.int32, device=dev)
+
+    def buffers():
+        return dict(counts=i32(wl.E), pi_out=i32(wl.E), swaps=i32(4 * 128), n=i32(1), lb=i32(wl.R), la=i32(wl.R),
+                    ids=i32(T * wl.k), w=torch.zeros(T * wl.k, device=dev), so=i32(wl.E + 1), ro=i32(wl.R + 1),
+                    perm=i32(T * wl.k), inv=i32(T * wl.k), rl=i32(wl.R))
+
+    def call(ctx, li_dev, o, stream):
+        ctx.fb_layer_step(li_dev["router"], li_dev["h"], li_dev["H"], T, li_dev["pi"], budget, 0, o["counts"],
+                          o["pi_out"], o["swaps"], o["n"], o["lb"], o["la"], o["ids"], o["w"], o["so"], o["ro"],
+                          o["perm"], o["inv"], o["rl"], stream=stream)
+
+    devs = [dict(router=B.make_router(li.W.to(dev), None, li.select_bias.to(dev)), h=li.h_prev.to(dev),
+                 H=li.H.to(dev), pi=li.expert_to_slot.to(dev)) for li in layers]
+    serial = [buffers() for _ in layers]
+    for ctx, d, o in zip(ctxs, devs, serial):
+        call(ctx, d, o, None)
+        torch.cuda.synchronize()
+    overlapped = [buffers() for _ in layers]
+    torch.cuda.synchronize()
+    for rep in range(5):
+        for ctx, d, o, st in zip(ctxs, devs, overlapped, streams):
+            call(ctx, d, o, st)
+    torch.cuda.synchronize()
+    for a, b in zip(serial, overlapped):
+        for key in a:
+            assert torch.equal(a[key], b[key]), key
+    assert all(c.fb_device_status() == 0 for c in ctxs)
+    for c in ctxs:
+        c.close()

@@ -128,6 +128,7 @@ __device__ __forceinline__ float fb_sigmoid(float z) {
 // group scores and group lower bounds [32][128] each, partial top-k lists of subs 1..,
 // partial softmax sums.
 constexpr int kCandCap = 32;           // candidates per row the fast selection path can hold
+constexpr int kBoundRows = 8;          // chunks per row on that path, at most (rows of the bound tables)
 __host__ __device__ constexpr size_t epilogue_scratch_bytes(int N) {
   return (static_cast<size_t>(N) * kTileM + 2 * FB_MAX_GROUPS * kTileM + 2 * kCandCap * kTileM) * 4;
 }
@@ -564,20 +565,26 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             m1 = -INFINITY; m2 = -INFINITY;
           }
         } else if (!sigmoid_gate && fast_select) {
-          // softmax gate, fast selection: the chunk's second-best key is what the bound needs
-          float a1[16], a2[16];
+          // softmax gate, fast selection: the chunk's three best keys (sorted) feed the bound
+          float a1[16], a2[16], a3[16];
 #pragma unroll
-          for (int j = 0; j < 16; ++j) { a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); }
+          for (int j = 0; j < 16; ++j) {
+            a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); a3[j] = -INFINITY;
+          }
 #pragma unroll
           for (int w = 8; w >= 1; w >>= 1) {
 #pragma unroll
             for (int j = 0; j < w; ++j) {
-              const float hi = fmaxf(a1[j], a1[j + w]);
-              a2[j] = fmaxf(fminf(a1[j], a1[j + w]), fmaxf(a2[j], a2[j + w]));
-              a1[j] = hi;
+              // best three of two sorted triples
+              const float lo1 = fminf(a1[j], a1[j + w]), hi2 = fmaxf(a2[j], a2[j + w]);
+              a1[j] = fmaxf(a1[j], a1[j + w]);
+              a2[j] = fmaxf(lo1, hi2);
+              a3[j] = fmaxf(fminf(lo1, hi2), fmaxf(a3[j], a3[j + w]));
             }
           }
-          glow_s[c * kTileM + row_in_tile] = a2[0];
+          gscore_s[c * kTileM + row_in_tile] = a1[0];
+          gscore_s[(kBoundRows + c) * kTileM + row_in_tile] = a2[0];
+          gscore_s[(2 * kBoundRows + c) * kTileM + row_in_tile] = a3[0];
         } else if (sigmoid_gate) {
           int g = c0 / gs, pos = c0 % gs;
 #pragma unroll
@@ -618,12 +625,20 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           }
         }
       } else {
-        for (int c = 0; c < n_chunks; ++c) floor_key = fminf(floor_key, glow_s[c * kTileM + row_in_tile]);
+        // bound for the k-th key: the k-th largest of the chunks' three best keys (3 n_chunks >= k of them)
+        TopK known;
+        known.init();
+        for (int i = 0; i < 3 * kBoundRows; ++i) {
+          const float x = (i % kBoundRows) < n_chunks ? gscore_s[i * kTileM + row_in_tile] : -INFINITY;
+          if (x > known.v[FB_MAX_TOPK - 1]) known.insert(x, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < FB_MAX_TOPK; ++j)
+          if (j == k - 1) floor_key = known.v[j];
         if (sub < n_chunks) my_groups[0] = sub;
         if (sub + kEpiSubs < n_chunks) my_groups[1] = sub + kEpiSubs;
       }
-      // ---------------- collect the keys >= floor (the kept groups' two best keys are >= floor,
-      // so at least k keys qualify)
+      // ---------------- collect the keys >= floor (at least k keys qualify: the bound is one of k known keys)
 #pragma unroll 1
       for (int gi = 0; gi < 2; ++gi) {
         if (my_groups[gi] < 0) continue;                  // no such group: true for the whole warp at once

@@ -260,8 +260,11 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.numAttrs = 2;
-    err = persistent ? cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel, *mx, *mx2, *mw, p)
-                     : cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mx2, *mw, p);
+    if (!persistent) err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mx2, *mw, p);
+    else if (c.gate == FB_GATE_SIGMOID_GROUP_TOPK)
+      err = cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel<true>, *mx, *mx2, *mw, p);
+    else
+      err = cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel<false>, *mx, *mx2, *mw, p);
   } else {
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
     err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1>, *mx, *mx2, *mw, p);
@@ -414,7 +417,9 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   bool ok = true;
   if (ctx->persist_stages >= 2) {
-    ok = cudaFuncSetAttribute(fb::fb_router_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    ok = cudaFuncSetAttribute(fb::fb_router_persistent_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(ctx->persist_smem)) == cudaSuccess &&
+         cudaFuncSetAttribute(fb::fb_router_persistent_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(ctx->persist_smem)) == cudaSuccess;
     // how many block pairs the GPU holds at once (the grid of the persistent kernel)
     cudaLaunchConfig_t occ;
@@ -428,7 +433,10 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
     occ.attrs = cl;
     occ.numAttrs = 1;
     int n_clusters = 0;
-    if (ok && cudaOccupancyMaxActiveClusters(&n_clusters, fb::fb_router_persistent_kernel, &occ) == cudaSuccess &&
+    const bool sig = cfg->gate == FB_GATE_SIGMOID_GROUP_TOPK;
+    if (ok && (sig ? cudaOccupancyMaxActiveClusters(&n_clusters, fb::fb_router_persistent_kernel<true>, &occ)
+                   : cudaOccupancyMaxActiveClusters(&n_clusters, fb::fb_router_persistent_kernel<false>, &occ)) ==
+                  cudaSuccess &&
         n_clusters >= 1)
       ctx->max_pairs = n_clusters;
     else

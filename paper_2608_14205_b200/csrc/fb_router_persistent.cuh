@@ -8,7 +8,7 @@
 //     into registers (64 columns per thread), hand tensor memory back to the MMA issuers
 //     at once, and do all gating / selection work from registers;
 //   * the epilogue's shared-memory scratch (group scores, candidate lists) has its own
-//     40 KB behind the pipeline stages instead of reusing them.
+//     44 KB behind the pipeline stages instead of reusing them.
 // Restricted to the gates the ranking selection handles (DeepSeek-V3-like sigmoid gates with
 // 32-expert groups, softmax gates over whole 32-column chunks); everything else, and
 // every call that fits one tile per block, runs fb_router_kernel.  Arithmetic, summation
@@ -24,7 +24,7 @@ namespace fb {
 
 constexpr int kPersistGroups = 8;            // 32-column chunks (= groups) per row, at most
 constexpr size_t kPersistScratchBytes =
-    (2 * kPersistGroups * kTileM + 2 * kCandCap * kTileM) * sizeof(float);   // 40 KB
+    (3 * kPersistGroups * kTileM + 2 * kCandCap * kTileM) * sizeof(float);   // 44 KB
 static_assert(2 * kCandCap >= 2 * (kEpiSubs - 1) * FB_MAX_TOPK, "merge lists must fit in the candidate area");
 static_assert(2 * kPersistGroups >= 2 * FB_MAX_TOPK, "result lists must fit in the group-score area");
 
@@ -59,6 +59,9 @@ __device__ __forceinline__ void ring_advance(int& s, uint32_t& phase, int stages
   if (++s == stages) { s = 0; phase ^= 1u; }
 }
 
+// kSigmoid: sigmoid + bias group-limited gate (true) or softmax gate (false); one instance per
+// gate keeps each one's code and register allocation to what that gate needs.
+template <bool kSigmoid>
 __global__ void __launch_bounds__(kRouterThreads, 1)
 fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x2,
                             const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ RouterParams p) {
@@ -186,7 +189,7 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     const int row_in_tile = quarter * 32 + lane;
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     const int E = p.E, N = p.N, k = p.k;
-    const bool sigmoid_gate = p.gate != FB_GATE_SOFTMAX_TOPK;
+    constexpr bool sigmoid_gate = kSigmoid;
     const int n_chunks = E >> 5;                           // E is a multiple of 32 here
     const bool has_lb = p.logit_bias != nullptr;
     const bool two_acc = p.num_kb > 1;
@@ -194,8 +197,9 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     float* gscore_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) +
                                                static_cast<size_t>(p.stages) * stage_bytes);   // [8][128]
     float* glow_s = gscore_s + kPersistGroups * kTileM;                                         // [8][128]
+    float* third_s = glow_s + kPersistGroups * kTileM;                                          // [8][128]
     // candidates [32][128]: ordered key bits in the high word, ~expert id in the low word
-    unsigned long long* cand = reinterpret_cast<unsigned long long*>(glow_s + kPersistGroups * kTileM);
+    unsigned long long* cand = reinterpret_cast<unsigned long long*>(third_s + kPersistGroups * kTileM);
     uint32_t* out_hi = reinterpret_cast<uint32_t*>(gscore_s);   // [8][128]: group scores are dead by then
     uint32_t* out_lo = reinterpret_cast<uint32_t*>(glow_s);
     float* merge_v = reinterpret_cast<float*>(cand);            // [3][8][128]: candidates are dead by then
@@ -281,24 +285,36 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
 #pragma unroll
             for (int j = 0; j < 32; ++j) key[ci][j] = key[ci][j] + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
           }
-          float m1[4], m2[4];                                // four interleaved running (best, second) pairs
+          // four interleaved running (best, second, third) triples; the third only feeds the
+          // softmax gate's bound
+          float m1[4], m2[4], m3[4];
 #pragma unroll
-          for (int a = 0; a < 4; ++a) { m1[a] = -INFINITY; m2[a] = -INFINITY; }
+          for (int a = 0; a < 4; ++a) { m1[a] = -INFINITY; m2[a] = -INFINITY; m3[a] = -INFINITY; }
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            m2[j & 3] = fmaxf(m2[j & 3], fminf(m1[j & 3], key[ci][j]));
+            const float t = fminf(m1[j & 3], key[ci][j]);
+            if (!sigmoid_gate) m3[j & 3] = fmaxf(m3[j & 3], fminf(m2[j & 3], t));
+            m2[j & 3] = fmaxf(m2[j & 3], t);
             m1[j & 3] = fmaxf(m1[j & 3], key[ci][j]);
           }
 #pragma unroll
           for (int a = 2; a >= 1; a >>= 1) {
 #pragma unroll
             for (int b = 0; b < a; ++b) {
-              m2[b] = fmaxf(fminf(m1[b], m1[b + a]), fmaxf(m2[b], m2[b + a]));
+              // best three of two sorted triples
+              const float lo1 = fminf(m1[b], m1[b + a]), hi2 = fmaxf(m2[b], m2[b + a]);
+              if (!sigmoid_gate) m3[b] = fmaxf(fminf(lo1, hi2), fmaxf(m3[b], m3[b + a]));
+              m2[b] = fmaxf(lo1, hi2);
               m1[b] = fmaxf(m1[b], m1[b + a]);
             }
           }
           glow_s[c * kTileM + row_in_tile] = m2[0];
-          if (sigmoid_gate) gscore_s[c * kTileM + row_in_tile] = m1[0] + m2[0];   // group score (gs == 32)
+          if (sigmoid_gate) {
+            gscore_s[c * kTileM + row_in_tile] = m1[0] + m2[0];   // group score (gs == 32)
+          } else {
+            gscore_s[c * kTileM + row_in_tile] = m1[0];
+            third_s[c * kTileM + row_in_tile] = m3[0];
+          }
         }
       }
       named_bar_sync(kPlanBarrierId, kEpilogueThreads);
@@ -322,11 +338,23 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
           }
         }
       } else {
-        for (int c = 0; c < n_chunks; ++c) floor_key = fminf(floor_key, glow_s[c * kTileM + row_in_tile]);
+        // the k-th largest of the chunks' three best keys (3 n_chunks >= k of them)
+        TopK known;
+        known.init();
+        for (int c = 0; c < n_chunks; ++c) {
+          const float t1 = gscore_s[c * kTileM + row_in_tile], t2 = glow_s[c * kTileM + row_in_tile];
+          const float t3 = third_s[c * kTileM + row_in_tile];
+          if (t1 > known.v[FB_MAX_TOPK - 1]) known.insert(t1, 0);
+          if (t2 > known.v[FB_MAX_TOPK - 1]) known.insert(t2, 0);
+          if (t3 > known.v[FB_MAX_TOPK - 1]) known.insert(t3, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < FB_MAX_TOPK; ++j)
+          if (j == k - 1) floor_key = known.v[j];
         kept = (1u << n_chunks) - 1u;
       }
-      // ---------------- collect the keys >= floor of this thread's kept chunks (the kept groups'
-      // two best keys are >= floor, so at least k keys qualify in the row)
+      // ---------------- collect the keys >= floor of this thread's kept chunks (the bound is one of
+      // k known keys of the row, so at least k keys qualify)
 #pragma unroll
       for (int ci = 0; ci < 2; ++ci) {
         const int c = sub + kEpiSubs * ci;

@@ -224,6 +224,10 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.ticket_target = tiles_pad;
   // More tile pairs than block pairs fit on the GPU (or than the caller allows): the
   // persistent kernel walks several tiles per block pair and overlaps their epilogues.
+  // selection code of this launch: the ranking selection only if it applies to every block
+  // (in layer mode the normal pass writes weights, the early pass does not)
+  const int sel = fb::select_kind(c.E, ctx->N, c.k, c.gate, p.n_group, p.topk_group,
+                                  topk_w != nullptr && !c.renorm && c.gate == FB_GATE_SOFTMAX_TOPK);
   bool persistent = false;
   if (pair && ctx->persist_stages >= 2 && logits == nullptr) {
     const bool want_sum = topk_w != nullptr && !c.renorm && c.gate == FB_GATE_SOFTMAX_TOPK;
@@ -260,14 +264,24 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.numAttrs = 2;
-    if (!persistent) err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2>, *mx, *mx2, *mw, p);
+    if (!persistent) {
+      err = sel == fb::kSelectSigmoidRank
+                ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2, fb::kSelectSigmoidRank>, *mx, *mx2, *mw, p)
+            : sel == fb::kSelectSoftmaxRank
+                ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2, fb::kSelectSoftmaxRank>, *mx, *mx2, *mw, p)
+                : cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2, fb::kSelectGeneral>, *mx, *mx2, *mw, p);
+    }
     else if (c.gate == FB_GATE_SIGMOID_GROUP_TOPK)
       err = cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel<true>, *mx, *mx2, *mw, p);
     else
       err = cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel<false>, *mx, *mx2, *mw, p);
   } else {
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
-    err = cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1>, *mx, *mx2, *mw, p);
+    err = sel == fb::kSelectSigmoidRank
+              ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1, fb::kSelectSigmoidRank>, *mx, *mx2, *mw, p)
+          : sel == fb::kSelectSoftmaxRank
+              ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1, fb::kSelectSoftmaxRank>, *mx, *mx2, *mw, p)
+              : cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1, fb::kSelectGeneral>, *mx, *mx2, *mw, p);
   }
   if (ctx->ev_after) cudaEventRecord(ctx->ev_after, stream);
   ctx->ev_before = ctx->ev_after = nullptr;
@@ -342,11 +356,15 @@ static fb_status setup_router_shape(fb_ctx* ctx, const cudaDeviceProp& prop) {
     ctx->smem_bytes[pair] = dyn + 1024;
   }
   ctx->max_tiles = (cfg.T_max + fb::kTileM - 1) / fb::kTileM;
-  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(ctx->smem_bytes[0])) == cudaSuccess;
+  const int bytes1 = static_cast<int>(ctx->smem_bytes[0]), bytes2 = static_cast<int>(ctx->smem_bytes[1]);
+  const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1, fb::kSelectGeneral>, attr, bytes1) == cudaSuccess &&
+            cudaFuncSetAttribute(fb::fb_router_kernel<1, fb::kSelectSigmoidRank>, attr, bytes1) == cudaSuccess &&
+            cudaFuncSetAttribute(fb::fb_router_kernel<1, fb::kSelectSoftmaxRank>, attr, bytes1) == cudaSuccess;
   if (ctx->stages[1] >= 2)
-    ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    static_cast<int>(ctx->smem_bytes[1])) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2, fb::kSelectGeneral>, attr, bytes2) == cudaSuccess &&
+         cudaFuncSetAttribute(fb::fb_router_kernel<2, fb::kSelectSigmoidRank>, attr, bytes2) == cudaSuccess &&
+         cudaFuncSetAttribute(fb::fb_router_kernel<2, fb::kSelectSoftmaxRank>, attr, bytes2) == cudaSuccess;
   return ok ? FB_OK : FB_ERR_CUDA;
 }
 

@@ -135,6 +135,20 @@ __host__ __device__ constexpr size_t epilogue_scratch_bytes(int N) {
 
 static_assert(2 * kCandCap >= 2 * (kEpiSubs - 1) * FB_MAX_TOPK + kEpiSubs * 2, "merge area must fit in the candidate area");
 
+// Which selection code a launch needs.  The ranking selection applies to DeepSeek-V3-like
+// sigmoid gates (groups of exactly one 32-column chunk, at most 8 groups, at most kEpiSubs
+// kept, two known keys per kept group >= k) and to softmax gates over whole chunks (every
+// chunk counts as a kept group; not when the softmax denominator is needed, i.e. weights
+// without renormalisation).  Everything else takes the general insertion code.
+enum SelectKind : int { kSelectGeneral = 0, kSelectSigmoidRank = 1, kSelectSoftmaxRank = 2 };
+__host__ __device__ inline int select_kind(int E, int N, int k, int gate, int n_group, int topk_group, bool want_sum) {
+  if (gate != FB_GATE_SOFTMAX_TOPK)
+    return (E / n_group == 32 && E % n_group == 0 && n_group <= 8 && topk_group <= kEpiSubs && topk_group * 2 >= k)
+               ? kSelectSigmoidRank : kSelectGeneral;
+  const int n_chunks = (N + 31) >> 5;
+  return (E % 32 == 0 && n_chunks <= 8 && n_chunks * 2 >= k && !want_sum) ? kSelectSoftmaxRank : kSelectGeneral;
+}
+
 struct RouterShared {
   uint64_t full_bar[kMaxStages];
   uint64_t empty_bar[kMaxStages];
@@ -292,7 +306,9 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32
 // of the W tile, which halves the W traffic out of L2 and leaves room for more pipeline
 // stages.  The even block of the pair issues the MMAs and owns the "full" barriers;
 // both blocks get their stage-free and accumulator-ready signals from its commits.
-template <int kCtas>
+// kSel (SelectKind): one instance per selection code, so that each carries only the code and
+// the registers its gate needs; the host picks it with select_kind().
+template <int kCtas, int kSel>
 __global__ void __launch_bounds__(kRouterThreads, 1)
 fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x2,
                  const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ RouterParams p) {
@@ -422,20 +438,16 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const bool valid = row < p.T;
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     const int E = p.E, N = p.N, k = p.k;
-    const bool sigmoid_gate = p.gate != FB_GATE_SOFTMAX_TOPK;
-    const int gs = sigmoid_gate ? E / p.n_group : E;       // experts per group
+    const bool sigmoid_gate = kSel == kSelectSigmoidRank ? true
+                              : kSel == kSelectSoftmaxRank ? false : p.gate != FB_GATE_SOFTMAX_TOPK;
+    const int gs = kSel == kSelectSigmoidRank ? 32 : (sigmoid_gate ? E / p.n_group : E);   // experts per group
     // Which sub owns chunk c: whole groups must stay with one sub.
     const int n_chunks = (N + 31) >> 5;
     const int chunks_per_group = (sigmoid_gate && gs % 32 == 0) ? gs / 32 : 1;
     const bool splittable = !sigmoid_gate || gs % 32 == 0 || 32 % gs == 0;
-    const bool want_sum = out_w != nullptr && !p.renorm && !sigmoid_gate;
-    // Selection by ranking a short candidate list instead of insertion.  Applies to
-    // DeepSeek-V3-like gates (groups of exactly one chunk, few groups kept) and to softmax
-    // gates over whole chunks, where every chunk counts as a kept group; needs at least k
-    // known keys (two per kept group) for the lower bound of the k-th key.
-    const bool fast_select =
-        sigmoid_gate ? (gs == 32 && p.n_group <= 8 && p.topk_group <= kEpiSubs && p.topk_group * 2 >= k)
-                     : (E % 32 == 0 && n_chunks <= 8 && n_chunks * 2 >= k && !want_sum);
+    const bool want_sum = kSel == kSelectGeneral && out_w != nullptr && !p.renorm && !sigmoid_gate;
+    // Selection by ranking a short candidate list instead of insertion (see select_kind).
+    constexpr bool fast_select = kSel != kSelectGeneral;
 
     // Chunk bookkeeping, worked out while the main loop runs (integer divisions by run-time
     // values are slow and would otherwise sit between the chunks of the epilogue):

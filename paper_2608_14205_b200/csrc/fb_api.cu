@@ -176,6 +176,24 @@ fb_status fill_plan(const fb_ctx* ctx, const fb_budget* b, const int32_t* pi, in
   return FB_OK;
 }
 
+// Kernel instances by (selection kind, logit bias present).
+using RouterKernelFn = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, fb::RouterParams);
+template <int kCtas>
+static RouterKernelFn router_kernel_fn(int sel, bool lb) {
+  switch (sel * 2 + (lb ? 1 : 0)) {
+    case 0: return fb::fb_router_kernel<kCtas, fb::kSelectGeneral, false>;
+    case 1: return fb::fb_router_kernel<kCtas, fb::kSelectGeneral, true>;
+    case 2: return fb::fb_router_kernel<kCtas, fb::kSelectSigmoidRank, false>;
+    case 3: return fb::fb_router_kernel<kCtas, fb::kSelectSigmoidRank, true>;
+    case 4: return fb::fb_router_kernel<kCtas, fb::kSelectSoftmaxRank, false>;
+    default: return fb::fb_router_kernel<kCtas, fb::kSelectSoftmaxRank, true>;
+  }
+}
+static RouterKernelFn persistent_kernel_fn(bool sigmoid, bool lb) {
+  if (sigmoid) return lb ? fb::fb_router_persistent_kernel<true, true> : fb::fb_router_persistent_kernel<true, false>;
+  return lb ? fb::fb_router_persistent_kernel<false, true> : fb::fb_router_persistent_kernel<false, false>;
+}
+
 // Launch the router kernel in one of its three modes.
 // x2 is the second input of kModeLayer (the normal router input), nullptr otherwise.
 fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T, int mode,
@@ -264,24 +282,12 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.numAttrs = 2;
-    if (!persistent) {
-      err = sel == fb::kSelectSigmoidRank
-                ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2, fb::kSelectSigmoidRank>, *mx, *mx2, *mw, p)
-            : sel == fb::kSelectSoftmaxRank
-                ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2, fb::kSelectSoftmaxRank>, *mx, *mx2, *mw, p)
-                : cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<2, fb::kSelectGeneral>, *mx, *mx2, *mw, p);
-    }
-    else if (c.gate == FB_GATE_SIGMOID_GROUP_TOPK)
-      err = cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel<true>, *mx, *mx2, *mw, p);
-    else
-      err = cudaLaunchKernelEx(&cfg, fb::fb_router_persistent_kernel<false>, *mx, *mx2, *mw, p);
+    const bool lb = router->logit_bias != nullptr;
+    err = cudaLaunchKernelEx(&cfg, persistent ? persistent_kernel_fn(c.gate == FB_GATE_SIGMOID_GROUP_TOPK, lb)
+                                              : router_kernel_fn<2>(sel, lb), *mx, *mx2, *mw, p);
   } else {
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
-    err = sel == fb::kSelectSigmoidRank
-              ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1, fb::kSelectSigmoidRank>, *mx, *mx2, *mw, p)
-          : sel == fb::kSelectSoftmaxRank
-              ? cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1, fb::kSelectSoftmaxRank>, *mx, *mx2, *mw, p)
-              : cudaLaunchKernelEx(&cfg, fb::fb_router_kernel<1, fb::kSelectGeneral>, *mx, *mx2, *mw, p);
+    err = cudaLaunchKernelEx(&cfg, router_kernel_fn<1>(sel, router->logit_bias != nullptr), *mx, *mx2, *mw, p);
   }
   if (ctx->ev_after) cudaEventRecord(ctx->ev_after, stream);
   ctx->ev_before = ctx->ev_after = nullptr;
@@ -358,13 +364,15 @@ static fb_status setup_router_shape(fb_ctx* ctx, const cudaDeviceProp& prop) {
   ctx->max_tiles = (cfg.T_max + fb::kTileM - 1) / fb::kTileM;
   const int bytes1 = static_cast<int>(ctx->smem_bytes[0]), bytes2 = static_cast<int>(ctx->smem_bytes[1]);
   const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-  bool ok = cudaFuncSetAttribute(fb::fb_router_kernel<1, fb::kSelectGeneral>, attr, bytes1) == cudaSuccess &&
-            cudaFuncSetAttribute(fb::fb_router_kernel<1, fb::kSelectSigmoidRank>, attr, bytes1) == cudaSuccess &&
-            cudaFuncSetAttribute(fb::fb_router_kernel<1, fb::kSelectSoftmaxRank>, attr, bytes1) == cudaSuccess;
-  if (ctx->stages[1] >= 2)
-    ok = ok && cudaFuncSetAttribute(fb::fb_router_kernel<2, fb::kSelectGeneral>, attr, bytes2) == cudaSuccess &&
-         cudaFuncSetAttribute(fb::fb_router_kernel<2, fb::kSelectSigmoidRank>, attr, bytes2) == cudaSuccess &&
-         cudaFuncSetAttribute(fb::fb_router_kernel<2, fb::kSelectSoftmaxRank>, attr, bytes2) == cudaSuccess;
+  bool ok = true;
+  for (int sel = 0; sel < 3; ++sel)
+    for (int lb = 0; lb < 2; ++lb) {
+      ok = ok && cudaFuncSetAttribute(reinterpret_cast<const void*>(router_kernel_fn<1>(sel, lb != 0)), attr, bytes1) ==
+                     cudaSuccess;
+      if (ctx->stages[1] >= 2)
+        ok = ok && cudaFuncSetAttribute(reinterpret_cast<const void*>(router_kernel_fn<2>(sel, lb != 0)), attr,
+                                        bytes2) == cudaSuccess;
+    }
   return ok ? FB_OK : FB_ERR_CUDA;
 }
 
@@ -435,10 +443,11 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   bool ok = true;
   if (ctx->persist_stages >= 2) {
-    ok = cudaFuncSetAttribute(fb::fb_router_persistent_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              static_cast<int>(ctx->persist_smem)) == cudaSuccess &&
-         cudaFuncSetAttribute(fb::fb_router_persistent_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              static_cast<int>(ctx->persist_smem)) == cudaSuccess;
+    for (int sg = 0; sg < 2; ++sg)
+      for (int lb = 0; lb < 2; ++lb)
+        ok = ok && cudaFuncSetAttribute(reinterpret_cast<const void*>(persistent_kernel_fn(sg != 0, lb != 0)),
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(ctx->persist_smem)) == cudaSuccess;
     // how many block pairs the GPU holds at once (the grid of the persistent kernel)
     cudaLaunchConfig_t occ;
     memset(&occ, 0, sizeof(occ));
@@ -451,10 +460,8 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
     occ.attrs = cl;
     occ.numAttrs = 1;
     int n_clusters = 0;
-    const bool sig = cfg->gate == FB_GATE_SIGMOID_GROUP_TOPK;
-    if (ok && (sig ? cudaOccupancyMaxActiveClusters(&n_clusters, fb::fb_router_persistent_kernel<true>, &occ)
-                   : cudaOccupancyMaxActiveClusters(&n_clusters, fb::fb_router_persistent_kernel<false>, &occ)) ==
-                  cudaSuccess &&
+    if (ok && cudaOccupancyMaxActiveClusters(&n_clusters, persistent_kernel_fn(cfg->gate == FB_GATE_SIGMOID_GROUP_TOPK, false),
+                                             &occ) == cudaSuccess &&
         n_clusters >= 1)
       ctx->max_pairs = n_clusters;
     else

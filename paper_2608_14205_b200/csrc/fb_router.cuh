@@ -308,7 +308,9 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32
 // both blocks get their stage-free and accumulator-ready signals from its commits.
 // kSel (SelectKind): one instance per selection code, so that each carries only the code and
 // the registers its gate needs; the host picks it with select_kind().
-template <int kCtas, int kSel>
+// kLogitBias: whether a logit bias (Eq. 2's "+ b") is given; without it the key computation
+// shrinks to one variant.
+template <int kCtas, int kSel, bool kLogitBias>
 __global__ void __launch_bounds__(kRouterThreads, 1)
 fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x2,
                  const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ RouterParams p) {
@@ -483,7 +485,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     TopK top;
     top.init();
     float sm_max = -INFINITY, sm_sum = 0.0f;               // softmax denominator (weights without renorm)
-    const bool has_lb = p.logit_bias != nullptr;
+    constexpr bool has_lb = kLogitBias;
     if (got) {
       // ---------------- pass 1
       float m1 = -INFINITY, m2 = -INFINITY;

@@ -59,9 +59,9 @@ __device__ __forceinline__ void ring_advance(int& s, uint32_t& phase, int stages
   if (++s == stages) { s = 0; phase ^= 1u; }
 }
 
-// kSigmoid: sigmoid + bias group-limited gate (true) or softmax gate (false); one instance per
-// gate keeps each one's code and register allocation to what that gate needs.
-template <bool kSigmoid>
+// kSigmoid: sigmoid + bias group-limited gate (true) or softmax gate (false); kLogitBias: a logit
+// bias is given.  One instance per combination keeps code and registers to what it needs.
+template <bool kSigmoid, bool kLogitBias>
 __global__ void __launch_bounds__(kRouterThreads, 1)
 fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x2,
                             const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ RouterParams p) {
@@ -191,7 +191,7 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     const int E = p.E, N = p.N, k = p.k;
     constexpr bool sigmoid_gate = kSigmoid;
     const int n_chunks = E >> 5;                           // E is a multiple of 32 here
-    const bool has_lb = p.logit_bias != nullptr;
+    constexpr bool has_lb = kLogitBias;
     const bool two_acc = p.num_kb > 1;
     // scratch behind the pipeline stages
     float* gscore_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) +

@@ -256,6 +256,11 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
       // block pairs just as fast as on 74 (measured), and the other SMs stay free for other streams
       const int rounds = (blocks / 2 + pairs_avail - 1) / pairs_avail;
       blocks = 2 * ((blocks / 2 + rounds - 1) / rounds);
+      // every block publishes its counts once: as many tickets as blocks that own a tile of the
+      // counted pass
+      p.ticket_target = blocks < tiles_pad ? blocks : tiles_pad;
+      // room for two accumulator sets (4 N columns) when the 512 tensor-memory columns allow it
+      if (4 * ctx->N <= 512) p.tmem_cols = next_pow2_at_least_32(4 * ctx->N);
       p.stages = ctx->persist_stages;
     }
   }

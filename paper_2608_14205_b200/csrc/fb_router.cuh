@@ -173,6 +173,33 @@ __device__ __forceinline__ float from_ordered_bits(uint32_t u) {
   return __uint_as_float(u ^ ((u >> 31) ? 0x80000000u : 0xffffffffu));
 }
 
+// The k-th largest of the known keys of a row: tab holds three tables of kBoundRows rows
+// (each chunk's best, second and third key), of which the first n_chunks rows are valid
+// (3 n_chunks >= k).  Counting instead of sorting: value v is the answer if at least k values
+// are >= v and it is the largest such value; all comparisons are independent of each other.
+template <int kRows>
+__device__ __forceinline__ float kth_largest_of_tables(const float* tab, int n_chunks, int k, int row_in_tile) {
+  float v[3 * kRows];
+#pragma unroll
+  for (int t = 0; t < 3; ++t)
+#pragma unroll
+    for (int c = 0; c < kRows; ++c)
+      v[t * kRows + c] = c < n_chunks ? tab[(t * kBoundRows + c) * kTileM + row_in_tile] : -INFINITY;
+  float best = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 3 * kRows; ++i) {
+    int at_least = 0;
+#pragma unroll
+    for (int j = 0; j < 3 * kRows; ++j) at_least += v[j] >= v[i] ? 1 : 0;
+    if (at_least >= k) best = fmaxf(best, v[i]);
+  }
+  return best;
+}
+__device__ __forceinline__ float kth_largest_known(const float* tab, int n_chunks, int k, int row_in_tile) {
+  return n_chunks <= 4 ? kth_largest_of_tables<4>(tab, n_chunks, k, row_in_tile)
+                       : kth_largest_of_tables<kBoundRows>(tab, n_chunks, k, row_in_tile);
+}
+
 // Ranking selection, shared by both router kernels.  cand[c * 128 + row] holds candidate c of
 // the row as one 64-bit word: ordered key bits in the high half, ~expert id in the low half,
 // so that "larger word" means "larger key, then lower id".  The kEpiSubs threads of a row
@@ -640,15 +667,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
       } else {
         // bound for the k-th key: the k-th largest of the chunks' three best keys (3 n_chunks >= k of them)
-        TopK known;
-        known.init();
-        for (int i = 0; i < 3 * kBoundRows; ++i) {
-          const float x = (i % kBoundRows) < n_chunks ? gscore_s[i * kTileM + row_in_tile] : -INFINITY;
-          if (x > known.v[FB_MAX_TOPK - 1]) known.insert(x, 0);
-        }
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j == k - 1) floor_key = known.v[j];
+        floor_key = kth_largest_known(gscore_s, n_chunks, k, row_in_tile);
         if (sub < n_chunks) my_groups[0] = sub;
         if (sub + kEpiSubs < n_chunks) my_groups[1] = sub + kEpiSubs;
       }

@@ -27,12 +27,15 @@ constexpr size_t kPersistScratchBytes =
     (3 * kPersistGroups * kTileM + 2 * kCandCap * kTileM) * sizeof(float);   // 44 KB
 static_assert(2 * kCandCap >= 2 * (kEpiSubs - 1) * FB_MAX_TOPK, "merge lists must fit in the candidate area");
 static_assert(2 * kPersistGroups >= 2 * FB_MAX_TOPK, "result lists must fit in the group-score area");
+static_assert(kPersistGroups == kBoundRows, "the three tables of best keys lie one after the other");
 
 struct PersistShared {
   uint64_t full_bar[kMaxStages];
   uint64_t empty_bar[kMaxStages];
-  uint64_t accum_bar;                        // both issuers' commits, once per tile
-  uint64_t tmem_empty_bar;                   // even block's copy: all epilogue warps of the pair, once per tile
+  // Accumulator sets: one (2 N of the 512 tensor-memory columns each) or, when 4 N <= 512, two that
+  // alternate from tile to tile, so that the next tile's MMAs need not wait for the drain.
+  uint64_t accum_bar[2];                     // per set: both issuers' commits, once per use
+  uint64_t tmem_empty_bar[2];                // per set, even block's copy: all epilogue warps of the pair, once per use
   uint32_t tmem_base;
   int32_t abort_flag;
   int32_t is_last;
@@ -91,8 +94,10 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
       mbar_init(smem_u32(&sh.full_bar[s]), 1);
       mbar_init(smem_u32(&sh.empty_bar[s]), 1);
     }
-    mbar_init(smem_u32(&sh.accum_bar), 2);
-    mbar_init(smem_u32(&sh.tmem_empty_bar), 2 * (kEpilogueThreads / 32));
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&sh.accum_bar[a]), 2);
+      mbar_init(smem_u32(&sh.tmem_empty_bar[a]), 2 * (kEpilogueThreads / 32));
+    }
     fence_mbar_init();
     prefetch_tensormap(&tmap_x);
     if (p.mode == kModeLayer) prefetch_tensormap(&tmap_x2);
@@ -149,18 +154,19 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     // ------------------------------------------------------------ MMA issuers (even block only)
     if (lane == 0 && cta_rank == 0) {
       const int first_kb = warp == 1 ? 0 : 1;
-      const uint32_t acc = tmem_base + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
+      const uint32_t acc_sets = 4 * p.N <= p.tmem_cols ? 2u : 1u;
       const uint32_t idesc = umma_idesc_bf16_f32(kTileM * 2, static_cast<uint32_t>(p.N));
       int s = 0;
       uint32_t phase = 0;
-      uint32_t drained = 0;                   // tiles whose accumulators the epilogue has taken over
+      uint32_t ti = 0;                        // this block pair's tile counter
       bool ok = true;
-      for (int pt = pair_first; pt < total_pairs && ok; pt += pair_stride) {
-        if (pt != pair_first) {
-          // the accumulators of the previous tile must have been read out by both blocks
-          ok = mbar_wait<true>(smem_u32(&sh.tmem_empty_bar), drained & 1u, abort_flag);
+      for (int pt = pair_first; pt < total_pairs && ok; pt += pair_stride, ++ti) {
+        const uint32_t set = ti % acc_sets, use = ti / acc_sets;
+        const uint32_t acc = tmem_base + set * 2u * static_cast<uint32_t>(p.N) + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
+        if (use != 0) {
+          // the set's previous contents must have been read out by both blocks
+          ok = mbar_wait<true>(smem_u32(&sh.tmem_empty_bar[set]), (use - 1u) & 1u, abort_flag);
           if (!ok) break;
-          ++drained;
           tcgen05_fence_after();
         }
         for (int kb = 0; kb < p.num_kb; ++kb) {
@@ -178,7 +184,7 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
           }
           ring_advance(s, phase, p.stages);
         }
-        if (ok) umma_commit_2cta(smem_u32(&sh.accum_bar), 0x3);   // this issuer's accumulator is complete
+        if (ok) umma_commit_2cta(smem_u32(&sh.accum_bar[set]), 0x3);   // this issuer's accumulator is complete
       }
     }
   } else {
@@ -187,7 +193,8 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     const int quarter = warp & 3;                          // TMEM lanes this warp may touch
     const int sub = (warp - 2) >> 2;                       // owns chunks sub and sub + 4
     const int row_in_tile = quarter * 32 + lane;
-    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const uint32_t taddr0 = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const uint32_t acc_sets = 4 * p.N <= p.tmem_cols ? 2u : 1u;
     const int E = p.E, N = p.N, k = p.k;
     constexpr bool sigmoid_gate = kSigmoid;
     const int n_chunks = E >> 5;                           // E is a multiple of 32 here
@@ -223,7 +230,9 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
       float* const out_w = (p.mode == kModeLayer && !second_pass) ? nullptr : p.topk_w;
 
       // one thread polls for the finished accumulators, the others sleep at the barrier
-      if (et == 0) sh.accum_ok = mbar_wait<true>(smem_u32(&sh.accum_bar), tiles_done & 1u, abort_flag) ? 1 : 0;
+      const uint32_t set = tiles_done % acc_sets, use = tiles_done / acc_sets;
+      const uint32_t taddr = taddr0 + set * 2u * static_cast<uint32_t>(N);
+      if (et == 0) sh.accum_ok = mbar_wait<true>(smem_u32(&sh.accum_bar[set]), use & 1u, abort_flag) ? 1 : 0;
       named_bar_sync(kAccumBarrierId, kEpilogueThreads);
       if (sh.accum_ok == 0) break;
       ++tiles_done;
@@ -259,7 +268,7 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
       // the issuers may overwrite the accumulators now
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(smem_u32(&sh.tmem_empty_bar), 0u);
+      if (lane == 0) mbar_arrive_cluster(smem_u32(&sh.tmem_empty_bar[set]), 0u);
 
       // ---------------- selection keys in place; best two keys of every chunk
 #pragma unroll
@@ -339,18 +348,7 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         }
       } else {
         // the k-th largest of the chunks' three best keys (3 n_chunks >= k of them)
-        TopK known;
-        known.init();
-        for (int c = 0; c < n_chunks; ++c) {
-          const float t1 = gscore_s[c * kTileM + row_in_tile], t2 = glow_s[c * kTileM + row_in_tile];
-          const float t3 = third_s[c * kTileM + row_in_tile];
-          if (t1 > known.v[FB_MAX_TOPK - 1]) known.insert(t1, 0);
-          if (t2 > known.v[FB_MAX_TOPK - 1]) known.insert(t2, 0);
-          if (t3 > known.v[FB_MAX_TOPK - 1]) known.insert(t3, 0);
-        }
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j == k - 1) floor_key = known.v[j];
+        floor_key = kth_largest_known(gscore_s, n_chunks, k, row_in_tile);
         kept = (1u << n_chunks) - 1u;
       }
       // ---------------- collect the keys >= floor of this thread's kept chunks (the bound is one of
@@ -442,7 +440,9 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
           if (owns) p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
           sh.hist[e] = 0;
         }
-      } else {
+      } else if (pt + pair_stride >= pairs_per_pass) {
+        // The histogram keeps accumulating over this block's tiles of the pass and is published
+        // once, after the last of them (one fence and one ticket per block, not per tile).
         publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
       }
     }

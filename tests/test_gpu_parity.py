@@ -503,3 +503,17 @@ def test_two_contexts_on_two_streams_do_not_interfere():
     assert all(c.fb_device_status() == 0 for c in ctxs)
     for c in ctxs:
         c.close()
+
+
+@pytest.mark.parametrize("kw,T,limit", [
+    # narrow gates: four accumulator sets' worth of columns fit, so tiles alternate between two sets
+    (dict(E=128, k=6, R=16, gate=1, n_group=4, topk_group=3, d=704), 1500, 1),
+    (dict(E=64, k=4, R=8, gate=1, n_group=2, topk_group=2, d=448), 2049, 2),
+    (dict(E=64, k=4, R=8, gate=0, d=1024), 1300, 1),
+    (dict(E=32, k=2, R=4, gate=0, d=64), 1100, 1),
+    (dict(E=256, k=8, R=32, gate=0, d=512), 900, 1),          # eight chunks: the wide bound tables
+])
+def test_persistent_kernel_narrow_and_wide_gates(kw, T, limit):
+    wl = _wl(**kw)
+    rep, gpu = _run(wl, T, layer=2, want_logits=False, pair_limit=limit)
+    assert gpu["persistent_launches"] == 4

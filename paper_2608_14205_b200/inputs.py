@@ -78,6 +78,9 @@ WORKLOADS = {
                         skew="zipf", zipf_s=1.2, max_swaps=1),
     "qwen3": Workload("qwen3", T=8192, d=2048, E=128, k=8, R=8, layers=48, rho=0.15,
                       skew="zipf", zipf_s=1.0, max_swaps=6, expert_bytes=9 * 2**20),
+    # The same model at the batch the paper evaluates it on: 16 sequences of 8K tokens.
+    "qwen3_b16": Workload("qwen3_b16", T=131072, d=2048, E=128, k=8, R=8, layers=48, rho=0.15,
+                          skew="zipf", zipf_s=1.0, max_swaps=6, expert_bytes=9 * 2**20),
     # Budget from the cost model: a 0.5 ms window, 44 MB per expert, 900 GB/s
     # (1111 fs per byte) and 2 us of fixed overhead give 99 858 ns per swap, so
     # exactly five swaps fit.

@@ -48,6 +48,7 @@ struct fb_ctx {
   size_t persist_smem = 0;
   int max_pairs = 0;
   int pair_limit = 0;
+  int dispatch_blocks_max = 296;       // resident blocks of the dispatch-index kernel (2 per SM)
   EncodeTiledFn encode = nullptr;
   // device scratch
   uint32_t* counts_scratch = nullptr;   // [256], zero between calls
@@ -327,7 +328,9 @@ fb_status launch_dispatch_index(fb_ctx* ctx, int32_t T, const int32_t* expert_to
   dp.inv_perm = inv_perm;
   dp.rank_load = rank_load;
   dp.status = ctx->status;
-  fb::fb_dispatch_kernel<<<dp.num_tiles, fb::kDispatchThreads, 0, stream>>>(dp);
+  // at most two blocks per SM are resident (1024 threads each): more tiles than that are walked in runs
+  const int dispatch_blocks = dp.num_tiles < ctx->dispatch_blocks_max ? dp.num_tiles : ctx->dispatch_blocks_max;
+  fb::fb_dispatch_kernel<<<dispatch_blocks, fb::kDispatchThreads, 0, stream>>>(dp);
   ++ctx->launches;
   return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
 }
@@ -367,6 +370,7 @@ static fb_status setup_router_shape(fb_ctx* ctx, const cudaDeviceProp& prop) {
     ctx->smem_bytes[pair] = dyn + 1024;
   }
   ctx->max_tiles = (cfg.T_max + fb::kTileM - 1) / fb::kTileM;
+  ctx->dispatch_blocks_max = 2 * prop.multiProcessorCount;
   const int bytes1 = static_cast<int>(ctx->smem_bytes[0]), bytes2 = static_cast<int>(ctx->smem_bytes[1]);
   const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
   bool ok = true;

@@ -4,7 +4,8 @@
 // position - so the result is unique and reproducible.
 //
 // Input: the router kernel's top-k ids and its per-tile expert histogram
-// tile_counts[tile][e] (tile = 128 consecutive tokens).  One block per tile.
+// tile_counts[tile][e] (tile = 128 consecutive tokens).  One block per tile, or per run of
+// consecutive tiles when there are more tiles than blocks fit on the GPU at once.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -32,30 +33,34 @@ struct DispatchParams {
   int32_t* status;
 };
 
-__global__ void __launch_bounds__(kDispatchThreads)
+__global__ void __launch_bounds__(kDispatchThreads, 2)
 fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
   __shared__ int32_t slot_of[FB_MAX_EXPERTS];
   __shared__ int32_t owner[FB_MAX_EXPERTS];
-  __shared__ uint32_t before[FB_MAX_EXPERTS];      // assignments to this slot in earlier tiles
+  __shared__ uint32_t before[2][FB_MAX_EXPERTS];   // assignments to this slot in earlier tiles (two buffers: see the tile loop)
   __shared__ uint32_t total[FB_MAX_EXPERTS];       // assignments to this slot in all tiles
   __shared__ uint32_t part_before[kDispatchThreads / FB_MAX_EXPERTS][FB_MAX_EXPERTS];
   __shared__ uint32_t part_total[kDispatchThreads / FB_MAX_EXPERTS][FB_MAX_EXPERTS];
   __shared__ uint32_t offs[FB_MAX_EXPERTS + 1];    // exclusive prefix of total over slots
-  __shared__ uint32_t mask[FB_MAX_EXPERTS][kDispatchTile / 32];
+  __shared__ uint32_t mask[3][FB_MAX_EXPERTS][kDispatchTile / 32];
   __shared__ uint32_t warp_sum[FB_MAX_EXPERTS / 32];
   __shared__ int32_t bad;
 
   const int t = threadIdx.x;
-  const int tile = blockIdx.x;
   const int E = p.E, k = p.k;
+  // This block's tiles: a contiguous range, so that "assignments in earlier tiles" can be carried
+  // from one tile to the next instead of being summed again.
+  const int per_block = (p.num_tiles + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  const int tile_begin = static_cast<int>(blockIdx.x) * per_block;
+  const int tile_end = min(p.num_tiles, tile_begin + per_block);
   // The next router kernel of the stream may set itself up while this grid runs (it waits for
   // this grid's completion before it reads anything).
   pdl_launch_dependents();
   if (t == 0) bad = 0;
   for (int s = t; s < FB_MAX_EXPERTS; s += kDispatchThreads) {
-    owner[s] = -1; before[s] = 0; total[s] = 0;
+    owner[s] = -1; before[0][s] = 0; before[1][s] = 0; total[s] = 0;
 #pragma unroll
-    for (int w = 0; w < kDispatchTile / 32; ++w) mask[s][w] = 0;
+    for (int w = 0; w < kDispatchTile / 32; ++w) { mask[0][s][w] = 0; mask[1][s][w] = 0; mask[2][s][w] = 0; }
   }
   __syncthreads();
   for (int e = t; e < E; e += kDispatchThreads) {
@@ -66,12 +71,14 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
   }
   __syncthreads();
   if (bad) {                                    // not a bijection: report, write nothing
-    if (t == 0 && tile == 0) atomicCAS(p.status, 0, FB_ERR_BAD_PLACEMENT);
+    if (t == 0 && blockIdx.x == 0) atomicCAS(p.status, 0, FB_ERR_BAD_PLACEMENT);
     return;
   }
-  // Column sums of the per-tile histogram, split at this tile.  The loop is bound by L2
-  // latency, so each column is shared by 4 threads and the loads are issued 32 at a time.
+  if (tile_begin >= tile_end) return;
+  // Column sums of the per-tile histogram, split at this block's first tile.  The loop is bound
+  // by L2 latency, so each column is shared by 4 threads and the loads are issued 32 at a time.
   {
+    const int tile = tile_begin;
     constexpr int kParts = kDispatchThreads / FB_MAX_EXPERTS;
     const int e = t % FB_MAX_EXPERTS, part = t / FB_MAX_EXPERTS;
     uint32_t bef = 0, tot = 0;
@@ -109,7 +116,7 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
       uint32_t b = 0, a = 0;
 #pragma unroll
       for (int q = 0; q < kParts; ++q) { b += part_before[q][e]; a += part_total[q][e]; }
-      before[slot_of[e]] = b;
+      before[0][slot_of[e]] = b;
       total[slot_of[e]] = a;
     }
   }
@@ -133,36 +140,57 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
     }
   }
   __syncthreads();
-  if (tile == 0) {
+  if (blockIdx.x == 0) {
     const int m = E / p.R;
     for (int s = t; s <= E; s += kDispatchThreads) p.slot_offsets[s] = offs[s];
     for (int r = t; r <= p.R; r += kDispatchThreads) p.rank_offsets[r] = offs[r * m];
     for (int r = t; r < p.R; r += kDispatchThreads) p.rank_load[r] = offs[(r + 1) * m] - offs[r * m];
   }
-  // Rank of each assignment among the rows of this tile that go to the same slot.
+  // Rank of each assignment among the rows of its tile that go to the same slot.
   // Thread (row, j) = (t % 128, t / 128) owns assignment j of the tile's row.
   static_assert(kDispatchThreads == kDispatchTile * FB_MAX_TOPK, "one thread per assignment of a tile");
   const int row = t % kDispatchTile, j = t / kDispatchTile;
-  const long long i = static_cast<long long>(tile) * kDispatchTile + row;
-  const bool active = j < k && i < p.T;
-  int my_slot = 0;
-  if (active) {
-    int e = p.topk_ids[i * k + j];
-    e = (e < 0 || e >= E) ? 0 : e;
-    my_slot = slot_of[e];
-    atomicOr(&mask[my_slot][row >> 5], 1u << (row & 31));
-  }
-  __syncthreads();
-  if (active) {
-    const long long n_assign = static_cast<long long>(p.T) * k;
-    uint32_t ahead = __popc(mask[my_slot][row >> 5] & ((1u << (row & 31)) - 1u));
-    for (int w = 0; w < (row >> 5); ++w) ahead += __popc(mask[my_slot][w]);
-    const long long pos = static_cast<long long>(offs[my_slot]) + before[my_slot] + ahead;
-    const long long flat = i * k + j;
-    if (pos < n_assign) {
-      p.perm[pos] = static_cast<int32_t>(flat);
-      p.inv_perm[flat] = static_cast<int32_t>(pos);
+  const long long n_assign = static_cast<long long>(p.T) * k;
+  // Tile loop with one barrier per tile.  Tile n reads the earlier-tile counts from buffer n % 2
+  // and writes the next tile's into the other one after its barrier (last read before that
+  // barrier).  The row masks rotate through three buffers: tile n uses n % 3 and, after its
+  // barrier, clears (n + 2) % 3, which tile n - 1 read before that barrier and tile n + 2 will
+  // fill after the next one.  The next tile's expert id and this tile's histogram row are loaded
+  // one iteration ahead.
+  auto load_id = [&](int tile) -> int {
+    const long long i = static_cast<long long>(tile) * kDispatchTile + row;
+    if (tile >= tile_end || j >= k || i >= p.T) return -1;
+    const int e = p.topk_ids[i * k + j];
+    return (e < 0 || e >= E) ? 0 : e;
+  };
+  int e_cur = load_id(tile_begin);
+  for (int tile = tile_begin; tile < tile_end; ++tile) {
+    const int n = tile - tile_begin, par = n & 1, mb = n % 3, mb_clear = (n + 2) % 3;
+    const int e_next = load_id(tile + 1);
+    // this tile's histogram row, needed to step the earlier-tile counts to the next tile
+    const uint32_t step = (t < E && tile + 1 < tile_end) ? __ldg(p.tile_counts + static_cast<size_t>(tile) * E + t) : 0u;
+    const bool active = e_cur >= 0;
+    const int my_slot = active ? slot_of[e_cur] : 0;
+    if (active) atomicOr(&mask[mb][my_slot][row >> 5], 1u << (row & 31));
+    __syncthreads();
+    if (active) {
+      uint32_t ahead = __popc(mask[mb][my_slot][row >> 5] & ((1u << (row & 31)) - 1u));
+      for (int w = 0; w < (row >> 5); ++w) ahead += __popc(mask[mb][my_slot][w]);
+      const long long pos = static_cast<long long>(offs[my_slot]) + before[par][my_slot] + ahead;
+      const long long flat = (static_cast<long long>(tile) * kDispatchTile + row) * k + j;
+      if (pos < n_assign) {
+        p.perm[pos] = static_cast<int32_t>(flat);
+        p.inv_perm[flat] = static_cast<int32_t>(pos);
+      }
     }
+    if (tile + 1 < tile_end) {
+      if (t < E) before[par ^ 1][slot_of[t]] = before[par][slot_of[t]] + step;
+      for (int s = t; s < FB_MAX_EXPERTS; s += kDispatchThreads) {
+#pragma unroll
+        for (int w = 0; w < kDispatchTile / 32; ++w) mask[mb_clear][s][w] = 0;
+      }
+    }
+    e_cur = e_next;
   }
 }
 

@@ -517,3 +517,14 @@ def test_persistent_kernel_narrow_and_wide_gates(kw, T, limit):
     wl = _wl(**kw)
     rep, gpu = _run(wl, T, layer=2, want_logits=False, pair_limit=limit)
     assert gpu["persistent_launches"] == 4
+
+
+def test_dispatch_index_with_several_tiles_per_block():
+    # more tiles than resident blocks of the dispatch-index kernel: every block walks a run of
+    # three tiles (the rotation of its mask buffers and the carried counts are exercised)
+    wl = _wl(E=64, k=4, R=8, gate=0, d=64, max_swaps=6)
+    T = 100_000
+    rng = np.random.default_rng(0)
+    sample = np.sort(rng.choice(T, size=512, replace=False))
+    rep, gpu = _run(wl, T, want_logits=False, sample=sample)
+    assert rep["early_mismatch_unflagged"] == 0 and rep["final_mismatch_unflagged"] == 0

@@ -186,14 +186,14 @@ fb_status fb_route_dispatch(fb_ctx* ctx, const fb_router* router, const void* x,
                             int32_t* perm, int32_t* inv_perm, uint32_t* rank_load,
                             float* logits, fb_stream stream);
 
-/* One whole layer with device buffers: stages 1, 2 and 4 in one call.  Same results as
- * fb_predict_and_plan followed by fb_route_dispatch under the new placement, but both
- * router passes (the early one on h_prev, the normal one on H) run in ONE kernel launch:
- * its second half of thread blocks moves onto the SMs as the first half retires, so the
- * selection and planning tail of the early pass overlaps the normal pass.  The dispatch
- * index follows in a second launch.  Arguments as in the two calls it replaces
- * (expert_to_slot_out may not alias expert_to_slot here: the plan is being written
- * while nothing reads it, but keep them distinct for clarity of ownership). */
+/* One whole layer with device buffers: stages 1, 2 and 4 in one call.  Same results, bit for
+ * bit, as fb_predict_and_plan followed by fb_route_dispatch under the new placement, but
+ * both router passes (the early one on h_prev, the normal one on H) run in ONE kernel
+ * launch: the tiles of the normal pass follow those of the early pass on the same blocks
+ * (or in the same grid), so the selection and planning tail of the early pass is hidden
+ * behind the normal pass.  The dispatch index follows in a second launch.  Arguments as in
+ * the two calls it replaces; h_prev and H must be different buffers of [T][d] bf16 each,
+ * and expert_to_slot_out must not alias expert_to_slot.  Errors as in those calls. */
 fb_status fb_layer_step(fb_ctx* ctx, const fb_router* router, const void* h_prev, const void* H, int32_t T,
                         const int32_t* expert_to_slot, const fb_budget* budget, int32_t layer_id,
                         uint32_t* counts, int32_t* expert_to_slot_out, fb_swap* swaps, int32_t* n_swaps,

@@ -10,7 +10,9 @@
  *                           model (Eq. 9), budgets (Eq. 10), deterministic greedy
  *                           pairwise swaps under the load objective (Eqs. 6-8)
  *      fb_predict_and_plan  1 + 2 in a single kernel launch
- *   3. (weight migration: not part of this library)
+ *      fb_layer_step        1 + 2 + 4 for one layer: both router passes in one launch
+ *   3. fb_apply_swaps       the accepted swaps applied to the expert weights (logical ranks
+ *                           on one GPU: an exchange of slot images inside one buffer)
  *   4. fb_route_dispatch    normal router pass g_l(H_l) (Eq. 3), authoritative top-k
  *                           and routing weights, and the token -> expert dispatch
  *                           index under the committed placement pi'
@@ -24,7 +26,8 @@
  *     dense row-major.  "host" pointers are ordinary host memory.
  *   - Structs (fb_config, fb_router, fb_budget) are host structs read during the call.
  *   - Calls enqueue work on `stream` and return without synchronising, except
- *     fb_layer_step_host and fb_device_status which block until the stream drains.
+ *     fb_layer_step_host and fb_device_status, which block until the stream drains,
+ *     fb_apply_swaps_staged (waits for the plan) and fb_calibrate_exchange (times itself).
  *   - No call throws or aborts.  Argument and shape problems are reported by the
  *     return value and nothing is launched.  Problems only the device can see (a
  *     placement that is not a bijection, count sums beyond the planner's range, a
@@ -116,7 +119,8 @@ typedef struct { int32_t src_rank, dst_rank, expert_src, expert_dst; } fb_swap;
 /* ------------------------------------------------------------------------------------
  * Context.  fb_create allocates all device scratch the other calls need (sized from
  * T_max and E) on `device`; fb_destroy frees it.  No other call allocates, except the
- * first fb_layer_step_host (its staging buffers).
+ * first fb_layer_step_host and fb_apply_swaps_staged (their staging buffers) and
+ * fb_calibrate_exchange (28 bytes for the duration of the call).
  * Limits (FB_ERR_UNSUPPORTED_SHAPE otherwise): 1 <= E <= 256, 1 <= k <= min(E, 8),
  * 1 <= R <= 64 with R | E, d >= 8 with 8 | d, 0 <= T <= T_max < 2^31 / max(E, k);
  * sigmoid gate: n_group | E, n_group <= 32, 1 <= topk_group <= min(n_group, 8),

@@ -119,8 +119,7 @@ typedef struct { int32_t src_rank, dst_rank, expert_src, expert_dst; } fb_swap;
 /* ------------------------------------------------------------------------------------
  * Context.  fb_create allocates all device scratch the other calls need (sized from
  * T_max and E) on `device`; fb_destroy frees it.  No other call allocates, except the
- * first fb_layer_step_host and fb_apply_swaps_staged (their staging buffers) and
- * fb_calibrate_exchange (28 bytes for the duration of the call).
+ * first fb_layer_step_host and fb_apply_swaps_staged (their staging buffers).
  * Limits (FB_ERR_UNSUPPORTED_SHAPE otherwise): 1 <= E <= 256, 1 <= k <= min(E, 8),
  * 1 <= R <= 64 with R | E, d >= 8 with 8 | d, 0 <= T <= T_max < 2^31 / max(E, k);
  * sigmoid gate: n_group | E, n_group <= 32, 1 <= topk_group <= min(n_group, 8),
@@ -236,9 +235,13 @@ fb_status fb_layer_step_host(fb_ctx* ctx, const fb_router* router,
  * every GPU that loads the library holds those bytes until the process exits.
  *   - cfg->E above FB_STATIC_MAX_EXPERTS is refused with FB_ERR_UNSUPPORTED_SHAPE; the
  *     other limits are those of fb_create.
- *   - The first call on a device looks up the array's device address and sets kernel
- *     attributes (once per device; the shape-dependent part again when cfg changes).
- *     Make that first call before starting any stream capture.
+ *   - The first call on a device looks up the array's device address and raises the
+ *     kernels' shared-memory ceiling (once per device); a change of cfg only redoes host
+ *     arithmetic.  Make that first call before starting any stream capture.
+ *   - What the call cannot rule out is the driver's own work: with lazy module loading the
+ *     first launch of a kernel variant on a device places its code (and this array) there.
+ *     The guarantee "takes nothing from the device" therefore holds from the second call
+ *     with a given gate type on; make one warm-up call before the memory pool is frozen.
  *   - All calls on a device share the one array.  Each call clears it on `stream` before
  *     its kernel, so a call is not disturbed by what an earlier one left behind, but two
  *     calls that overlap on the GPU (different streams) race on it: serialise them.
@@ -254,9 +257,6 @@ fb_status fb_predict_load_static(const fb_config* cfg, int device, const fb_rout
  * first FB_ERR_BAD_PLACEMENT / FB_ERR_TIMEOUT / FB_ERR_RANGE raised since the last
  * query) and clears it. */
 fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream);
-
-/* Kernels this library has launched through `ctx` so far (for benchmarks). */
-uint64_t fb_launch_count(const fb_ctx* ctx);
 
 /* ---- stage 3 on one device (Method overview, "Weight Transfer"): apply a plan to the weights ----
  * slot_weights is a device buffer of E slot images of expert_bytes each (slot p at byte
@@ -286,7 +286,8 @@ fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, c
  * bytes_small and of bytes_large bytes (slot_weights: device buffer of 2 * bytes_large
  * bytes, 16-byte aligned; its contents are not preserved),
  * reps times each after two warm-up runs, keeps the fastest, and fits.  Blocking (it waits
- * for its own events); allocates 28 bytes of device memory for the duration of the call.
+ * for its own events); allocates no device memory.  Runs on the device that holds
+ * slot_weights, whichever device is current (so does fb_apply_swaps).
  * t_small_ns_out / t_large_ns_out (optional) receive the two timings. */
 fb_status fb_fit_cost_model(uint64_t t_small_ns, uint64_t t_large_ns, uint64_t bytes_small, uint64_t bytes_large,
                             uint64_t* alpha_ns, uint64_t* fs_per_byte);
@@ -338,17 +339,9 @@ fb_status fb_topk_hits(const int32_t* ids_a, const int32_t* ids_b, int32_t T, in
  * weights are renormalised); other shapes ignore it.  Returns FB_ERR_INVALID_ARG for a
  * negative limit. */
 fb_status fb_set_pair_limit(fb_ctx* ctx, int32_t pairs);
-/* Measurement aid: the next router-kernel launch made through ctx records the two CUDA
- * events (cudaEvent_t handles owned by the caller, either may be NULL) on its stream,
- * one directly before and one directly after the launch, and then forgets them.  Lets a
- * caller time that kernel alone inside a call that launches several kernels. */
-fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
 /* Block pairs of the persistent router kernel that fit on the GPU at once (0 when the
  * configuration does not support that kernel). */
 int32_t fb_max_pairs(const fb_ctx* ctx);
-/* How many of the launches counted by fb_launch_count were the persistent router kernel. */
-uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
-
 /* Text for a status code; never NULL. */
 const char* fb_status_string(fb_status s);
 

@@ -1,0 +1,42 @@
+/*
+ * freebalance_aids.h - measurement and diagnostic aids of the FreeBalance library.
+ *
+ * Nothing here is part of the per-layer path of the paper's method (the paper has no
+ * counterpart for any of these calls); benchmarks and tests use them to count launches, to
+ * time one kernel inside a multi-kernel call, and to exercise the bounded device-side wait.
+ * Same conventions as freebalance.h.
+ */
+#ifndef FREEBALANCE_AIDS_H_
+#define FREEBALANCE_AIDS_H_
+
+#include "freebalance.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Kernels this library has launched through `ctx` so far. */
+uint64_t fb_launch_count(const fb_ctx* ctx);
+
+/* How many of the launches counted by fb_launch_count were the persistent router kernel. */
+uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
+
+/* The next router-kernel launch made through ctx records the two CUDA events (cudaEvent_t
+ * handles owned by the caller, either may be NULL) on its stream, one directly before and
+ * one directly after the launch, and then forgets them.  Lets a caller time that kernel
+ * alone inside a call that launches several kernels. */
+fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
+
+/* Self-test of the bounded wait that every kernel of the library uses for its barriers: a
+ * one-block kernel waits for at most limit_ns (1 .. 100 000 000) on a barrier at which
+ * nobody ever arrives, gives up, records FB_ERR_TIMEOUT in ctx's device status word and
+ * returns normally; nothing traps and the context stays usable.  fb_device_status then
+ * reports FB_ERR_TIMEOUT once and clears it.  waited_ns (dev u64 [1], optional) receives
+ * the time the wait actually took.  Asynchronous on `stream`.  Errors: FB_ERR_INVALID_ARG
+ * for a NULL context or a limit outside the range. */
+fb_status fb_selftest_wait_timeout(fb_ctx* ctx, uint64_t limit_ns, uint64_t* waited_ns, fb_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* FREEBALANCE_AIDS_H_ */

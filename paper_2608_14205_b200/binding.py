@@ -51,7 +51,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
            "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
-           "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange"]
+           "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout"]
 
 _lib = None
 
@@ -99,6 +99,8 @@ def lib() -> ctypes.CDLL:
     L.fb_set_pair_limit.restype = ctypes.c_int
     L.fb_max_pairs.argtypes = [vp]
     L.fb_max_pairs.restype = i32
+    L.fb_selftest_wait_timeout.argtypes = [vp, u64, vp, vp]
+    L.fb_selftest_wait_timeout.restype = ctypes.c_int
     L.fb_row_cosine_mean.argtypes = [vp, vp, ctypes.c_int64, i32, i32, vp, vp, vp]
     L.fb_row_cosine_mean.restype = ctypes.c_int
     L.fb_topk_hits.argtypes = [vp, vp, i32, i32, vp, vp]
@@ -307,6 +309,10 @@ class Context:
 
     def fb_max_pairs(self) -> int:
         return int(lib().fb_max_pairs(self._h))
+
+    def fb_selftest_wait_timeout(self, limit_ns: int, waited_ns=None, stream=None) -> None:
+        _check(lib().fb_selftest_wait_timeout(self._h, limit_ns, _ptr(waited_ns), _stream(stream)),
+               "fb_selftest_wait_timeout")
 
     def fb_time_next_router_launch(self, event_before, event_after) -> None:
         """torch.cuda.Event objects (created with enable_timing=True); either may be None."""

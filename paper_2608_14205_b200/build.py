@@ -10,8 +10,8 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libfreebalance.so")
 SOURCES = ["fb_api.cu"]
-HEADERS = ["fb_ptx.cuh", "fb_planner.cuh", "fb_router.cuh", "fb_dispatch.cuh",
-           os.path.join("..", "..", "include", "freebalance.h")]
+HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))) + \
+          [os.path.join("..", "..", "include", h) for h in ("freebalance.h", "freebalance_aids.h")]
 
 
 def _nvcc() -> str:

@@ -9,6 +9,7 @@
 #include <new>
 
 #include "../../include/freebalance.h"
+#include "../../include/freebalance_aids.h"
 #include "fb_dispatch.cuh"
 #include "fb_migrate.cuh"
 #include "fb_planner.cuh"
@@ -341,6 +342,17 @@ fb_status launch_plan(fb_ctx* ctx, const fb::PlanParams& pp, const uint32_t* cou
   return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
 }
 
+// The device that owns a device pointer (-1 if it is not device memory).
+int device_of(const void* p) {
+  cudaPointerAttributes pa;
+  if (cudaPointerGetAttributes(&pa, p) != cudaSuccess) { cudaGetLastError(); return -1; }
+  return (pa.type == cudaMemoryTypeDevice || pa.type == cudaMemoryTypeManaged) ? pa.device : -1;
+}
+
+// A fixed one-swap plan over two slots for fb_calibrate_exchange: [placement: 2][swap: 4][n: 1].
+// Constant data inside the library image, so the calibration allocates nothing.
+__device__ const int32_t g_calibration_plan[8] = {0, 1, 0, 1, 0, 1, 1, 0};
+
 template <typename Tp>
 bool dev_alloc(Tp** p, size_t count) {
   return cudaMalloc(reinterpret_cast<void**>(p), (count ? count : 1) * sizeof(Tp)) == cudaSuccess;
@@ -348,8 +360,8 @@ bool dev_alloc(Tp** p, size_t count) {
 
 }  // namespace
 
-// Shape-dependent launch parameters of the one-tile router kernel (host arithmetic and
-// function attributes only): padded width, TMEM columns, pipeline depth and dynamic shared
+// Shape-dependent launch parameters of the one-tile router kernel (host arithmetic
+// only): padded width, TMEM columns, pipeline depth and dynamic shared
 // memory of the single-block and the pair variant.
 static fb_status setup_router_shape(fb_ctx* ctx, const cudaDeviceProp& prop) {
   const fb_config& cfg = ctx->cfg;
@@ -371,18 +383,35 @@ static fb_status setup_router_shape(fb_ctx* ctx, const cudaDeviceProp& prop) {
   }
   ctx->max_tiles = (cfg.T_max + fb::kTileM - 1) / fb::kTileM;
   ctx->dispatch_blocks_max = 2 * prop.multiProcessorCount;
-  const int bytes1 = static_cast<int>(ctx->smem_bytes[0]), bytes2 = static_cast<int>(ctx->smem_bytes[1]);
-  const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  return FB_OK;
+}
+
+// The ceiling on a kernel's dynamic shared memory belongs to the function on a device, not
+// to a context: contexts of different shapes share the kernel instances.  It is therefore
+// raised once per device, for every router kernel instance, to the most the device allows
+// beside the kernel's static shared memory, and never lowered again.
+static fb_status ensure_kernel_attributes(int device, const cudaDeviceProp& prop) {
+  static bool done[64] = {};
+  if (device >= 0 && device < 64 && done[device]) return FB_OK;
   bool ok = true;
+  auto raise = [&](RouterKernelFn fn) {
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, reinterpret_cast<const void*>(fn)) != cudaSuccess) { ok = false; return; }
+    const int most = static_cast<int>(prop.sharedMemPerBlockOptin) - static_cast<int>(fa.sharedSizeBytes);
+    ok = ok && most > 0 &&
+         cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, most) ==
+             cudaSuccess;
+  };
   for (int sel = 0; sel < 3; ++sel)
     for (int lb = 0; lb < 2; ++lb) {
-      ok = ok && cudaFuncSetAttribute(reinterpret_cast<const void*>(router_kernel_fn<1>(sel, lb != 0)), attr, bytes1) ==
-                     cudaSuccess;
-      if (ctx->stages[1] >= 2)
-        ok = ok && cudaFuncSetAttribute(reinterpret_cast<const void*>(router_kernel_fn<2>(sel, lb != 0)), attr,
-                                        bytes2) == cudaSuccess;
+      raise(router_kernel_fn<1>(sel, lb != 0));
+      raise(router_kernel_fn<2>(sel, lb != 0));
     }
-  return ok ? FB_OK : FB_ERR_CUDA;
+  for (int sg = 0; sg < 2; ++sg)
+    for (int lb = 0; lb < 2; ++lb) raise(persistent_kernel_fn(sg != 0, lb != 0));
+  if (!ok) { cudaGetLastError(); return FB_ERR_CUDA; }
+  if (device >= 0 && device < 64) done[device] = true;
+  return FB_OK;
 }
 
 extern "C" {
@@ -428,7 +457,8 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   ctx->cfg = *cfg;
   ctx->device = device;
   {
-    const fb_status ss = setup_router_shape(ctx, prop);
+    fb_status ss = setup_router_shape(ctx, prop);
+    if (ss == FB_OK) ss = ensure_kernel_attributes(device, prop);
     if (ss != FB_OK) { delete ctx; return ss; }
   }
   if (ctx->stages[1] >= 2 && ctx->N % 32 == 0 && ctx->N == cfg->E) {
@@ -452,11 +482,6 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   bool ok = true;
   if (ctx->persist_stages >= 2) {
-    for (int sg = 0; sg < 2; ++sg)
-      for (int lb = 0; lb < 2; ++lb)
-        ok = ok && cudaFuncSetAttribute(reinterpret_cast<const void*>(persistent_kernel_fn(sg != 0, lb != 0)),
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(ctx->persist_smem)) == cudaSuccess;
     // how many block pairs the GPU holds at once (the grid of the persistent kernel)
     cudaLaunchConfig_t occ;
     memset(&occ, 0, sizeof(occ));
@@ -700,6 +725,11 @@ fb_status fb_apply_swaps(void* slot_weights, uint64_t expert_bytes, int32_t E, c
   if (max_swaps == 0 || expert_bytes == 0) return FB_OK;
   if (!slot_weights || !expert_to_slot || !swaps || !n_swaps) return FB_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(slot_weights) % 16 != 0) return FB_ERR_INVALID_ARG;
+  // the launch goes to the device that holds the weights, whichever device is current
+  const int device = device_of(slot_weights);
+  if (device < 0) return FB_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return FB_ERR_CUDA;
   fb::MigrateParams mp;
   mp.slot_weights = static_cast<uint8_t*>(slot_weights);
   mp.expert_bytes = expert_bytes;
@@ -740,13 +770,17 @@ fb_status fb_calibrate_exchange(void* slot_weights, uint64_t bytes_small, uint64
       bytes_small % 16 != 0 || bytes_large % 16 != 0 || bytes_large <= bytes_small)
     return FB_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  // a one-swap plan over two slots, kept on the device for the duration of the call
-  int32_t* plan = nullptr;                       // [pi: 2][swap: 4][n: 1]
-  if (cudaMalloc(&plan, 7 * sizeof(int32_t)) != cudaSuccess) return FB_ERR_CUDA;
-  const int32_t h_plan[7] = {0, 1, 0, 1, 0, 1, 1};
+  const int device = device_of(slot_weights);
+  if (device < 0) return FB_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  // a one-swap plan over two slots: constant data of the library image on this device
+  const int32_t* plan = nullptr;                 // [pi: 2][swap: 4][n: 1]
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(const_cast<int32_t**>(&plan)), g_calibration_plan) !=
+          cudaSuccess || plan == nullptr)
+    return FB_ERR_CUDA;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
-  bool ok = cudaMemcpyAsync(plan, h_plan, sizeof(h_plan), cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-            cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess;
+  bool ok = cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess;
   uint64_t t_ns[2] = {0, 0};
   const uint64_t sizes[2] = {bytes_small, bytes_large};
   for (int which = 0; which < 2 && ok; ++which) {
@@ -777,7 +811,6 @@ fb_status fb_calibrate_exchange(void* slot_weights, uint64_t bytes_small, uint64
   }
   if (e0) cudaEventDestroy(e0);
   if (e1) cudaEventDestroy(e1);
-  cudaFree(plan);
   if (!ok) return FB_ERR_CUDA;
   if (t_small_ns_out) *t_small_ns_out = t_ns[0];
   if (t_large_ns_out) *t_large_ns_out = t_ns[1];
@@ -877,6 +910,15 @@ fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* even
 
 int32_t fb_max_pairs(const fb_ctx* ctx) { return ctx ? ctx->max_pairs : 0; }
 
+fb_status fb_selftest_wait_timeout(fb_ctx* ctx, uint64_t limit_ns, uint64_t* waited_ns, fb_stream stream_) {
+  if (!ctx || limit_ns == 0 || limit_ns > 100ull * 1000 * 1000) return FB_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  fb::fb_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream_)>>>(limit_ns, ctx->status, waited_ns);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
 uint64_t fb_persistent_launch_count(const fb_ctx* ctx) { return ctx ? ctx->persistent_launches : 0; }
 
 }  // extern "C"
@@ -942,7 +984,8 @@ extern "C" fb_status fb_predict_load_static(const fb_config* cfg, int device, co
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FB_ERR_CUDA;
     ctx.cfg = *cfg;
-    const fb_status ss = setup_router_shape(&ctx, prop);
+    fb_status ss = setup_router_shape(&ctx, prop);
+    if (ss == FB_OK) ss = ensure_kernel_attributes(device, prop);
     if (ss != FB_OK) { ctx.cfg.E = -1; return ss; }
     for (int i = 0; i < kMapCache; ++i) { ctx.x_maps[i] = MapEntry(); ctx.w_maps[i] = MapEntry(); }
   }

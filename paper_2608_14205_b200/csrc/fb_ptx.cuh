@@ -73,11 +73,12 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // one second per wait
 
-// Wait for the phase with the given parity.  Gives up after kWaitLimitNs, or as soon
+// Wait for the phase with the given parity.  Gives up after limit_ns, or as soon
 // as another thread of the block has given up (abort flag in shared memory), and
 // returns false; the caller then skips to its clean-up.
 template <bool kCluster = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   uint32_t polls = 0;
   uint64_t t0 = 0;
   for (;;) {
@@ -87,7 +88,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
   }
 }

@@ -891,6 +891,25 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   }
 }
 
+// Self-test of the bounded wait every kernel of this library relies on: one thread waits, for
+// at most limit_ns, on a barrier that nobody ever arrives at.  The wait gives up, the kernel
+// records FB_ERR_TIMEOUT in the status word and returns normally - the same path a router
+// kernel takes when a copy or an MMA it waits for never completes.
+__global__ void __launch_bounds__(32, 1)
+fb_wait_selftest_kernel(uint64_t limit_ns, int32_t* status, uint64_t* waited_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int32_t abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    fence_mbar_init();
+    const uint64_t t0 = global_timer_ns();
+    const bool ok = mbar_wait<false>(smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    if (waited_ns != nullptr) *waited_ns = global_timer_ns() - t0;
+    if (!ok) atomicCAS(status, 0, FB_ERR_TIMEOUT);
+  }
+}
+
 // Stand-alone planner: one warp.
 __global__ void __launch_bounds__(kPlanThreads, 1)
 fb_plan_kernel(const __grid_constant__ PlanParams p, const uint32_t* __restrict__ counts, int32_t* status) {

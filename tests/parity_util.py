@@ -5,7 +5,10 @@ Comparison rules
 * logits: |gpu - oracle| <= LOGIT_TOL everywhere.
 * top-k: per-token expert sets must be equal, except for tokens whose oracle margin
   (gap between the k-th and (k+1)-th eligible key, or between the last kept and first
-  dropped group score) is below the near-tie threshold; those are counted.
+  dropped group score) is below the near-tie threshold; those are counted.  Two
+  thresholds are asserted: 2e-3 (the stated one) and a tight one, 1e-4 or - when it is
+  larger - the bound that the measured logit error of this very comparison implies
+  (two keys can only change order if their gap is below twice the key error).
 * everything integer (counts, plan, placement, loads, dispatch index) is rechecked
   bit-exactly by feeding the GPU's own top-k to the oracle, and must additionally equal
   the oracle's own pipeline when no token differed.
@@ -49,6 +52,42 @@ def make_context(wl: I.Workload, T_max: int) -> B.Context:
                      wl.route_scale)
 
 
+GUARD_WORDS = 64                      # 256 bytes of known pattern before and after every output
+GUARD_PATTERN = 0x5A5AA5A5
+
+
+class GuardedOutputs:
+    """Output buffers with guard regions.  compute-sanitizer is not available to these tests, so
+    every output the library writes sits between two 256-byte regions of a known pattern; a write
+    past either end of a buffer shows up as a damaged guard."""
+
+    def __init__(self, dev):
+        self.dev = dev
+        self._all = []
+
+    def _alloc(self, n, dtype, fill):
+        n = max(1, int(n))
+        whole = torch.full((n + 2 * GUARD_WORDS,), GUARD_PATTERN, dtype=torch.int32, device=self.dev)
+        body = whole[GUARD_WORDS:GUARD_WORDS + n]
+        view = body.view(dtype)
+        view.fill_(fill)
+        self._all.append((whole, n))
+        return view
+
+    def i32(self, n):
+        return self._alloc(n, torch.int32, 0x7FFFFFFF)
+
+    def f32(self, n):
+        return self._alloc(n, torch.float32, float("nan"))
+
+    def check(self):
+        for whole, n in self._all:
+            front = whole[:GUARD_WORDS]
+            back = whole[GUARD_WORDS + n:]
+            assert bool((front == GUARD_PATTERN).all()) and bool((back == GUARD_PATTERN).all()), \
+                f"a kernel wrote outside an output buffer of {n} words"
+
+
 def run_gpu_layer(ctx: B.Context, wl: I.Workload, li: I.LayerInputs, bkw: dict, want_logits=True,
                   placement=None, pair_limit=0):
     """All entry points on one layer; returns numpy copies of every output.
@@ -73,9 +112,10 @@ def run_gpu_layer(ctx: B.Context, wl: I.Workload, li: I.LayerInputs, bkw: dict, 
     budget = B.make_budget(**bkw)
     ms = max(1, budget.max_swaps)
 
-    def u32(n): return torch.full((n,), 0x7FFFFFFF, dtype=torch.int32, device=dev)
+    guarded = GuardedOutputs(dev)
+    u32 = guarded.i32
     counts, ids_early = u32(E), u32(max(1, T * k)).view(-1)
-    logits_early = torch.full((max(1, T * E),), float("nan"), device=dev) if want_logits else None
+    logits_early = guarded.f32(T * E) if want_logits else None
     ctx.fb_predict_load(router, h_prev, T, counts, ids_early, logits_early)
     pi_out, swaps, n_swaps, lb4, la4 = u32(E), u32(4 * ms), u32(1), u32(R), u32(R)
     ctx.fb_plan_swaps(counts, pi, budget, 0, pi_out, swaps, n_swaps, lb4, la4)
@@ -83,21 +123,22 @@ def run_gpu_layer(ctx: B.Context, wl: I.Workload, li: I.LayerInputs, bkw: dict, 
     f_counts, f_pi_out, f_swaps, f_n, f_lb, f_la = u32(E), u32(E), u32(4 * ms), u32(1), u32(R), u32(R)
     ctx.fb_predict_and_plan(router, h_prev, T, pi, budget, 0, f_counts, f_pi_out, f_swaps, f_n, f_lb, f_la)
     ids = u32(max(1, T * k))
-    w = torch.full((max(1, T * k),), float("nan"), device=dev)
+    w = guarded.f32(T * k)
     slot_offsets, rank_offsets, rank_load = u32(E + 1), u32(R + 1), u32(R)
     perm, inv_perm = u32(max(1, T * k)), u32(max(1, T * k))
-    logits = torch.full((max(1, T * E),), float("nan"), device=dev) if want_logits else None
+    logits = guarded.f32(T * E) if want_logits else None
     ctx.fb_route_dispatch(router, H, T, f_pi_out, ids, w, slot_offsets, rank_offsets, perm, inv_perm, rank_load,
                           logits)
     # the whole layer in one call, into buffers of its own
     l_counts, l_pi_out, l_swaps, l_n, l_lb, l_la = u32(E), u32(E), u32(4 * ms), u32(1), u32(R), u32(R)
-    l_ids, l_w = u32(max(1, T * k)), torch.full((max(1, T * k),), float("nan"), device=dev)
+    l_ids, l_w = u32(max(1, T * k)), guarded.f32(T * k)
     l_so, l_ro, l_rl = u32(E + 1), u32(R + 1), u32(R)
     l_perm, l_inv = u32(max(1, T * k)), u32(max(1, T * k))
     ctx.fb_layer_step(router, h_prev, H, T, pi, budget, 0, l_counts, l_pi_out, l_swaps, l_n, l_lb, l_la,
                       l_ids, l_w, l_so, l_ro, l_perm, l_inv, l_rl)
     status = ctx.fb_device_status()
     torch.cuda.synchronize(dev)
+    guarded.check()
     ctx.fb_set_pair_limit(0)
     n = int(n_swaps.item())
     fn = int(f_n.item())
@@ -158,12 +199,21 @@ def compare_routing(name, z_gpu, ids_gpu, z_ref, ids_ref, gate, select_bias, rep
         assert (np.diff(srt, axis=1) > 0).all() if gate.k > 1 else True, f"{name}: duplicate expert in a token"
     key_gap, group_gap = O.near_tie_margins(z_ref, gate, select_bias)
     mism = _set_mismatch(ids_gpu, ids_ref)
-    for tag, eps in (("", NEAR_TIE), ("_tight", NEAR_TIE_TIGHT)):
+    # How far a selection key can be off, given the logit error measured above: a softmax key
+    # is the logit; a sigmoid key moves by at most a quarter of the logit error, plus the
+    # kernel's approximate exp / reciprocal and the fp32 rounding of the key (< 1e-6 together).
+    tight = NEAR_TIE_TIGHT
+    if z_gpu is not None and T:
+        key_err = err if gate.gate == O.GATE_SOFTMAX_TOPK else 0.25 * err + 1e-6
+        tight = max(tight, 2.0 * key_err)
+    report[f"{name}_tight_eps"] = tight
+    for tag, eps in (("", NEAR_TIE), ("_tight", tight)):
         flagged = (key_gap < eps) | (group_gap < 2 * eps)
         report[f"{name}_flagged{tag}"] = int(flagged.sum())
         report[f"{name}_mismatch_flagged{tag}"] = int((mism & flagged).sum())
         report[f"{name}_mismatch_unflagged{tag}"] = int((mism & ~flagged).sum())
     assert report[f"{name}_mismatch_unflagged"] == 0, f"{name}: {report}"
+    assert report[f"{name}_mismatch_unflagged_tight"] == 0, f"{name}: {report}"
     return mism
 
 

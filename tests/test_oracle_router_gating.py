@@ -182,3 +182,56 @@ def test_near_tie_margins():
     assert np.isinf(group_gap).all()
     key_gap, _ = O.near_tie_margins(z, O.Gate(E=4, k=4))
     assert np.isinf(key_gap).all()
+
+
+def test_near_tie_margins_group_gap_hand_worked():
+    """The group-score gap decides which tokens a parity check may exempt, so it is pinned to
+    hand-worked numbers: zero logits make every sigmoid exactly 0.5 and the key 0.5 + bias."""
+    import json
+    import os
+    with open(os.path.join(os.path.dirname(__file__), "golden", "near_tie_group_gap.json")) as f:
+        g = json.load(f)
+    keys = np.array(g["keys"], dtype=np.float64)
+    gate = O.Gate(E=g["E"], k=g["k"], gate=O.GATE_SIGMOID_GROUP_TOPK, n_group=g["n_group"],
+                  topk_group=g["topk_group"])
+    all_kept = O.Gate(E=g["E"], k=g["k"], gate=O.GATE_SIGMOID_GROUP_TOPK, n_group=g["n_group"],
+                      topk_group=g["n_group"])
+    for r in range(keys.shape[0]):               # one token at a time: its keys as the per-expert bias
+        z1 = np.zeros((1, g["E"]))
+        key_gap, group_gap = O.near_tie_margins(z1, gate, keys[r] - 0.5)
+        assert abs(key_gap[0] - g["key_gap"][r]) < 1e-12
+        assert abs(group_gap[0] - g["group_gap"][r]) < 1e-12
+        # every group kept: no dropped group, every expert eligible
+        key_gap3, group_gap3 = O.near_tie_margins(z1, all_kept, keys[r] - 0.5)
+        assert np.isinf(group_gap3).all()
+        assert abs(key_gap3[0] - g["key_gap_all_groups_kept"][r]) < 1e-12
+    # both tokens in one call, the keys reached through the logits (sigmoid of the logit of a
+    # key returns it to rounding error); then with the rows swapped: the gaps travel with
+    # their rows, which catches a sort along the wrong axis
+    z = np.log(keys.clip(1e-300) / (1.0 - keys))
+    z[keys == 0.0] = -800.0                      # sigmoid(-800) == 0 in float64
+    key_gap, group_gap = O.near_tie_margins(z, gate)
+    assert np.allclose(key_gap, g["key_gap"], atol=1e-9) and np.allclose(group_gap, g["group_gap"], atol=1e-9)
+    key_gap2, group_gap2 = O.near_tie_margins(z[::-1], gate)
+    assert np.allclose(key_gap2, g["key_gap"][::-1], atol=1e-9)
+    assert np.allclose(group_gap2, g["group_gap"][::-1], atol=1e-9)
+
+
+def test_near_tie_margins_bound_actual_flips():
+    """Property: perturbing every logit by less than half the smaller margin (scaled to key
+    units) never changes a token's expert set; a token whose set changes under a perturbation
+    has a margin below twice that perturbation."""
+    rng = np.random.default_rng(11)
+    T, E = 400, 16
+    gate = O.Gate(E=E, k=4, gate=O.GATE_SIGMOID_GROUP_TOPK, n_group=4, topk_group=2)
+    z = rng.standard_normal((T, E))
+    bias = 0.02 * rng.standard_normal(E)
+    ids, _ = O.select_topk(z, gate, bias)
+    key_gap, group_gap = O.near_tie_margins(z, gate, bias)
+    eps = 2e-2                                   # logit perturbation; keys move by at most eps / 4
+    ids2, _ = O.select_topk(z + rng.uniform(-eps, eps, size=z.shape), gate, bias)
+    changed = (np.sort(ids, axis=1) != np.sort(ids2, axis=1)).any(axis=1)
+    assert changed.any()                         # the perturbation is large enough to matter
+    dk = eps / 4                                 # |d sigmoid| <= |dz| / 4
+    safe = (key_gap > 2 * dk) & (group_gap > 4 * dk)
+    assert not (changed & safe).any()

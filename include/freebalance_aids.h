@@ -27,6 +27,16 @@ uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
  * alone inside a call that launches several kernels. */
 fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
 
+/* Phase time stamps of the one-tile router kernel.  Only a library built with -DFB_TIMING
+ * carries the stamp code (paper_2608_14205_b200/phase_timing.py builds one beside the normal
+ * library and prints the table); the normal build returns FB_ERR_UNSUPPORTED_SHAPE here and
+ * its kernels contain none of it.  stamps: dev u64 [blocks][64], or NULL to stop stamping:
+ * every block of every following router launch through ctx writes the global nanosecond
+ * timer in slots 0..31 and the SM cycle counter in slots 32..63 at its phase boundaries
+ * (the slot list is at the top of csrc/fb_router.cuh).  The buffer must hold 64 words per
+ * block of the largest launch. */
+fb_status fb_set_stamp_buffer(fb_ctx* ctx, uint64_t* stamps);
+
 /* Self-test of the bounded wait that every kernel of the library uses for its barriers: a
  * one-block kernel waits for at most limit_ns (1 .. 100 000 000) on a barrier at which
  * nobody ever arrives, gives up, records FB_ERR_TIMEOUT in ctx's device status word and

@@ -51,7 +51,8 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
            "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
-           "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout"]
+           "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
+           "fb_set_stamp_buffer"]
 
 _lib = None
 
@@ -69,7 +70,7 @@ def lib() -> ctypes.CDLL:
     if _lib is not None:
         return _lib
     path = _build.LIB_PATH
-    if _build.is_stale():
+    if _build.is_stale():                    # (a variant selected with build.use_library is built by its caller)
         path = _build.build()
     if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing: build it with paper_2608_14205_b200/build.py")
@@ -99,6 +100,8 @@ def lib() -> ctypes.CDLL:
     L.fb_set_pair_limit.restype = ctypes.c_int
     L.fb_max_pairs.argtypes = [vp]
     L.fb_max_pairs.restype = i32
+    L.fb_set_stamp_buffer.argtypes = [vp, vp]
+    L.fb_set_stamp_buffer.restype = ctypes.c_int
     L.fb_selftest_wait_timeout.argtypes = [vp, u64, vp, vp]
     L.fb_selftest_wait_timeout.restype = ctypes.c_int
     L.fb_row_cosine_mean.argtypes = [vp, vp, ctypes.c_int64, i32, i32, vp, vp, vp]
@@ -309,6 +312,10 @@ class Context:
 
     def fb_max_pairs(self) -> int:
         return int(lib().fb_max_pairs(self._h))
+
+    def fb_set_stamp_buffer(self, stamps) -> None:
+        """Only libraries built with -DFB_TIMING accept this (see phase_timing.py)."""
+        _check(lib().fb_set_stamp_buffer(self._h, _ptr(stamps)), "fb_set_stamp_buffer")
 
     def fb_selftest_wait_timeout(self, limit_ns: int, waited_ns=None, stream=None) -> None:
         _check(lib().fb_selftest_wait_timeout(self._h, limit_ns, _ptr(waited_ns), _stream(stream)),

@@ -75,7 +75,8 @@ struct fb_ctx {
   int32_t* st_perm = nullptr; int32_t* st_inv_perm = nullptr; uint32_t* st_rank_load = nullptr;
   uint64_t launches = 0;
   uint64_t persistent_launches = 0;
-  cudaEvent_t ev_before = nullptr, ev_after = nullptr;   // one-shot: recorded around the next router launch     // of those, launches of the persistent router kernel
+  cudaEvent_t ev_before = nullptr, ev_after = nullptr;   // one-shot: recorded around the next router launch
+  unsigned long long* stamps = nullptr;                  // caller's phase-stamp buffer (FB_TIMING builds)
 };
 
 namespace {
@@ -166,6 +167,7 @@ fb_status fill_plan(const fb_ctx* ctx, const fb_budget* b, const int32_t* pi, in
     pp->fs_per_byte[c] = b->fs_per_byte[c];
     pp->uniform_cost_ns[c] = uniform_cost(*b, c);
     if (b->expert_bytes_table == nullptr && pp->uniform_cost_ns[c] == 0) return FB_ERR_INVALID_ARG;
+    pp->uniform_link_cap[c] = pp->uniform_cost_ns[c] ? b->link_ns / pp->uniform_cost_ns[c] : 0;
   }
   pp->ranks_per_node = b->ranks_per_node;
   pp->expert_bytes_table = b->expert_bytes_table;
@@ -237,6 +239,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.topk_w = topk_w;
   p.logits = logits;
   p.tile_counts = ctx->tile_counts;
+  p.stamps = ctx->stamps;
   if (plan) p.plan = *plan;
   const int tiles_pad = pair ? (tiles + 1) / 2 * 2 : tiles;       // a pair never straddles the two passes
   int blocks = mode == fb::kModeLayer ? 2 * tiles_pad : tiles_pad;
@@ -909,6 +912,17 @@ fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* even
 }
 
 int32_t fb_max_pairs(const fb_ctx* ctx) { return ctx ? ctx->max_pairs : 0; }
+
+fb_status fb_set_stamp_buffer(fb_ctx* ctx, uint64_t* stamps) {
+  if (!ctx) return FB_ERR_INVALID_ARG;
+#ifdef FB_TIMING
+  ctx->stamps = reinterpret_cast<unsigned long long*>(stamps);
+  return FB_OK;
+#else
+  (void)stamps;
+  return FB_ERR_UNSUPPORTED_SHAPE;      // this build carries no stamp code
+#endif
+}
 
 fb_status fb_selftest_wait_timeout(fb_ctx* ctx, uint64_t limit_ns, uint64_t* waited_ns, fb_stream stream_) {
   if (!ctx || limit_ns == 0 || limit_ns > 100ull * 1000 * 1000) return FB_ERR_INVALID_ARG;

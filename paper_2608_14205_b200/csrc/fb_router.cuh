@@ -33,6 +33,31 @@
 #include "fb_planner.cuh"
 #include "fb_ptx.cuh"
 
+#ifndef FB_PDL_TRIGGER
+#define FB_PDL_TRIGGER 0
+#endif
+
+// Phase time stamps (builds with -DFB_TIMING only; see fb_set_stamp_buffer): one designated
+// thread per role writes %globaltimer (slot i) and clock64 (slot 32 + i) of its block at the
+// phase boundaries below.  Without the flag the macro is empty and the kernels carry none of it.
+//   0 block start          1 set-up done            2 accumulators complete  3 keys computed
+//   4 barrier              5 groups chosen          7 candidates collected   8 candidates ranked
+//   9 top-k read back     10 outputs written       11 counts published      12 planner done
+//  13 block exit          14 first load issued     15 last load issued      16 first operands landed
+//  17 last MMA issued     18 planner entered       19 rank loads formed    20 greedy loop left
+#ifdef FB_TIMING
+#define FB_STAMP(i, who)                                                                    \
+  do {                                                                                      \
+    if (p.stamps != nullptr && threadIdx.x == (who)) {                                      \
+      unsigned long long* st_ = p.stamps + static_cast<size_t>(blockIdx.x) * 64;           \
+      st_[i] = global_timer_ns();                                                           \
+      st_[32 + (i)] = static_cast<unsigned long long>(clock64());                           \
+    }                                                                                       \
+  } while (0)
+#else
+#define FB_STAMP(i, who) do { } while (0)
+#endif
+
 namespace fb {
 
 constexpr int kTileM = 128;            // token rows per block
@@ -75,6 +100,7 @@ struct RouterParams {
   float* topk_w;                     // [T][k] or nullptr
   float* logits;                     // [T][E] or nullptr
   uint32_t* tile_counts;             // [tiles][E]    (dispatch mode)
+  unsigned long long* stamps;        // [blocks][64] phase time stamps (FB_TIMING builds) or nullptr
   PlanParams plan;
 };
 
@@ -301,22 +327,38 @@ __device__ __forceinline__ void publish_counts(Shared& sh, const RouterParams& p
     // fence (cumulative) publishes them device-wide before the ticket is taken.
     __threadfence();
     const uint32_t prev = atomicAdd(p.ticket, 1u);
-    sh.is_last = (prev == static_cast<uint32_t>(p.ticket_target) - 1) ? 1 : 0;
+    const bool last = prev == static_cast<uint32_t>(p.ticket_target) - 1;
+    // Acquire side of the same hand-shake: the other blocks' counts are visible to this thread
+    // after the fence and, through the barrier below, to the whole block.
+    if (last) __threadfence();
+    sh.is_last = last ? 1 : 0;
   }
   named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+  FB_STAMP(11, 64);
   if (sh.is_last) {
     // Every other tile has published its counts: this block finishes the pass.
-    __threadfence();
     for (int e = et; e < p.E; e += kEpilogueThreads) {
       const uint32_t c = __ldcg(&p.counts_scratch[e]);
       p.counts_out[e] = c;
-      sh.plan.cnt[e] = c;
+      if (run_planner) plan_put_count(sh.plan, e, c);
       p.counts_scratch[e] = 0;           // ready for the next call
     }
     if (et == 0) *p.ticket = 0;
     if (sh.abort_flag) { if (et == 0) atomicCAS(p.status, 0, FB_ERR_TIMEOUT); }
-    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-    if (run_planner && warp == 2) plan_swaps_warp(p.plan, sh.plan, lane, p.status);
+    if (run_planner) {
+      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      if (warp == 2) {
+#ifdef FB_TIMING
+        PlanParams pt = p.plan;
+        pt.stamps = p.stamps != nullptr ? p.stamps + static_cast<size_t>(blockIdx.x) * 64 : nullptr;
+        plan_swaps_warp(pt, sh.plan, lane, p.status);
+#else
+        plan_swaps_warp(p.plan, sh.plan, lane, p.status);
+#endif
+      }
+      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      plan_write_placement(p.plan, sh.plan, et, kEpilogueThreads);
+    }
   }
 }
 
@@ -359,6 +401,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   const uint32_t stage_bytes = kATileBytes + b_tile_bytes;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzle atoms need 1024-byte alignment
   volatile int* abort_flag = &sh.abort_flag;
+  FB_STAMP(0, 64);
 
   if (threadIdx.x == 0) {
     sh.abort_flag = 0;
@@ -391,7 +434,11 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   // Everything above touched only this block's own state and the call's parameters; from here on
   // the kernel reads memory that earlier work of the stream may have written.
   pdl_wait();
+#if FB_PDL_TRIGGER == 1
+  pdl_launch_dependents();
+#endif
   const uint32_t tmem_base = sh.tmem_base;
+  FB_STAMP(1, 64);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -402,6 +449,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int s = kb % p.stages;
         const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
         if (!mbar_wait<kCtas == 2>(smem_u32(&sh.empty_bar[s]), phase ^ 1u, abort_flag)) break;
+        if (kb == 0) FB_STAMP(14, 0);
+        if (kb == p.num_kb - 1) FB_STAMP(15, 0);
         const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
         if (kCtas == 1) {
           const uint32_t full = smem_u32(&sh.full_bar[s]);
@@ -419,6 +468,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
       }
     }
+    __syncwarp();
+    if (kCtas == 2) cluster_arrive();          // this warp is done with the pair's shared state (see the teardown)
   } else if (warp == 1 || warp == kSecondIssuerWarp) {
     // ------------------------------------------------------------ MMA issuers
     // warp 1: k-blocks 0, 2, 4, ... into accumulator 0; the last warp: 1, 3, 5, ... into
@@ -434,6 +485,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         ok = mbar_wait<kCtas == 2>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
         if (!ok) break;
         tcgen05_fence_after();
+        if (kb == 0) FB_STAMP(16, 32);
         const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
         const uint64_t adesc = umma_smem_desc_sw128(a_addr);
         const uint64_t bdesc = umma_smem_desc_sw128(a_addr + kATileBytes);
@@ -446,6 +498,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.empty_bar[s]));
         else umma_commit_2cta(smem_u32(&sh.empty_bar[s]), 0x3);
       }
+      if (warp == 1) FB_STAMP(17, 32);
       // this issuer's accumulator is complete
       if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.accum_bar));
       else umma_commit_2cta(smem_u32(&sh.accum_bar), 0x3);
@@ -457,6 +510,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     __syncwarp();
     named_bar_arrive(kAccumBarrierId, kEpilogueThreads + 32);
     }
+    __syncwarp();
+    if (kCtas == 2) cluster_arrive();
   } else {
     // ------------------------------------------------------------ epilogue
     const int et = threadIdx.x - 64;                       // 0 .. kEpilogueThreads-1
@@ -500,6 +555,10 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     named_bar_sync(kAccumBarrierId, kEpilogueThreads + 32);
     const bool got = sh.accum_ok != 0;
     tcgen05_fence_after();
+    FB_STAMP(2, 64);
+#if FB_PDL_TRIGGER == 2
+    pdl_launch_dependents();
+#endif
 
     // scratch carved out of the (now idle) pipeline stages
     float* key_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // [N][128]
@@ -643,8 +702,13 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
       }
     }
+    FB_STAMP(3, 64);
     tcgen05_fence_before();
+    // This warp has read its part of tensor memory: its share of the pair's closing barrier
+    // is delivered now, so that nobody waits for it at the end (see the teardown).
+    if (kCtas == 2) cluster_arrive();
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    FB_STAMP(4, 64);
     if (got && fast_select) {
       // ---------------- choose: rank the (at most 8) group scores of this row
       unsigned long long* cand = reinterpret_cast<unsigned long long*>(merge_v);   // [kCandCap][128], see rank_candidates
@@ -671,6 +735,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (sub < n_chunks) my_groups[0] = sub;
         if (sub + kEpiSubs < n_chunks) my_groups[1] = sub + kEpiSubs;
       }
+      FB_STAMP(5, 64);
       // ---------------- collect the keys >= floor (at least k keys qualify: the bound is one of k known keys)
 #pragma unroll 1
       for (int gi = 0; gi < 2; ++gi) {
@@ -696,6 +761,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
     }
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    FB_STAMP(7, 64);
     uint32_t* out_hi = reinterpret_cast<uint32_t*>(gscore_s);               // [8][128], group scores are dead now
     uint32_t* out_lo = out_hi + FB_MAX_TOPK * kTileM;
     bool overflow = false;
@@ -704,6 +770,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                  row_in_tile, out_hi, out_lo);
     }
     named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+    FB_STAMP(8, 64);
     if (got && fast_select && sub == 0) {
       if (!overflow) read_ranked(top, k, out_hi, out_lo, row_in_tile);
       if (__any_sync(0xffffffffu, overflow)) {
@@ -849,8 +916,10 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
     }
 
+    FB_STAMP(9, 64);
     // ---- outputs per row
     if (writer) write_row_outputs(top, p, row, out_ids, out_w, sh.select_bias, sm_max, sm_sum);
+    FB_STAMP(10, 64);
     // ---- histogram: one shared-memory atomic per distinct expert per warp (Eq. 5)
     if (sub == 0) {
       if (E > 32) {
@@ -878,17 +947,23 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     } else {
       publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
     }
+    FB_STAMP(12, 64);
   }
 
   // ---------------------------------------------------------------- teardown
+  // Tensor memory may be released, and a block may leave, only when both blocks of the pair
+  // are done with it: every warp has delivered its arrival for the pair's barrier as soon as
+  // its own last access was over (producer and issuers after their loops, epilogue warps after
+  // reading the accumulators), so this wait normally finds the barrier complete.
   tcgen05_fence_before();
   __syncthreads();
-  if (kCtas == 2) { cluster_arrive(); cluster_wait(); }   // nobody leaves while the partner may still signal it
+  if (kCtas == 2) cluster_wait();
   if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(p.status, 0, FB_ERR_TIMEOUT);
   if (warp == 1) {
     tcgen05_fence_after();
     tmem_dealloc<kCtas>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
   }
+  FB_STAMP(13, 64);
 }
 
 // Self-test of the bounded wait every kernel of this library relies on: one thread waits, for
@@ -916,10 +991,13 @@ fb_plan_kernel(const __grid_constant__ PlanParams p, const uint32_t* __restrict_
   __shared__ PlanShared sh;
   const int t = threadIdx.x;
   plan_clear(sh, t, kPlanThreads);
-  for (int e = t; e < p.E; e += kPlanThreads) sh.cnt[e] = counts[e];
   __syncwarp();
   plan_load_placement(p, sh, t, kPlanThreads);
+  __syncwarp();
+  for (int e = t; e < p.E; e += kPlanThreads) plan_put_count(sh, e, counts[e]);
   plan_swaps_warp(p, sh, t, status);
+  __syncwarp();
+  plan_write_placement(p, sh, t, kPlanThreads);
 }
 
 }  // namespace fb

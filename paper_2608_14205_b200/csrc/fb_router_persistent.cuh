@@ -122,6 +122,9 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
   // Everything above touched only this block's own state and the call's parameters; from here on
   // the kernel reads memory that earlier work of the stream may have written.
   pdl_wait();
+#if FB_PDL_TRIGGER == 1
+  pdl_launch_dependents();
+#endif
   const uint32_t tmem_base = sh.tmem_base;
 
   if (warp == 0) {

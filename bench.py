@@ -21,7 +21,6 @@ import json
 import os
 import statistics
 import sys
-import threading
 import time
 
 import torch
@@ -56,54 +55,81 @@ def budget_kwargs(wl: I.Workload, T: int):
                 ranks_per_node=wl.ranks_per_node, expert_bytes=wl.expert_bytes)
 
 
-class ClockSampler:
-    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
-
-    def __init__(self, index: int, period_s: float = 0.002):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
-        self._stop = threading.Event()
-        self._thread = None
-        self._period = period_s
-        try:
-            import pynvml
-            pynvml.nvmlInit()
-            self._nv = pynvml
-            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
-            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
-        except Exception:
-            self._nv = None
-
-    def _loop(self):
-        nv = self._nv
-        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
-                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
-                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
-                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+def _clock_sampler_main(index, period_s, go, stop, times, mhz, reasons, count, max_mhz):
+    """Body of the sampler process: polls NVML (read-only) as fast as `period_s` allows."""
+    try:
+        import pynvml as nv
+        nv.nvmlInit()
+        h = nv.nvmlDeviceGetHandleByIndex(index)
+        max_mhz.value = int(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
         get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
             getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons", None)
-        while not self._stop.is_set():
-            try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
-                if get_reasons is not None:
-                    r = int(get_reasons(self._h))
-                    for name, bit in names.items():
-                        if r & bit:
-                            self.reasons.add(name)
-            except Exception:
-                pass
-            time.sleep(self._period)
+    except Exception:
+        max_mhz.value = -1
+        return
+    go.wait()
+    n, cap = 0, len(times)
+    while not stop.is_set() and n < cap:
+        try:
+            mhz[n] = int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+            reasons[n] = int(get_reasons(h)) if get_reasons is not None else 0
+            times[n] = time.perf_counter()
+            n += 1
+            count.value = n
+        except Exception:
+            pass
+        if period_s > 0:
+            time.sleep(period_s)
+
+
+class ClockSampler:
+    """SM clock and throttle reasons through NVML (read-only) while the timed region runs.
+
+    The polling loop lives in a process of its own: a thread of this process would share the
+    interpreter lock with the loop that launches the kernels and get a sample every few
+    milliseconds at best.  Samples carry host time stamps (the same monotonic clock in both
+    processes); the caller marks the timed region with `window`."""
+    REASONS = {"sw_power_cap": 0x4, "hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40}
+
+    def __init__(self, index: int, period_s: float = 0.0001, capacity: int = 200000):
+        import multiprocessing as mp
+        ctx = mp.get_context("spawn")
+        self.window = [None, None]           # host times that bracket the timed region
+        self._go, self._stop = ctx.Event(), ctx.Event()
+        self._times = ctx.Array("d", capacity, lock=False)
+        self._mhz = ctx.Array("i", capacity, lock=False)
+        self._reasons = ctx.Array("q", capacity, lock=False)
+        self._count = ctx.Value("i", 0, lock=False)
+        self._max = ctx.Value("i", 0, lock=False)
+        self._proc = ctx.Process(target=_clock_sampler_main, daemon=True,
+                                 args=(index, period_s, self._go, self._stop, self._times, self._mhz, self._reasons,
+                                       self._count, self._max))
+        try:
+            self._proc.start()
+        except Exception:
+            self._proc = None
 
     def start(self):
-        if self._nv is not None:
-            self._thread = threading.Thread(target=self._loop, daemon=True)
-            self._thread.start()
+        self._go.set()
 
     def stop(self):
         self._stop.set()
-        if self._thread is not None:
-            self._thread.join(timeout=2)
-        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        self._go.set()
+        if self._proc is not None:
+            self._proc.join(timeout=5)
+        n = int(self._count.value)
+        t0, t1 = self.window
+        idx = [i for i in range(n) if t0 is not None and t1 is not None and t0 <= self._times[i] <= t1]
+        use = idx if len(idx) >= 3 else list(range(n))
+        mhz = [self._mhz[i] for i in use]
+        bits = 0
+        for i in use:
+            bits |= int(self._reasons[i])
+        return {"sm_mhz": statistics.median(mhz) if mhz else None,
+                "sm_max_mhz": int(self._max.value) if self._max.value > 0 else None,
+                "reasons": sorted(name for name, bit in self.REASONS.items() if bits & bit),
+                "samples": len(use), "samples_in_timed_region": len(idx), "samples_total": n,
+                "sm_mhz_min": min(mhz) if mhz else None}
 
 
 def max_over_ranks(value: float, device=None) -> float:
@@ -197,6 +223,8 @@ def main():
                     help="layer: fb_layer_step (default); separate: fb_predict_and_plan + fb_route_dispatch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
+    ap.add_argument("--no-probe", action="store_true",
+                    help="skip the per-kernel timing passes after the bracketed region (for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -220,6 +248,8 @@ def main():
     if distributed:
         dist.init_process_group("nccl", device_id=dev)
 
+    # the clock sampler's process starts now (it needs a second to load NVML) and waits for start()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
     T, E, R, k, d = wl.T, wl.E, wl.R, wl.k, wl.d
     bkw = budget_kwargs(wl, T)
     budget = B.make_budget(**bkw)
@@ -268,44 +298,75 @@ def main():
     if ctx.fb_device_status() != 0:
         raise SystemExit("device status non-zero after warm-up")
 
-    # ---- timed region: exactly K steps; events on the launching (current) stream
+    # ---- timed region: exactly K steps; two events on the launching (current) stream
     K = args.steps
-    # The whole region is bracketed by two events.  The duration of the dominant kernel (the
-    # router kernel: the first launch of the step) comes from a pair of events that the library
-    # records directly around that launch, on every `sample_every`-th step only: an event
-    # between two launches keeps the GPU from starting the next kernel's launch early and
-    # costs about 2 us per record, which would otherwise be charged to every step.
-    sample_every = 8 if K >= 16 else 1
-    sampled = [i for i in range(K) if i % sample_every == 0]
-    ev = {i: [torch.cuda.Event(enable_timing=True) for _ in range(2)] for i in sampled}
-    for pair in ev.values():                 # torch creates the CUDA event on its first record
-        for e in pair:
-            e.record()
     ev_begin, ev_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(physical_gpu_index(local_rank))
     launches0 = ctx.fb_launch_count()
     persistent0 = ctx.fb_persistent_launch_count()
+    # in-kernel clock probe on a side stream: (time, cycle counter) pairs every ~4 us for the
+    # expected length of the region (estimated from a few untimed steps), plus one device time
+    # stamp on the main stream at each end of the region
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(3):
+        step(layers[i % ring])
+    e1.record()
+    barrier()
+    est_region_ns = e0.elapsed_time(e1) / 3 * K * 1e6
+    probe_period_ns = 4000
+    probe_n = int(min(65536, max(64, 1.5 * est_region_ns / probe_period_ns + 64)))
+    probe = torch.zeros(2 * probe_n, dtype=torch.int64, device=dev)
+    marks = torch.zeros(4, dtype=torch.int64, device=dev)
+    side = torch.cuda.Stream(device=dev)
     barrier()
     sampler.start()
+    sampler.window[0] = time.perf_counter()
+    B.fb_clock_probe(probe, probe_n, probe_period_ns, stream=side)
+    B.fb_clock_probe(marks[0:2], 1, 0)
     ev_begin.record()
     for i in range(K):
-        e2 = ev.get(i)
-        if e2:
-            ctx.fb_time_next_router_launch(e2[0], e2[1])
         step(layers[i % ring])
     ev_end.record()
+    B.fb_clock_probe(marks[2:4], 1, 0)
     barrier()
-    clocks = sampler.stop()
+    sampler.window[1] = time.perf_counter()
     launches = ctx.fb_launch_count() - launches0
     persistent_launches = ctx.fb_persistent_launch_count() - persistent0
     total_ms = ev_begin.elapsed_time(ev_end)
-    router_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in sampled]
     total_ms = max_over_ranks(total_ms, dev)
     status = ctx.fb_device_status()
 
-    # ---- the fused predictor + planner alone (fb_predict_and_plan), outside the timed region:
-    # per-launch events, for the roofline fraction of that call by itself
-    pp_n = 0 if args.no_e2e else 24
+    # ---- the dominant kernel (the router kernel: the first launch of a step), timed on
+    # `n_probe` further steps by a pair of events that the library records directly around that
+    # launch.  Kept out of the bracketed region: an event between two launches keeps the GPU from
+    # preparing the next launch early and costs about 2 us per record.  The clock sampler keeps
+    # running, so short bracketed regions still get enough clock samples.
+    n_probe = 0 if args.no_probe else max(16, min(K, 64))
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n_probe)]
+    for pair in ev:                          # torch creates the CUDA event on its first record
+        for e in pair:
+            e.record()
+    barrier()
+    for i in range(n_probe):
+        ctx.fb_time_next_router_launch(ev[i][0], ev[i][1])
+        step(layers[i % ring])
+    barrier()
+    router_ms = [a.elapsed_time(b) for a, b in ev]
+
+    # ---- the fused predictor + planner alone (fb_predict_and_plan), the unit the roofline target
+    # of the method's prediction stage refers to: (1) launches back to back between two events,
+    # repeated, median of the repeats; (2) one event pair per launch
+    pp_n = 0 if args.no_probe else 24
+    pp_b2b = []
+    for _ in range(0 if args.no_probe else 5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(pp_n):
+            predict_and_plan(layers[i % ring])
+        b.record()
+        barrier()
+        pp_b2b.append(a.elapsed_time(b) / pp_n)
     pp_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(pp_n)]
     for i in range(pp_n):
         pp_ev[i][0].record()
@@ -313,15 +374,43 @@ def main():
         pp_ev[i][1].record()
     barrier()
     pp_ms = [a.elapsed_time(b) for a, b in pp_ev]
+    clocks = sampler.stop()
+    # SM clock seen from inside a kernel during the bracketed region
+    side.synchronize()
+    pr = probe.cpu().view(-1, 2).tolist()
+    t_lo, t_hi = int(marks[0].item()), int(marks[2].item())
+    inside = [(t, c) for t, c in pr if t_lo <= t <= t_hi]
+    mhz = []
+    stride = max(1, len(inside) // 64)                    # ~64 windows over the region
+    for i in range(0, len(inside) - stride, stride):
+        dt, dc = inside[i + stride][0] - inside[i][0], inside[i + stride][1] - inside[i][1]
+        if dt > 0:
+            mhz.append(dc / dt * 1e3)
+    clocks["in_kernel"] = {"sm_mhz_median": statistics.median(mhz) if mhz else None,
+                           "sm_mhz_min": min(mhz) if mhz else None, "sm_mhz_max": max(mhz) if mhz else None,
+                           "windows": len(mhz), "samples_in_timed_region": len(inside),
+                           "how": "fb_clock_probe: cycle counter / global timer of a one-thread kernel running "
+                                  "beside the timed steps"}
+
+    # ---- realised rank loads before / after the plan of the last timed step, from the library's
+    # own outputs: counts of the normal pass (fb_predict_load on H), loads under the old placement
+    # (fb_plan_swaps with an empty budget), loads under the new one (rank_load of the step)
+    L_last = layers[(K - 1) % ring]
+    step(L_last)
+    real_counts, real_before, scratch_after = i32(E), i32(R), i32(R)
+    ctx.fb_predict_load(L_last["router"], L_last["H"], T, real_counts)
+    no_swaps = B.make_budget(**dict(bkw, max_swaps=0))
+    ctx.fb_plan_swaps(real_counts, L_last["pi"], no_swaps, 0, i32(E), None, i32(1), real_before, scratch_after)
+    barrier()
 
     # ---- stage 3 on this device (not part of the step): the plan just produced, applied to a buffer
     # of E slot images of the workload's expert size; HBM bound, 4 bytes of traffic per byte moved
     mig = None
-    if not args.no_e2e and wl.expert_bytes > 0 and bkw["max_swaps"] > 0:
+    if not args.no_e2e and not args.no_probe and wl.expert_bytes > 0 and bkw["max_swaps"] > 0:
         S = wl.expert_bytes // 16 * 16
         weights = torch.empty(E * S, dtype=torch.uint8, device=dev)      # content does not matter for timing
         cap = int(bkw["max_swaps"])
-        L0d = layers[(K - 1) % ring]
+        L0d = L_last
         run_mig = lambda: B.fb_apply_swaps(weights, S, E, L0d["pi"], out["swaps"], out["n_swaps"], cap)
         for _ in range(3):
             run_mig()
@@ -373,7 +462,6 @@ def main():
         passes = 2 if layer_api else 1
         alg_bytes = passes * 2 * T * d + 2 * d * E + 4 * E + (8 * T * k if layer_api else 0)
         alg_flops = passes * 2 * T * d * E
-        k1_ms = statistics.mean(router_ms)
 
         def roofline(ms, nbytes, nflops, kernel):
             gbs = nbytes / (ms * 1e-3) / 1e9
@@ -389,31 +477,50 @@ def main():
                     "tensor_tflops": tf, "tensor_frac_of_burst": tf / peaks["bf16_tflops"],
                     "tensor_frac_of_sustained": tf / peaks["bf16_tflops_sustained"]}
 
+        def spread(xs):
+            xs = sorted(xs)
+            return {"min_us": xs[0] * 1e3, "median_us": statistics.median(xs) * 1e3, "max_us": xs[-1] * 1e3,
+                    "n": len(xs)}
+
+        def attach_traffic(block, key):
+            # DRAM bytes per launch come from an ncu capture of the same kernel (not from this run)
+            traffic_file = os.path.join(ROOT, "profiles", "router_kernel_traffic.json")
+            if os.path.exists(traffic_file):
+                with open(traffic_file) as f:
+                    tr = json.load(f)
+                if key in tr:
+                    block["traffic"] = tr[key]
+                    block["traffic_source"] = "profiles/router_kernel_traffic.json (ncu capture of this kernel; " \
+                                              "not measured in this run)"
+
         persistent = persistent_launches > 0
-        kname = ("fb_router_persistent_kernel" if persistent else "fb_router_kernel") + \
-                (" (fb_layer_step: both router passes in one launch)" if layer_api else " (fb_predict_and_plan)")
-        roof = roofline(k1_ms, alg_bytes, alg_flops, kname)
-        roof["kernel_us_median"] = statistics.median(router_ms) * 1e3
-        roof["launches_timed"] = len(router_ms)
-        roof["rest_of_step_us"] = ms_per_step * 1e3 - k1_ms * 1e3
-        traffic_key = wl.name + ("/layer" if layer_api else "")
-        traffic_file = os.path.join(ROOT, "profiles", "router_kernel_traffic.json")
-        if os.path.exists(traffic_file):
-            with open(traffic_file) as f:
-                tr = json.load(f)
-            if traffic_key in tr:
-                roof["traffic"] = tr[traffic_key]
+        roof = None
+        if router_ms:
+            kname = ("fb_router_persistent_kernel" if persistent else "fb_router_kernel") + \
+                    (" (fb_layer_step: both router passes in one launch)" if layer_api else " (fb_predict_and_plan)")
+            k1_ms = statistics.median(router_ms)
+            roof = roofline(k1_ms, alg_bytes, alg_flops, kname)
+            roof["timing"] = "median of one event pair per launch, recorded by the library around the launch"
+            roof["launches_timed"] = len(router_ms)
+            roof["spread"] = spread(router_ms)
+            roof["rest_of_step_us"] = ms_per_step * 1e3 - k1_ms * 1e3
+            attach_traffic(roof, wl.name + ("/layer" if layer_api else ""))
+        roof_pp = None
+        if pp_b2b:
+            pp_bytes, pp_flops = 2 * T * d + 2 * d * E + 4 * E, 2 * T * d * E
+            roof_pp = roofline(statistics.median(pp_b2b), pp_bytes, pp_flops,
+                               "fb_router_kernel + planner tail (fb_predict_and_plan)")
+            roof_pp["timing"] = f"{pp_n} launches back to back between two events, median of {len(pp_b2b)} repeats"
+            roof_pp["spread"] = spread(pp_b2b)
+            roof_pp["tokens_per_s"] = T / (statistics.median(pp_b2b) * 1e-3)
+            per_launch = roofline(statistics.median(pp_ms), pp_bytes, pp_flops, "")
+            roof_pp["per_launch_events"] = dict(spread(pp_ms), frac=per_launch["frac"],
+                                                 note="one event pair per launch: includes launch latency and "
+                                                      "event granularity that back-to-back launches hide")
+            attach_traffic(roof_pp, wl.name)
 
         lb, la = out["load_before"].cpu().tolist(), out["load_after"].cpu().tolist()
-        pi_new = out["pi_out"].cpu().tolist()
-        so = out["slot_offsets"].cpu().tolist()
-        m = E // R
-        realized = [so[pi_new[e] + 1] - so[pi_new[e]] for e in range(E)]
-        pi_old = layers_cpu[(K - 1) % ring].expert_to_slot.tolist()
-        real_before = [0] * R
-        for e in range(E):
-            real_before[pi_old[e] // m] += realized[e]
-        real_after = out["rank_load"].cpu().tolist()
+        real_b, real_a = real_before.cpu().tolist(), out["rank_load"].cpu().tolist()
         mom = lambda L: (max(L) * len(L) / sum(L)) if sum(L) else 1.0
 
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
@@ -432,14 +539,14 @@ def main():
                         "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
                 "gpu_launches": int(launches), "device_status": status,
                 "roofline": roof,
-                "predict_and_plan": None if not pp_ms else dict(
-                    roofline(statistics.mean(pp_ms), 2 * T * d + 2 * d * E + 4 * E, 2 * T * d * E,
-                             "fb_router_kernel (fb_predict_and_plan alone, one event pair per launch)"),
-                    tokens_per_s=T / (statistics.mean(pp_ms) * 1e-3), launches_timed=len(pp_ms)),
+                "roofline_predict_and_plan": roof_pp,
+                "roofline_note": "roofline: the dominant kernel of the timed step; roofline_predict_and_plan: the "
+                                 "fused predictor + planner call by itself (the unit the 70 % target names), "
+                                 "timed back to back",
                 "migration": None if mig is None else dict(
                     mig, frac_of_hbm_peak=(mig["achieved_GBps"] / peaks["hbm_gbs"]) if mig["achieved_GBps"] else None),
                 "load_balance": {"predicted_max_over_mean": [mom(lb), mom(la)],
-                                 "realized_max_over_mean": [mom(real_before), mom(real_after)],
+                                 "realized_max_over_mean": [mom(real_b), mom(real_a)],
                                  "n_swaps": int(out["n_swaps"].item())}}
         if not args.no_cpu_baseline:
             T_s = min(T, 16384)

@@ -27,6 +27,15 @@ uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
  * alone inside a call that launches several kernels. */
 fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
 
+/* SM clock probe.  A one-thread kernel on `stream` writes n pairs (global nanosecond timer,
+ * SM cycle counter) into samples (dev u64 [2 n]), about period_ns apart, and ends by itself
+ * (n <= 65536, period_ns <= 100000: at most a few seconds).  Between two samples the SMs ran
+ * at (cycle difference) / (time difference) GHz: launched on a side stream beside other work
+ * it shows the clock that work really got, at microsecond resolution; with n = 1 on the
+ * work's own stream it is a device time stamp.  Reads counters only; changes no setting.
+ * Errors: FB_ERR_INVALID_ARG for a NULL or non-device buffer or a size out of range. */
+fb_status fb_clock_probe(uint64_t* samples, int32_t n, uint32_t period_ns, fb_stream stream);
+
 /* Phase time stamps of the one-tile router kernel.  Only a library built with -DFB_TIMING
  * carries the stamp code (paper_2608_14205_b200/phase_timing.py builds one beside the normal
  * library and prints the table); the normal build returns FB_ERR_UNSUPPORTED_SHAPE here and

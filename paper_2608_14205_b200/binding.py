@@ -52,7 +52,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
            "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
            "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
-           "fb_set_stamp_buffer"]
+           "fb_set_stamp_buffer", "fb_clock_probe"]
 
 _lib = None
 
@@ -100,6 +100,8 @@ def lib() -> ctypes.CDLL:
     L.fb_set_pair_limit.restype = ctypes.c_int
     L.fb_max_pairs.argtypes = [vp]
     L.fb_max_pairs.restype = i32
+    L.fb_clock_probe.argtypes = [vp, i32, ctypes.c_uint32, vp]
+    L.fb_clock_probe.restype = ctypes.c_int
     L.fb_set_stamp_buffer.argtypes = [vp, vp]
     L.fb_set_stamp_buffer.restype = ctypes.c_int
     L.fb_selftest_wait_timeout.argtypes = [vp, u64, vp, vp]
@@ -230,6 +232,11 @@ def fb_predict_load_static(cfg: FbConfig, device: int, router: FbRouter, x, T: i
     _check(lib().fb_predict_load_static(ctypes.byref(cfg), device, ctypes.byref(router), _ptr(x), T, _ptr(counts),
                                         _ptr(topk_ids), _ptr(status_word), _stream(stream)),
            "fb_predict_load_static")
+
+
+def fb_clock_probe(samples, n: int, period_ns: int, stream=None) -> None:
+    """(global timer ns, SM cycle counter) pairs into `samples` (int64 [2 n]) from a one-thread kernel."""
+    _check(lib().fb_clock_probe(_ptr(samples), n, period_ns, _stream(stream)), "fb_clock_probe")
 
 
 class Context:

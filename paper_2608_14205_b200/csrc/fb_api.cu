@@ -913,6 +913,18 @@ fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* even
 
 int32_t fb_max_pairs(const fb_ctx* ctx) { return ctx ? ctx->max_pairs : 0; }
 
+fb_status fb_clock_probe(uint64_t* samples, int32_t n, uint32_t period_ns, fb_stream stream_) {
+  // bounded by construction: at most 65536 samples, at most 100 us apart
+  if (!samples || n < 1 || n > 65536 || period_ns > 100000) return FB_ERR_INVALID_ARG;
+  const int device = device_of(samples);
+  if (device < 0) return FB_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  fb::fb_clock_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream_)>>>(
+      reinterpret_cast<unsigned long long*>(samples), n, period_ns);
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
 fb_status fb_set_stamp_buffer(fb_ctx* ctx, uint64_t* stamps) {
   if (!ctx) return FB_ERR_INVALID_ARG;
 #ifdef FB_TIMING

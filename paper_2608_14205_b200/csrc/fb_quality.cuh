@@ -105,4 +105,20 @@ fb_topk_hits_kernel(const int32_t* __restrict__ ids_a, const int32_t* __restrict
   if ((threadIdx.x & 31) == 0 && mine) atomicAdd(hits, mine);      // integer sum: order does not matter
 }
 
+// SM clock probe: one thread records (global nanosecond timer, SM cycle counter) pairs, `n` of
+// them about `period_ns` apart, and ends by itself.  The ratio of the differences between two
+// samples is the clock the SMs actually ran at in between - what a kernel sees under load,
+// which the driver's clock query (a few samples per second) cannot resolve.
+__global__ void __launch_bounds__(32, 1)
+fb_clock_probe_kernel(unsigned long long* __restrict__ samples, int n, unsigned period_ns) {
+  if (threadIdx.x != 0) return;
+  for (int i = 0; i < n; ++i) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    samples[2 * i] = t;
+    samples[2 * i + 1] = static_cast<unsigned long long>(clock64());
+    if (period_ns) __nanosleep(period_ns);
+  }
+}
+
 }  // namespace fb

@@ -33,10 +33,6 @@
 #include "fb_planner.cuh"
 #include "fb_ptx.cuh"
 
-#ifndef FB_PDL_TRIGGER
-#define FB_PDL_TRIGGER 0
-#endif
-
 // Phase time stamps (builds with -DFB_TIMING only; see fb_set_stamp_buffer): one designated
 // thread per role writes %globaltimer (slot i) and clock64 (slot 32 + i) of its block at the
 // phase boundaries below.  Without the flag the macro is empty and the kernels carry none of it.
@@ -434,9 +430,13 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   // Everything above touched only this block's own state and the call's parameters; from here on
   // the kernel reads memory that earlier work of the stream may have written.
   pdl_wait();
-#if FB_PDL_TRIGGER == 1
+  // From here on the next kernel of the stream may be scheduled (if it was launched with
+  // programmatic stream serialization - the library's own router launches are): its blocks
+  // take the SMs as this grid's blocks leave them and do their set-up while the last blocks
+  // of this grid finish; they read nothing before their own griddepcontrol.wait, which returns
+  // only when this grid has completed.  Issued after this block's wait, so a dependent never
+  // starts before everything this grid itself depended on is complete.
   pdl_launch_dependents();
-#endif
   const uint32_t tmem_base = sh.tmem_base;
   FB_STAMP(1, 64);
 
@@ -556,9 +556,6 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const bool got = sh.accum_ok != 0;
     tcgen05_fence_after();
     FB_STAMP(2, 64);
-#if FB_PDL_TRIGGER == 2
-    pdl_launch_dependents();
-#endif
 
     // scratch carved out of the (now idle) pipeline stages
     float* key_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // [N][128]

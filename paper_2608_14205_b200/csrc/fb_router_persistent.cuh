@@ -122,9 +122,13 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
   // Everything above touched only this block's own state and the call's parameters; from here on
   // the kernel reads memory that earlier work of the stream may have written.
   pdl_wait();
-#if FB_PDL_TRIGGER == 1
+  // From here on the next kernel of the stream may be scheduled (if it was launched with
+  // programmatic stream serialization - the library's own router launches are): its blocks
+  // take the SMs as this grid's blocks leave them and do their set-up while the last blocks
+  // of this grid finish; they read nothing before their own griddepcontrol.wait, which returns
+  // only when this grid has completed.  Issued after this block's wait, so a dependent never
+  // starts before everything this grid itself depended on is complete.
   pdl_launch_dependents();
-#endif
   const uint32_t tmem_base = sh.tmem_base;
 
   if (warp == 0) {

@@ -26,6 +26,15 @@ itself live in ``tests/test_oracle_*.py``):
                           every iteration's choice, the paper's invariants
                           (budget, no max-load increase, permutation, once per
                           expert), degenerate cases with known empty plans.
+* ``plan_swaps_sweep``   pinned: a hand-worked plan (the first worked example's counts, where
+                          the one pass accepts a second pair that raises the maximum), an
+                          independent integer-only sort-and-sweep on random cases, its
+                          invariants (budget, bijection, once per expert), and agreement with
+                          ``plan_swaps`` whenever at most one swap is allowed.
+* ``plan_swaps_wide``    pinned: a hand-worked plan in which only the second most loaded rank
+                          offers a beneficial swap, exhaustive integer-only replay over the
+                          widened frontier on random cases, equality with ``plan_swaps`` at
+                          width 1.
 * ``dispatch_index``     pinned: brute-force ``sorted`` on tiny inputs, a
                           hand-worked example, permutation/offset invariants.
 * ``budget_ns``          pinned: Eq. 10 special cases.
@@ -225,6 +234,13 @@ class Budget:
     ranks_per_node: int = 0                     # 0 -> every rank in one node
     expert_bytes: int = 0                       # S(e), uniform ...
     expert_bytes_table: Optional[Tuple[int, ...]] = None   # ... or one size per expert
+    mode: int = 0                               # PLAN_LOOP, PLAN_SWEEP or PLAN_WIDE (see plan())
+    frontier_width: int = 1                     # PLAN_WIDE: ranks taken from each end of the load order
+
+
+PLAN_LOOP = 0        # Algorithm 1: re-enumerate the frontier after every accepted swap
+PLAN_SWEEP = 1       # the planner prose: enumerate once, sort once, one pass over the sorted list
+PLAN_WIDE = 2        # Algorithm 1 with the frontier widened to several ranks at each end
 
 
 def budget_ns(t_attn_ns: int, delta_ns: int) -> int:
@@ -342,6 +358,153 @@ def plan_swaps(counts: Sequence[int], expert_to_slot: Sequence[int], R: int, bud
             l_res[lk] = lres - cost
         swaps.append((a, b, ea, eb))
     return swaps, pi, load_before, list(L)
+
+
+def plan_swaps_sweep(counts: Sequence[int], expert_to_slot: Sequence[int], R: int, bud: Budget,
+                     layer_id: int = 0):
+    """The one-pass reading of the planner's ordering paragraph ("Budgeted Expert-Swap
+    Planning"): on the frontier of the given placement (most and least loaded rank)
+    every expert pair is enumerated ONCE, pairs with non-positive benefit (Eq. 8,
+    evaluated under the initial loads) are removed, the rest is sorted ONCE by
+    decreasing benefit / cost (ties: layer, source rank, destination rank, expert
+    ids), and the sorted list is swept: a pair is accepted if neither expert has been
+    selected and every residual budget covers its cost; loads (Eqs. 6, 7) and residual
+    budgets are updated after each accepted pair, the order is not.  Same return value
+    as plan_swaps.  Unlike Algorithm 1's loop, later pairs were scored against loads
+    that earlier acceptances have since changed, so the maximum rank load can rise."""
+    E = len(counts)
+    m = E // R
+    n = [int(c) for c in counts]
+    pi = [int(p) for p in expert_to_slot]
+    gamma = Fraction(bud.gamma_num, bud.gamma_den) if bud.gamma_den else Fraction(0)
+    L = rank_loads(n, pi, R)
+    load_before = list(L)
+    swaps = []
+    a = max(range(R), key=lambda r: (L[r], -r))
+    b = min(range(R), key=lambda r: (L[r], r))
+    if bud.max_swaps == 0 or L[a] - L[b] <= bud.tau_tokens:
+        return swaps, pi, load_before, list(L)
+    phi = objective(L, gamma)
+    cands = []
+    for ea in (e for e in range(E) if rank_of_slot(pi[e], m) == a):
+        for eb in (e for e in range(E) if rank_of_slot(pi[e], m) == b):
+            Ln = list(L)
+            Ln[a] = L[a] - n[ea] + n[eb]
+            Ln[b] = L[b] - n[eb] + n[ea]
+            benefit = phi - objective(Ln, gamma)
+            if benefit <= 0:
+                continue
+            cost = swap_cost_ns(bud, a, b, ea, eb)
+            cands.append((-(benefit / cost), (layer_id, a, b, ea, eb), cost))
+    cands.sort()                                   # decreasing ratio, then the tie-break tuple
+    selected = [False] * E
+    g_res, ra_res, rb_res, l_res = bud.global_ns, bud.rank_ns, bud.rank_ns, bud.link_ns
+    for _, (_, _, _, ea, eb), cost in cands:
+        if len(swaps) == bud.max_swaps:
+            break
+        if selected[ea] or selected[eb]:
+            continue
+        if bud.global_ns != U64_OFF and cost > g_res:
+            continue
+        if bud.rank_ns != U64_OFF and (cost > ra_res or cost > rb_res):
+            continue
+        if bud.link_ns != U64_OFF and cost > l_res:
+            continue
+        L[a] += n[eb] - n[ea]                       # Eq. 6
+        L[b] += n[ea] - n[eb]                       # Eq. 7
+        pi[ea], pi[eb] = pi[eb], pi[ea]
+        selected[ea] = selected[eb] = True
+        if bud.global_ns != U64_OFF:
+            g_res -= cost
+        if bud.rank_ns != U64_OFF:
+            ra_res -= cost
+            rb_res -= cost
+        if bud.link_ns != U64_OFF:
+            l_res -= cost
+        swaps.append((a, b, ea, eb))
+    return swaps, pi, load_before, list(L)
+
+
+def plan_swaps_wide(counts: Sequence[int], expert_to_slot: Sequence[int], R: int, bud: Budget,
+                    layer_id: int = 0):
+    """Algorithm 1's loop with a wider frontier: instead of only the most and the
+    least loaded rank (the restriction the end of "Budgeted Expert-Swap Planning"
+    describes as the practical choice), every iteration considers the
+    ``frontier_width`` most loaded ranks as sources and the ``frontier_width`` least
+    loaded ranks as destinations (lowest index on equal loads; a source must carry
+    strictly more than its destination).  Benefit (Eq. 8), cost (Eq. 9), budgets,
+    conflicts and the ordering rule are those of plan_swaps; the source and
+    destination rank now take part in the tie-break.  Width 1 is plan_swaps."""
+    E = len(counts)
+    m = E // R
+    W = max(1, min(int(bud.frontier_width), R))
+    n = [int(c) for c in counts]
+    pi = [int(p) for p in expert_to_slot]
+    gamma = Fraction(bud.gamma_num, bud.gamma_den) if bud.gamma_den else Fraction(0)
+    L = rank_loads(n, pi, R)
+    load_before = list(L)
+    selected = [False] * E
+    g_res = bud.global_ns
+    r_res = [bud.rank_ns] * R
+    l_res = {}
+    swaps = []
+    while len(swaps) < bud.max_swaps:
+        top = sorted(range(R), key=lambda r: (-L[r], r))[:W]
+        bottom = sorted(range(R), key=lambda r: (L[r], r))[:W]
+        if L[top[0]] - L[bottom[0]] <= bud.tau_tokens:
+            break
+        phi = objective(L, gamma)
+        best = None
+        for a in top:
+            for b in bottom:
+                if a == b or L[a] <= L[b]:
+                    continue
+                lk = link_id(a, b, bud.ranks_per_node)
+                lres = l_res.get(lk, bud.link_ns)
+                for ea in (e for e in range(E) if rank_of_slot(pi[e], m) == a and not selected[e]):
+                    for eb in (e for e in range(E) if rank_of_slot(pi[e], m) == b and not selected[e]):
+                        Ln = list(L)
+                        Ln[a] = L[a] - n[ea] + n[eb]
+                        Ln[b] = L[b] - n[eb] + n[ea]
+                        benefit = phi - objective(Ln, gamma)
+                        if benefit <= 0:
+                            continue
+                        cost = swap_cost_ns(bud, a, b, ea, eb)
+                        if bud.global_ns != U64_OFF and cost > g_res:
+                            continue
+                        if bud.rank_ns != U64_OFF and (cost > r_res[a] or cost > r_res[b]):
+                            continue
+                        if bud.link_ns != U64_OFF and cost > lres:
+                            continue
+                        ratio = benefit / cost
+                        tie = (layer_id, a, b, ea, eb)
+                        if best is None or ratio > best[0] or (ratio == best[0] and tie < best[1]):
+                            best = (ratio, tie, cost, Ln)
+        if best is None:
+            break
+        _, (_, a, b, ea, eb), cost, L = best
+        pi[ea], pi[eb] = pi[eb], pi[ea]
+        selected[ea] = selected[eb] = True
+        if bud.global_ns != U64_OFF:
+            g_res -= cost
+        if bud.rank_ns != U64_OFF:
+            r_res[a] -= cost
+            r_res[b] -= cost
+        if bud.link_ns != U64_OFF:
+            lk = link_id(a, b, bud.ranks_per_node)
+            l_res[lk] = l_res.get(lk, bud.link_ns) - cost
+        swaps.append((a, b, ea, eb))
+    return swaps, pi, load_before, list(L)
+
+
+def plan(counts: Sequence[int], expert_to_slot: Sequence[int], R: int, bud: Budget, layer_id: int = 0):
+    """The planner in the mode the budget names: Algorithm 1's loop (default), the one-pass
+    sorted sweep, or the loop with a widened frontier."""
+    if bud.mode == PLAN_SWEEP:
+        return plan_swaps_sweep(counts, expert_to_slot, R, bud, layer_id)
+    if bud.mode == PLAN_WIDE:
+        return plan_swaps_wide(counts, expert_to_slot, R, bud, layer_id)
+    return plan_swaps(counts, expert_to_slot, R, bud, layer_id)
 
 
 # ----------------------------------------------------------------------------

@@ -176,6 +176,163 @@ def test_planner_matches_exhaustive_replay(seed):
     assert again == (swaps, pi_out, before, after)       # deterministic
 
 
+# ---------------------------------------------------------------- planner variants
+def _random_plan_case(seed):
+    rng = random.Random(1000 + seed)
+    R = rng.choice([2, 3, 4, 6, 8])
+    m = rng.choice([1, 2, 3, 4])
+    E = R * m
+    counts = [rng.randrange(0, 60) ** rng.choice([1, 2]) for _ in range(E)]
+    pi = list(range(E))
+    if seed % 2:
+        rng.shuffle(pi)
+    kw = dict(max_swaps=rng.choice([1, 2, 5, E]), gamma_num=rng.choice([0, 1, 3]),
+              gamma_den=rng.choice([1, 8, 1000]), tau_tokens=rng.choice([0, 0, 10, 500]))
+    if seed % 3 == 0:
+        kw.update(alpha_ns=(100, 700), fs_per_byte=(2000, 9000), expert_bytes=rng.randrange(1, 10**6),
+                  ranks_per_node=rng.choice([0, 2]), global_ns=rng.choice([O.U64_OFF, 10**4, 10**5]),
+                  rank_ns=rng.choice([O.U64_OFF, 5000, 10**5]), link_ns=rng.choice([O.U64_OFF, 3000, 10**5]))
+    if seed % 5 == 0:
+        kw.update(alpha_ns=(50, 50), fs_per_byte=(10**6, 10**6),
+                  expert_bytes_table=tuple(rng.randrange(1, 500) for _ in range(E)))
+    return counts, pi, R, kw
+
+
+def _int_benefit(L, Ln, gn, gd):
+    """gd * (Phi(L) - Phi(Ln)) in integers: the mean is swap-invariant, so the variance term is
+    a difference of sums of squares."""
+    return gd * (max(L) - max(Ln)) + gn * (sum(x * x for x in L) - sum(x * x for x in Ln))
+
+
+def test_sweep_worked_example(golden):
+    gd = golden("planner_sweep_overshoots.json")
+    b = O.Budget(max_swaps=gd["max_swaps"], gamma_num=gd["gamma_num"], gamma_den=gd["gamma_den"],
+                 tau_tokens=gd["tau_tokens"], mode=O.PLAN_SWEEP)
+    swaps, pi, before, after = O.plan(gd["counts"], gd["expert_to_slot"], gd["R"], b)
+    assert [list(s) for s in swaps] == gd["swaps"]
+    assert pi == gd["expert_to_slot_out"] and before == gd["load_before"] and after == gd["load_after"]
+    assert max(after) >= max(before)          # the recorded weakness of the one-pass reading
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_sweep_matches_independent_sort_and_sweep(seed):
+    counts, pi0, R, kw = _random_plan_case(seed)
+    bud = O.Budget(mode=O.PLAN_SWEEP, **kw)
+    swaps, pi_out, before, after = O.plan(counts, pi0, R, bud, layer_id=seed)
+    # independent restatement: integers only, Python's sort on exact keys
+    E, m = len(counts), len(counts) // R
+    L = [sum(counts[e] for e in range(E) if pi0[e] // m == r) for r in range(R)]
+    assert L == before
+    gn, gd = (bud.gamma_num, bud.gamma_den) if bud.gamma_den else (0, 1)
+    a, b = L.index(max(L)), L.index(min(L))
+    expect, pi, sel, spent = [], list(pi0), set(), 0
+    if L[a] - L[b] > bud.tau_tokens:
+        cands = []
+        for ea in range(E):
+            for eb in range(E):
+                if pi0[ea] // m != a or pi0[eb] // m != b:
+                    continue
+                Ln = list(L)
+                Ln[a] += counts[eb] - counts[ea]
+                Ln[b] += counts[ea] - counts[eb]
+                ben = _int_benefit(L, Ln, gn, gd)
+                if ben > 0:
+                    c = O.swap_cost_ns(bud, a, b, ea, eb)
+                    cands.append((Fraction(-ben, c), ea, eb, c))
+        Lc = list(L)
+        for _, ea, eb, c in sorted(cands):
+            if len(expect) == bud.max_swaps:
+                break
+            if ea in sel or eb in sel:
+                continue
+            # one source, one destination and one link throughout: all three residuals see `spent`
+            if any(lim != O.U64_OFF and spent + c > lim for lim in (bud.global_ns, bud.rank_ns, bud.link_ns)):
+                continue
+            expect.append((a, b, ea, eb))
+            sel |= {ea, eb}
+            spent += c
+            Lc[a] += counts[eb] - counts[ea]
+            Lc[b] += counts[ea] - counts[eb]
+            pi[ea], pi[eb] = pi[eb], pi[ea]
+        L = Lc
+    assert swaps == expect and pi_out == pi and after == L
+    assert sorted(pi_out) == list(range(E)) and sum(after) == sum(before) and len(swaps) <= bud.max_swaps
+    # with room for one swap only, the sweep and Algorithm 1's loop take the same pair
+    one = dict(kw, max_swaps=1)
+    assert O.plan(counts, pi0, R, O.Budget(mode=O.PLAN_SWEEP, **one), seed) == \
+        O.plan_swaps(counts, pi0, R, O.Budget(**one), seed)
+
+
+def test_wide_frontier_worked_example(golden):
+    gd = golden("planner_wide_frontier.json")
+    kw = dict(max_swaps=gd["max_swaps"], gamma_num=gd["gamma_num"], gamma_den=gd["gamma_den"],
+              tau_tokens=gd["tau_tokens"])
+    swaps, pi, before, after = O.plan(gd["counts"], gd["expert_to_slot"], gd["R"],
+                                      O.Budget(mode=O.PLAN_WIDE, frontier_width=gd["frontier_width"], **kw))
+    assert [list(s) for s in swaps] == gd["swaps"]
+    assert pi == gd["expert_to_slot_out"] and before == gd["load_before"] and after == gd["load_after"]
+    narrow = O.plan_swaps(gd["counts"], gd["expert_to_slot"], gd["R"], O.Budget(**kw))
+    assert [list(s) for s in narrow[0]] == gd["narrow_frontier_swaps"]
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_wide_frontier_matches_exhaustive_replay(seed):
+    counts, pi0, R, kw = _random_plan_case(seed)
+    W = 1 + seed % 3
+    bud = O.Budget(mode=O.PLAN_WIDE, frontier_width=W, **kw)
+    swaps, pi_out, before, after = O.plan(counts, pi0, R, bud, layer_id=seed)
+    if W == 1:
+        assert (swaps, pi_out, before, after) == O.plan_swaps(counts, pi0, R, O.Budget(**kw), seed)
+    E, m = len(counts), len(counts) // R
+    gn, gd = (bud.gamma_num, bud.gamma_den) if bud.gamma_den else (0, 1)
+    pi, L = list(pi0), list(before)
+    moved, spent, spent_rank, spent_link = set(), 0, [0] * R, {}
+    for it in range(len(swaps) + 1):
+        order = sorted(range(R), key=lambda r: (-L[r], r))
+        top = order[:min(W, R)]
+        bottom = sorted(range(R), key=lambda r: (L[r], r))[:min(W, R)]
+        cands = []
+        if it < bud.max_swaps and max(L) - min(L) > bud.tau_tokens:
+            for a in top:
+                for b in bottom:
+                    if a == b or L[a] <= L[b]:
+                        continue
+                    for ea in range(E):
+                        for eb in range(E):
+                            if pi[ea] // m != a or pi[eb] // m != b or ea in moved or eb in moved:
+                                continue
+                            Ln = list(L)
+                            Ln[a] += counts[eb] - counts[ea]
+                            Ln[b] += counts[ea] - counts[eb]
+                            ben = _int_benefit(L, Ln, gn, gd)
+                            if ben <= 0:
+                                continue
+                            c = O.swap_cost_ns(bud, a, b, ea, eb)
+                            lk = O.link_id(a, b, bud.ranks_per_node)
+                            if bud.global_ns != O.U64_OFF and spent + c > bud.global_ns:
+                                continue
+                            if bud.rank_ns != O.U64_OFF and max(spent_rank[a], spent_rank[b]) + c > bud.rank_ns:
+                                continue
+                            if bud.link_ns != O.U64_OFF and spent_link.get(lk, 0) + c > bud.link_ns:
+                                continue
+                            cands.append((Fraction(-ben, c), (seed, a, b, ea, eb), c, Ln))
+        if it == len(swaps):
+            assert not cands
+            break
+        assert cands
+        _, (_, a, b, ea, eb), c, Ln = min(cands, key=lambda t: (t[0], t[1]))
+        assert swaps[it] == (a, b, ea, eb)
+        L = Ln
+        pi[ea], pi[eb] = pi[eb], pi[ea]
+        moved |= {ea, eb}
+        spent += c
+        spent_rank[a] += c
+        spent_rank[b] += c
+        lk = O.link_id(a, b, bud.ranks_per_node)
+        spent_link[lk] = spent_link.get(lk, 0) + c
+    assert pi == pi_out and L == after and sorted(pi_out) == list(range(E))
+
+
 def test_ratio_prefers_cheap_swap_over_larger_benefit():
     # experts 0,1 on rank 0, experts 2,3 on rank 1; per-expert sizes make the
     # largest-benefit pair expensive enough to lose on benefit / cost

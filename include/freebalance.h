@@ -94,6 +94,20 @@ typedef struct {
                              /* only (never to the routing weight); ignored by the softmax gate */
 } fb_router;
 
+/* How the planner walks the candidates ("Budgeted Expert-Swap Planning").  The paper's
+ * Algorithm 1 loops and re-enumerates after every accepted swap; its prose describes one
+ * enumeration and one sorted pass; its last paragraph restricts the candidates to the most
+ * and the least loaded rank "in practice".  The default follows Algorithm 1 on that narrow
+ * frontier; the other two modes are the readings left over, kept for comparison. */
+typedef enum {
+  FB_PLAN_LOOP = 0,    /* Algorithm 1: most -> least loaded rank, re-enumerated per accepted swap      */
+  FB_PLAN_SWEEP = 1,   /* one enumeration on the initial frontier, one sort by benefit / cost, one     */
+                       /* pass: a pair is accepted if both experts are unselected and the budgets hold */
+                       /* (later pairs keep the score of the initial loads, so the maximum can rise)   */
+  FB_PLAN_WIDE = 2     /* Algorithm 1 with frontier_width ranks at each end of the load order; a       */
+                       /* source must carry strictly more than its destination; ties also by ranks     */
+} fb_plan_mode;
+
 /* Planner parameters: Algorithm 1's budget B and threshold tau, the weight gamma of
  * Eq. 8 and the cost model of Eq. 9 in integer units so that every rank (and the CPU
  * oracle) reproduces the same plan bit for bit. */
@@ -110,6 +124,8 @@ typedef struct {
   int32_t  ranks_per_node;   /* <= 0: all ranks in one node                                    */
   uint64_t expert_bytes;     /* S(e) when every expert has the same size                       */
   const uint64_t* expert_bytes_table; /* dev u64 [E] per-expert S(e), or NULL for the uniform size */
+  int32_t  mode;             /* fb_plan_mode; 0 (all-zero tail of the struct) is Algorithm 1's loop */
+  int32_t  frontier_width;   /* FB_PLAN_WIDE: 1..4 ranks from each end (values outside are clamped)  */
 } fb_budget;
 
 /* One accepted swap: expert_src leaves src_rank (the overloaded one) for dst_rank,

@@ -35,7 +35,11 @@ class FbBudget(ctypes.Structure):
                 ("tau_tokens", ctypes.c_uint32), ("gamma_num", ctypes.c_uint32),
                 ("gamma_den", ctypes.c_uint32), ("alpha_ns", ctypes.c_uint64 * 2),
                 ("fs_per_byte", ctypes.c_uint64 * 2), ("ranks_per_node", ctypes.c_int32),
-                ("expert_bytes", ctypes.c_uint64), ("expert_bytes_table", ctypes.c_void_p)]
+                ("expert_bytes", ctypes.c_uint64), ("expert_bytes_table", ctypes.c_void_p),
+                ("mode", ctypes.c_int32), ("frontier_width", ctypes.c_int32)]
+
+
+FB_PLAN_LOOP, FB_PLAN_SWEEP, FB_PLAN_WIDE = 0, 1, 2
 
 
 FB_OK = 0
@@ -155,7 +159,8 @@ def _check(status: int, where: str) -> None:
 
 def make_budget(max_swaps=0, global_ns=_U64_OFF, rank_ns=_U64_OFF, link_ns=_U64_OFF, tau_tokens=0,
                 gamma_num=0, gamma_den=1, alpha_ns=(0, 0), fs_per_byte=(0, 0), ranks_per_node=0,
-                expert_bytes=0, expert_bytes_table: Optional[torch.Tensor] = None) -> FbBudget:
+                expert_bytes=0, expert_bytes_table: Optional[torch.Tensor] = None, mode=FB_PLAN_LOOP,
+                frontier_width=1) -> FbBudget:
     b = FbBudget()
     b.max_swaps, b.global_ns, b.rank_ns, b.link_ns = max_swaps, global_ns, rank_ns, link_ns
     b.tau_tokens, b.gamma_num, b.gamma_den = tau_tokens, gamma_num, gamma_den
@@ -163,6 +168,7 @@ def make_budget(max_swaps=0, global_ns=_U64_OFF, rank_ns=_U64_OFF, link_ns=_U64_
     b.fs_per_byte = (ctypes.c_uint64 * 2)(*fs_per_byte)
     b.ranks_per_node, b.expert_bytes = ranks_per_node, expert_bytes
     b.expert_bytes_table = _ptr(expert_bytes_table)
+    b.mode, b.frontier_width = mode, frontier_width
     b._keepalive = expert_bytes_table
     return b
 

@@ -169,6 +169,9 @@ fb_status fill_plan(const fb_ctx* ctx, const fb_budget* b, const int32_t* pi, in
     if (b->expert_bytes_table == nullptr && pp->uniform_cost_ns[c] == 0) return FB_ERR_INVALID_ARG;
     pp->uniform_link_cap[c] = pp->uniform_cost_ns[c] ? b->link_ns / pp->uniform_cost_ns[c] : 0;
   }
+  if (b->mode != FB_PLAN_LOOP && b->mode != FB_PLAN_SWEEP && b->mode != FB_PLAN_WIDE) return FB_ERR_INVALID_ARG;
+  pp->mode = b->mode;
+  pp->frontier_width = b->frontier_width;
   pp->ranks_per_node = b->ranks_per_node;
   pp->expert_bytes_table = b->expert_bytes_table;
   pp->expert_to_slot = pi;

@@ -25,6 +25,8 @@ struct PlanParams {
   uint64_t uniform_cost_ns[2];          // Eq. 9 evaluated on the host for the uniform expert size
   uint64_t uniform_link_cap[2];         // link_ns / uniform_cost_ns: swaps one link can carry (host)
   int32_t ranks_per_node;
+  int32_t mode;                         // fb_plan_mode
+  int32_t frontier_width;               // FB_PLAN_WIDE: ranks taken from each end of the load order (1..4)
   const uint64_t* expert_bytes_table;   // device [E] or nullptr
   const int32_t* expert_to_slot;        // device [E]
   int32_t* expert_to_slot_out;          // device [E]
@@ -54,8 +56,11 @@ struct PlanParams {
 struct PlanCandidate {
   long long benefit;                    // gamma_den * (Phi(L) - Phi(L')), > 0 when valid
   unsigned long long cost;              // C(s) in ns, >= 1
+  int32_t a, b;                         // source and destination rank
   int32_t ea, eb;                       // ea < 0: no candidate
 };
+
+constexpr int kMaxFrontierWidth = 4;
 
 struct PlanShared {
   uint32_t cnt[FB_MAX_EXPERTS];
@@ -83,13 +88,15 @@ constexpr uint32_t kSlotMoved = 1u << 31;
 static_assert(FB_MAX_COUNT_SUM <= kSlotCountMask && FB_MAX_EXPERTS <= 256, "slot word layout");
 
 // true if x is a better choice than y: larger benefit / cost, compared exactly as
-// cross products in 128 bits; equal ratios -> smaller (ea, eb).
+// cross products in 128 bits; equal ratios -> smaller (a, b, ea, eb).
 __device__ __forceinline__ bool plan_better(const PlanCandidate& x, const PlanCandidate& y) {
   if (x.ea < 0) return false;
   if (y.ea < 0) return true;
   const unsigned __int128 l = static_cast<unsigned __int128>(static_cast<unsigned long long>(x.benefit)) * y.cost;
   const unsigned __int128 r = static_cast<unsigned __int128>(static_cast<unsigned long long>(y.benefit)) * x.cost;
   if (l != r) return l > r;
+  if (x.a != y.a) return x.a < y.a;
+  if (x.b != y.b) return x.b < y.b;
   if (x.ea != y.ea) return x.ea < y.ea;
   return x.eb < y.eb;
 }
@@ -370,7 +377,7 @@ __device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh
   __syncwarp();
   FB_PLAN_STAMP(19);
 
-  if (p.expert_bytes_table == nullptr && m <= 16) {
+  if (p.expert_bytes_table == nullptr && m <= 16 && p.mode == FB_PLAN_LOOP) {
     int l0 = static_cast<int>(L0), l1 = static_cast<int>(L1);
     const int mm = m * m;
     // largest benefit any swap of this call can have (rank loads never exceed the initial maximum)
@@ -400,135 +407,135 @@ __device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh
     if (lane + 32 < R) p.load_after[lane + 32] = static_cast<uint32_t>(l1);
     return;
   }
+  // ---- general loop: per-expert sizes, more than 16 experts per rank, or a planner variant
+  // (the one-pass sweep of the ordering paragraph, a widened frontier).  Plain and slow.
   const long long gnum = p.gamma_den ? p.gamma_num : 0;
   const long long gden = p.gamma_den ? p.gamma_den : 1;
   const int rpn = p.ranks_per_node;
   const bool uniform = p.expert_bytes_table == nullptr;     // one cost per link class
-  // Candidate c (0 <= c < m*m) pairs slot c / m of the heavy rank with slot c % m of the
-  // light one.  A lane's first candidates are fixed for the whole call: divide once.
-  constexpr int kSlotsPerLane = 8;                          // covers m <= 16 without a loop
-  int cand_ia[kSlotsPerLane], cand_ib[kSlotsPerLane];
-#pragma unroll
-  for (int t = 0; t < kSlotsPerLane; ++t) {
-    const int c = lane + 32 * t;
-    cand_ia[t] = c / m;
-    cand_ib[t] = c % m;
-  }
+  const bool sweep = p.mode == FB_PLAN_SWEEP;
+  int W = p.mode == FB_PLAN_WIDE ? p.frontier_width : 1;
+  W = W < 1 ? 1 : (W > kMaxFrontierWidth ? kMaxFrontierWidth : W);
+  if (W > R) W = R;
+  const int mm = m * m;
   unsigned long long global_spent = 0;
   uint32_t n = 0;
+  // the sweep scores every pair once, against the frontier and the loads of the placement as given
+  int top[kMaxFrontierWidth], bot[kMaxFrontierWidth];
+  long long Ltop[kMaxFrontierWidth], Lbot[kMaxFrontierWidth], other_max[kMaxFrontierWidth * kMaxFrontierWidth];
   while (n < p.max_swaps) {
-    // frontier: most and least loaded rank, lowest index on ties.  Loads are below 2^22
-    // (checked above), so (load, rank) packs into 32 bits and one warp reduction finds
-    // each extreme: max of load<<6 | (63 - rank), min of load<<6 | rank.
-    const uint32_t none_hi = 0u, none_lo = 0xffffffffu;
-    const uint32_t h0 = L0 >= 0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(63 - lane)) : none_hi;
-    const uint32_t h1 = L1 >= 0 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(31 - lane)) : none_hi;
-    const uint32_t l0 = L0 >= 0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(lane)) : none_lo;
-    const uint32_t l1 = L1 >= 0 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(lane + 32)) : none_lo;
-    const uint32_t hi_key = __reduce_max_sync(full, h0 > h1 ? h0 : h1);
-    const uint32_t lo_key = __reduce_min_sync(full, l0 < l1 ? l0 : l1);
-    const int a = 63 - static_cast<int>(hi_key & 63u), b = static_cast<int>(lo_key & 63u);
-    const long long La = hi_key >> 6, Lb = lo_key >> 6;
-    if (La - Lb <= static_cast<long long>(p.tau_tokens)) break;
-    uint32_t m2 = 0;                               // largest load among the other ranks
-    if (lane != a && lane != b && L0 > 0) m2 = static_cast<uint32_t>(L0);
-    if (lane + 32 != a && lane + 32 != b && L1 > static_cast<long long>(m2)) m2 = static_cast<uint32_t>(L1);
-    const long long M2 = __reduce_max_sync(full, m2);
+    if (!sweep || n == 0) {
+      // The W most and the W least loaded ranks, lowest index on ties, by repeated extraction.
+      // Loads are below 2^22, so (load, rank) packs into 32 bits: max of load<<6 | (63 - rank),
+      // min of load<<6 | rank.
+      unsigned long long taken_hi = 0, taken_lo = 0;
+#pragma unroll
+      for (int w = 0; w < kMaxFrontierWidth; ++w) {
+        if (w < W) {
+          const bool f0 = L0 >= 0 && !((taken_hi >> lane) & 1ull), f1 = L1 >= 0 && !((taken_hi >> (lane + 32)) & 1ull);
+          const uint32_t h0 = f0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(63 - lane)) : 0u;
+          const uint32_t h1 = f1 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(31 - lane)) : 0u;
+          const uint32_t hi_key = __reduce_max_sync(full, h0 > h1 ? h0 : h1);
+          top[w] = 63 - static_cast<int>(hi_key & 63u);
+          Ltop[w] = hi_key >> 6;
+          taken_hi |= 1ull << top[w];
+          const bool g0 = L0 >= 0 && !((taken_lo >> lane) & 1ull), g1 = L1 >= 0 && !((taken_lo >> (lane + 32)) & 1ull);
+          const uint32_t l0 = g0 ? (static_cast<uint32_t>(L0) << 6 | static_cast<uint32_t>(lane)) : 0xffffffffu;
+          const uint32_t l1 = g1 ? (static_cast<uint32_t>(L1) << 6 | static_cast<uint32_t>(lane + 32)) : 0xffffffffu;
+          const uint32_t lo_key = __reduce_min_sync(full, l0 < l1 ? l0 : l1);
+          bot[w] = static_cast<int>(lo_key & 63u);
+          Lbot[w] = lo_key >> 6;
+          taken_lo |= 1ull << bot[w];
+        }
+      }
+      // largest load among the ranks other than the two of a pair
+#pragma unroll
+      for (int wa = 0; wa < kMaxFrontierWidth; ++wa)
+#pragma unroll
+        for (int wb = 0; wb < kMaxFrontierWidth; ++wb)
+          if (wa < W && wb < W) {
+            const int a = top[wa], b = bot[wb];
+            uint32_t o = 0;
+            if (lane != a && lane != b && L0 > 0) o = static_cast<uint32_t>(L0);
+            if (lane + 32 != a && lane + 32 != b && L1 > static_cast<long long>(o)) o = static_cast<uint32_t>(L1);
+            other_max[wa * kMaxFrontierWidth + wb] = __reduce_max_sync(full, o);
+          }
+    }
+    if (Ltop[0] - Lbot[0] <= static_cast<long long>(p.tau_tokens)) break;
+    const long long M = Ltop[0];                                  // the maximum rank load
+    PlanCandidate best;
+    best.benefit = 0; best.cost = 1; best.a = -1; best.b = -1; best.ea = -1; best.eb = -1;
+#pragma unroll
+    for (int wa = 0; wa < kMaxFrontierWidth; ++wa) {
+#pragma unroll
+      for (int wb = 0; wb < kMaxFrontierWidth; ++wb) {
+        if (wa >= W || wb >= W) continue;
+        const int a = top[wa], b = bot[wb];
+        const long long La = Ltop[wa], Lb = Lbot[wb];
+        if (a == b || La <= Lb) continue;                         // a source carries strictly more than its destination
+        const long long O = other_max[wa * kMaxFrontierWidth + wb];
+        const int cls = (rpn <= 0 || a / rpn == b / rpn) ? 0 : 1;
+        const int lo = a < b ? a : b, hi = a < b ? b : a;
+        const uint32_t lkey = cls == 0 ? (static_cast<uint32_t>(lo) << 8 | static_cast<uint32_t>(hi))
+                                       : (0x10000u | static_cast<uint32_t>(lo / rpn) << 8 | static_cast<uint32_t>(hi / rpn));
+        unsigned long long link_spent = 0;
+        if (p.link_ns != FB_BUDGET_OFF)
+          for (uint32_t i = 0; i < n; ++i)
+            if (sh.link_key[i] == lkey) link_spent += sh.link_cost[i];
+        const unsigned long long rs_a = sh.rank_spent[a], rs_b = sh.rank_spent[b];
+        const unsigned long long rank_spent = rs_a > rs_b ? rs_a : rs_b;
+        const long long D = La - Lb;
+        for (int c = lane; c < mm; c += 32) {
+          const int ea = sh.expert_at[a * m + c / m];
+          const int eb = sh.expert_at[b * m + c % m];
+          if (sh.moved[ea] || sh.moved[eb]) continue;
+          const long long dlt = static_cast<long long>(sh.cnt[ea]) - static_cast<long long>(sh.cnt[eb]);   // tokens moved a -> b
+          long long Mn = La - dlt;                                // Eq. 6
+          if (Lb + dlt > Mn) Mn = Lb + dlt;                       // Eq. 7
+          if (O > Mn) Mn = O;
+          // gamma_den * (Phi(L) - Phi(L')): the mean is unchanged by a swap, so the
+          // variance term reduces to 2 dlt (La - Lb - dlt).
+          const long long benefit = gden * (M - Mn) + 2 * gnum * (dlt * (D - dlt));
+          if (benefit <= 0) continue;
+          PlanCandidate cand;
+          cand.benefit = benefit;
+          cand.a = a; cand.b = b; cand.ea = ea; cand.eb = eb;
+          cand.cost = uniform ? p.uniform_cost_ns[cls] : plan_cost_ns(p, cls, ea, eb);   // Eq. 9
+          if (p.global_ns != FB_BUDGET_OFF && (cand.cost > p.global_ns || global_spent > p.global_ns - cand.cost)) continue;
+          if (p.rank_ns != FB_BUDGET_OFF && (cand.cost > p.rank_ns || rank_spent > p.rank_ns - cand.cost)) continue;
+          if (p.link_ns != FB_BUDGET_OFF && (cand.cost > p.link_ns || link_spent > p.link_ns - cand.cost)) continue;
+          if (plan_better(cand, best)) best = cand;
+        }
+      }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      PlanCandidate o;
+      o.benefit = __shfl_xor_sync(full, best.benefit, off);
+      o.cost = __shfl_xor_sync(full, best.cost, off);
+      o.a = __shfl_xor_sync(full, best.a, off);
+      o.b = __shfl_xor_sync(full, best.b, off);
+      o.ea = __shfl_xor_sync(full, best.ea, off);
+      o.eb = __shfl_xor_sync(full, best.eb, off);
+      if (plan_better(o, best)) best = o;
+    }
+    if (best.ea < 0) break;                                     // Algorithm 1 lines 6-7
+    const int a = best.a, b = best.b;
+    const long long dlt = static_cast<long long>(sh.cnt[best.ea]) - static_cast<long long>(sh.cnt[best.eb]);
     const int cls = (rpn <= 0 || a / rpn == b / rpn) ? 0 : 1;
     const int lo = a < b ? a : b, hi = a < b ? b : a;
     const uint32_t lkey = cls == 0 ? (static_cast<uint32_t>(lo) << 8 | static_cast<uint32_t>(hi))
                                    : (0x10000u | static_cast<uint32_t>(lo / rpn) << 8 | static_cast<uint32_t>(hi / rpn));
-    unsigned long long link_spent = 0;
-    if (p.link_ns != FB_BUDGET_OFF)
-      for (uint32_t i = 0; i < n; ++i)
-        if (sh.link_key[i] == lkey) link_spent += sh.link_cost[i];
-    const unsigned long long rs_a = sh.rank_spent[a], rs_b = sh.rank_spent[b];
-    const unsigned long long rank_spent = rs_a > rs_b ? rs_a : rs_b;
-
-    if (uniform) {
-      // same cost for every candidate of this iteration: one budget test decides for all
-      const unsigned long long c_ns = p.uniform_cost_ns[cls];
-      if (p.global_ns != FB_BUDGET_OFF && (c_ns > p.global_ns || global_spent > p.global_ns - c_ns)) break;
-      if (p.rank_ns != FB_BUDGET_OFF && (c_ns > p.rank_ns || rank_spent > p.rank_ns - c_ns)) break;
-      if (p.link_ns != FB_BUDGET_OFF && (c_ns > p.link_ns || link_spent > p.link_ns - c_ns)) break;
-    }
-    PlanCandidate best;
-    best.benefit = 0; best.cost = 1; best.ea = -1; best.eb = -1;
-    const int D = static_cast<int>(La - Lb);                    // > tau >= 0, below 2^22
-    const int mm = m * m;
-    auto consider = [&](int ia, int ib) {
-      const int ea = sh.expert_at[a * m + ia];
-      const int eb = sh.expert_at[b * m + ib];
-      if (sh.moved[ea] || sh.moved[eb]) return;
-      const int dlt = static_cast<int>(sh.cnt[ea]) - static_cast<int>(sh.cnt[eb]);   // tokens moved a -> b
-      long long Mn = La - dlt;                                  // Eq. 6
-      if (Lb + dlt > Mn) Mn = Lb + dlt;                         // Eq. 7
-      if (M2 > Mn) Mn = M2;
-      // gamma_den * (Phi(L) - Phi(L')): the mean is unchanged by a swap, so the
-      // variance term reduces to 2 dlt (La - Lb - dlt).
-      const long long var2 = static_cast<long long>(dlt) * static_cast<long long>(D - dlt);
-      const long long benefit = gden * (La - Mn) + 2 * gnum * var2;
-      if (benefit <= 0) return;
-      PlanCandidate cand;
-      cand.benefit = benefit;
-      cand.ea = ea; cand.eb = eb;
-      if (uniform) {
-        cand.cost = 1;                                          // equal for all: compare benefits only
-        if (best.ea < 0 || benefit > best.benefit ||
-            (benefit == best.benefit && (ea < best.ea || (ea == best.ea && eb < best.eb)))) best = cand;
-      } else {
-        cand.cost = plan_cost_ns(p, cls, ea, eb);               // Eq. 9
-        if (p.global_ns != FB_BUDGET_OFF && (cand.cost > p.global_ns || global_spent > p.global_ns - cand.cost)) return;
-        if (p.rank_ns != FB_BUDGET_OFF && (cand.cost > p.rank_ns || rank_spent > p.rank_ns - cand.cost)) return;
-        if (p.link_ns != FB_BUDGET_OFF && (cand.cost > p.link_ns || link_spent > p.link_ns - cand.cost)) return;
-        if (plan_better(cand, best)) best = cand;
-      }
-    };
-#pragma unroll
-    for (int t = 0; t < kSlotsPerLane; ++t)
-      if (lane + 32 * t < mm) consider(cand_ia[t], cand_ib[t]);
-    for (int c = lane + 32 * kSlotsPerLane; c < mm; c += 32) consider(c / m, c % m);
-    if (p.expert_bytes_table == nullptr) {
-      // every candidate of this iteration has the same cost: the largest benefit wins,
-      // ties go to the smallest (ea, eb).  Three 32-bit warp reductions.
-      const unsigned long long ben = best.ea >= 0 ? static_cast<unsigned long long>(best.benefit) : 0ull;
-      const uint32_t top_hi = __reduce_max_sync(full, static_cast<uint32_t>(ben >> 32));
-      const uint32_t lo_part = static_cast<uint32_t>(ben >> 32) == top_hi ? static_cast<uint32_t>(ben) : 0u;
-      const uint32_t top_lo = __reduce_max_sync(full, lo_part);
-      const unsigned long long top_ben = static_cast<unsigned long long>(top_hi) << 32 | top_lo;
-      const uint32_t pair = (best.ea >= 0 && ben == top_ben)
-                                ? (static_cast<uint32_t>(best.ea) << 16 | static_cast<uint32_t>(best.eb)) : 0xffffffffu;
-      const uint32_t win = __reduce_min_sync(full, pair);
-      if (top_ben == 0 || win == 0xffffffffu) { best.ea = -1; }
-      else {
-        best.benefit = static_cast<long long>(top_ben);
-        best.cost = p.uniform_cost_ns[cls];
-        best.ea = static_cast<int32_t>(win >> 16);
-        best.eb = static_cast<int32_t>(win & 0xffffu);
-      }
-    } else {
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        PlanCandidate o;
-        o.benefit = __shfl_xor_sync(full, best.benefit, off);
-        o.cost = __shfl_xor_sync(full, best.cost, off);
-        o.ea = __shfl_xor_sync(full, best.ea, off);
-        o.eb = __shfl_xor_sync(full, best.eb, off);
-        if (plan_better(o, best)) best = o;
-      }
-    }
-    if (best.ea < 0) break;                                     // Algorithm 1 lines 6-7
-    const long long dlt = static_cast<long long>(sh.cnt[best.ea]) - static_cast<long long>(sh.cnt[best.eb]);
     __syncwarp();                                               // all lanes are done reading the tables
     if (lane == 0) {
       const int sa = sh.slot_of[best.ea], sb = sh.slot_of[best.eb];
       sh.slot_of[best.ea] = sb; sh.slot_of[best.eb] = sa;
       sh.expert_at[sa] = best.eb; sh.expert_at[sb] = best.ea;
       sh.moved[best.ea] = 1; sh.moved[best.eb] = 1;
-      sh.rank_spent[a] = rs_a + best.cost; sh.rank_spent[b] = rs_b + best.cost;
+      sh.rank_spent[a] += best.cost; sh.rank_spent[b] += best.cost;
       sh.link_key[n] = lkey; sh.link_cost[n] = best.cost;
-      fb_swap s; s.src_rank = a; s.dst_rank = b; s.expert_src = best.ea; s.expert_dst = best.eb;
-      p.swaps[n] = s;
+      fb_swap sw; sw.src_rank = a; sw.dst_rank = b; sw.expert_src = best.ea; sw.expert_dst = best.eb;
+      p.swaps[n] = sw;
     }
     if (lane == a) L0 -= dlt;
     if (lane + 32 == a) L1 -= dlt;

@@ -157,6 +157,69 @@ def test_plan_swaps_alone_on_random_counts(seed):
     assert (got_swaps, out_pi.cpu().tolist(), lb.cpu().tolist(), la.cpu().tolist()) == want
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_planner_variants_random_plans_exact(seed):
+    """The one-pass sweep, the widened frontier, per-expert sizes and ranks of more than 16
+    experts all run the general planner loop: exact agreement with the oracle's variant."""
+    rng = np.random.default_rng(500 + seed)
+    R = int(rng.choice([2, 3, 4, 8, 16, 64]))
+    m = int(rng.choice([1, 2, 4, 8, 32]))
+    E = R * m
+    if E > 256:
+        m = 256 // R
+        E = R * m
+    counts = I.random_counts(E, int(rng.integers(0, 200_000)), seed, zipf_s=float(rng.choice([0.5, 1.0, 1.5])))
+    pi = I.random_placement(E, seed)
+    mode = [B.FB_PLAN_SWEEP, B.FB_PLAN_WIDE, B.FB_PLAN_LOOP][seed % 3]
+    bkw = dict(max_swaps=int(rng.integers(1, E // 2 + 1)) if E >= 2 else 0, gamma_num=int(rng.choice([0, 1, 5])),
+               gamma_den=int(rng.choice([1, 64, 100_000])), tau_tokens=int(rng.choice([0, 0, 50])),
+               alpha_ns=(int(rng.integers(0, 500)), int(rng.integers(0, 5000))),
+               fs_per_byte=(int(rng.integers(0, 3000)), int(rng.integers(0, 20000))),
+               expert_bytes=int(rng.integers(0, 10**7)), ranks_per_node=int(rng.choice([0, 2, 8])),
+               global_ns=[O.U64_OFF, 10**5, 10**6][int(rng.integers(0, 3))],
+               rank_ns=[O.U64_OFF, 10**5][int(rng.integers(0, 2))],
+               link_ns=[O.U64_OFF, 5 * 10**4][int(rng.integers(0, 2))],
+               mode=mode, frontier_width=int(rng.integers(1, 5)))
+    table = None
+    if mode == B.FB_PLAN_LOOP or seed % 4 == 0:                  # the loop mode reaches this path through a size table
+        table = torch.as_tensor(rng.integers(1, 10**6, size=E), dtype=torch.int64)
+    ctx = B.Context(128, 64, E, 1, R)
+    dev = torch.device("cuda")
+    ms = max(1, bkw["max_swaps"])
+    out_pi = torch.zeros(E, dtype=torch.int32, device=dev)
+    swaps = torch.zeros(4 * ms, dtype=torch.int32, device=dev)
+    n = torch.zeros(1, dtype=torch.int32, device=dev)
+    lb = torch.zeros(R, dtype=torch.int32, device=dev)
+    la = torch.zeros(R, dtype=torch.int32, device=dev)
+    gbud = B.make_budget(expert_bytes_table=None if table is None else table.to(dev), **bkw)
+    ctx.fb_plan_swaps(counts.to(torch.int32).to(dev), pi.to(dev), gbud, seed, out_pi, swaps, n, lb, la)
+    assert ctx.fb_device_status() == 0
+    obud = O.Budget(expert_bytes_table=None if table is None else tuple(int(x) for x in table), **bkw)
+    want = O.plan(counts.tolist(), pi.tolist(), R, obud, layer_id=seed)
+    got_swaps = [tuple(r) for r in swaps.cpu().numpy().reshape(-1, 4)[:int(n.item())].tolist()]
+    assert (got_swaps, out_pi.cpu().tolist(), lb.cpu().tolist(), la.cpu().tolist()) == want
+    ctx.close()
+
+
+def test_planner_variant_worked_examples_on_gpu(golden):
+    for name, mode in [("planner_sweep_overshoots.json", B.FB_PLAN_SWEEP), ("planner_wide_frontier.json", B.FB_PLAN_WIDE)]:
+        gd = golden(name)
+        E, R = gd["E"], gd["R"]
+        ctx = B.Context(128, 64, E, 1, R)
+        dev = torch.device("cuda")
+        t = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
+        out_pi, swaps, n, lb, la = t([0] * E), t([0] * 16), t([0]), t([0] * R), t([0] * R)
+        bud = B.make_budget(max_swaps=min(gd["max_swaps"], E // 2), gamma_num=gd["gamma_num"], gamma_den=gd["gamma_den"],
+                            mode=mode, frontier_width=gd.get("frontier_width", 1))
+        ctx.fb_plan_swaps(t(gd["counts"]), t(gd["expert_to_slot"]), bud, 0, out_pi, swaps, n, lb, la)
+        assert ctx.fb_device_status() == 0
+        k = int(n.item())
+        assert swaps.cpu().numpy().reshape(-1, 4)[:k].tolist() == gd["swaps"]
+        assert out_pi.cpu().tolist() == gd["expert_to_slot_out"]
+        assert lb.cpu().tolist() == gd["load_before"] and la.cpu().tolist() == gd["load_after"]
+        ctx.close()
+
+
 def test_planner_worked_examples_on_gpu(golden):
     for name in ["planner_two_swaps_one_tie.json", "planner_tie_then_stop.json"]:
         gd = golden(name)

@@ -147,6 +147,30 @@ fb_status fb_destroy(fb_ctx* ctx);
 /* Eq. 10: B = max(0, t_attn - delta), all in nanoseconds.  Pure host arithmetic. */
 uint64_t fb_budget_ns(uint64_t t_attn_ns, uint64_t delta_ns);
 
+/* ---- attention profiling for the budget of Eq. 10 ("Budgeted Expert-Swap Planning": attention
+ * is profiled once per attention type and the measurement is reused for later layers of that
+ * type; r(l) is the first layer that uses the attention mechanism of layer l) ----
+ * The caller brackets the attention of every layer with fb_attention_begin / fb_attention_end
+ * on the stream the attention kernels run on.  For the first layer of an attention type (its
+ * r(l)) the pair records two CUDA events around the region; for every later layer of a type
+ * that already has a measurement (or one under way) both calls do nothing, so they cost nothing
+ * in steady state.  attn_type is a caller-chosen id in [0, FB_MAX_ATTENTION_TYPES): 0 for a
+ * homogeneous model, one id per mechanism (full, linear, sparse, ...) for a hybrid one.
+ *   fb_layer_budget_ns   B_l = max(0, T_attn[r(l)] - delta_ns) for a layer of that type, in
+ *                        *budget_ns; *profiled_layer (optional) receives r(l).  The first
+ *                        query after a measurement waits for its closing event (blocking, once
+ *                        per type); FB_ERR_INVALID_ARG if the type has never been profiled.
+ *   fb_attention_set_time_ns  installs a measurement taken elsewhere (or replaces one).
+ *   fb_attention_reset   forgets every measurement (the input shape changed).
+ * Host-side bookkeeping plus event records; nothing is launched. */
+#define FB_MAX_ATTENTION_TYPES 8
+fb_status fb_attention_begin(fb_ctx* ctx, int32_t layer_id, int32_t attn_type, fb_stream stream);
+fb_status fb_attention_end(fb_ctx* ctx, int32_t layer_id, int32_t attn_type, fb_stream stream);
+fb_status fb_layer_budget_ns(fb_ctx* ctx, int32_t attn_type, uint64_t delta_ns, uint64_t* budget_ns,
+                             int32_t* profiled_layer);
+fb_status fb_attention_set_time_ns(fb_ctx* ctx, int32_t attn_type, int32_t layer_id, uint64_t t_attn_ns);
+fb_status fb_attention_reset(fb_ctx* ctx);
+
 /* Eq. 9 for a pair of ranks with uniform expert size: C = alpha + 2 S / beta in whole
  * nanoseconds (transfer term rounded up, total at least 1).  Pure host arithmetic;
  * returns 0 if the product overflows 64 bits. */

@@ -56,7 +56,8 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
            "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
            "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
-           "fb_set_stamp_buffer", "fb_clock_probe"]
+           "fb_set_stamp_buffer", "fb_clock_probe", "fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns",
+           "fb_attention_set_time_ns", "fb_attention_reset"]
 
 _lib = None
 
@@ -104,6 +105,14 @@ def lib() -> ctypes.CDLL:
     L.fb_set_pair_limit.restype = ctypes.c_int
     L.fb_max_pairs.argtypes = [vp]
     L.fb_max_pairs.restype = i32
+    L.fb_attention_begin.argtypes = [vp, i32, i32, vp]
+    L.fb_attention_end.argtypes = [vp, i32, i32, vp]
+    L.fb_layer_budget_ns.argtypes = [vp, i32, u64, ctypes.POINTER(u64), ctypes.POINTER(i32)]
+    L.fb_attention_set_time_ns.argtypes = [vp, i32, i32, u64]
+    L.fb_attention_reset.argtypes = [vp]
+    for name in ("fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns", "fb_attention_set_time_ns",
+                 "fb_attention_reset"):
+        getattr(L, name).restype = ctypes.c_int
     L.fb_clock_probe.argtypes = [vp, i32, ctypes.c_uint32, vp]
     L.fb_clock_probe.restype = ctypes.c_int
     L.fb_set_stamp_buffer.argtypes = [vp, vp]
@@ -325,6 +334,25 @@ class Context:
 
     def fb_max_pairs(self) -> int:
         return int(lib().fb_max_pairs(self._h))
+
+    def fb_attention_begin(self, layer_id: int, attn_type: int = 0, stream=None) -> None:
+        _check(lib().fb_attention_begin(self._h, layer_id, attn_type, _stream(stream)), "fb_attention_begin")
+
+    def fb_attention_end(self, layer_id: int, attn_type: int = 0, stream=None) -> None:
+        _check(lib().fb_attention_end(self._h, layer_id, attn_type, _stream(stream)), "fb_attention_end")
+
+    def fb_layer_budget_ns(self, attn_type: int, delta_ns: int):
+        """(B_l of Eq. 10 for a layer of this attention type, the layer r(l) it was measured on)."""
+        budget, layer = ctypes.c_uint64(0), ctypes.c_int32(-1)
+        _check(lib().fb_layer_budget_ns(self._h, attn_type, delta_ns, ctypes.byref(budget), ctypes.byref(layer)),
+               "fb_layer_budget_ns")
+        return int(budget.value), int(layer.value)
+
+    def fb_attention_set_time_ns(self, attn_type: int, layer_id: int, t_attn_ns: int) -> None:
+        _check(lib().fb_attention_set_time_ns(self._h, attn_type, layer_id, t_attn_ns), "fb_attention_set_time_ns")
+
+    def fb_attention_reset(self) -> None:
+        _check(lib().fb_attention_reset(self._h), "fb_attention_reset")
 
     def fb_set_stamp_buffer(self, stamps) -> None:
         """Only libraries built with -DFB_TIMING accept this (see phase_timing.py)."""

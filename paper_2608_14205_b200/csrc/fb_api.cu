@@ -77,6 +77,15 @@ struct fb_ctx {
   uint64_t persistent_launches = 0;
   cudaEvent_t ev_before = nullptr, ev_after = nullptr;   // one-shot: recorded around the next router launch
   unsigned long long* stamps = nullptr;                  // caller's phase-stamp buffer (FB_TIMING builds)
+  // attention profile (Eq. 10): one measurement per attention type, taken on the first layer of the type
+  struct AttnSlot {
+    int32_t layer = -1;                // r(l): the layer whose attention is (being) measured; -1 = none yet
+    bool open = false;                 // begin recorded, end not yet
+    bool pending = false;              // both events recorded, time not read yet
+    bool has_time = false;
+    uint64_t t_ns = 0;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+  } attn[FB_MAX_ATTENTION_TYPES];
 };
 
 namespace {
@@ -533,6 +542,10 @@ fb_status fb_destroy(fb_ctx* ctx) {
     if (p) cudaFree(p);
   if (ctx->mig_stage) cudaFree(ctx->mig_stage);
   if (ctx->mig_host) cudaFreeHost(ctx->mig_host);
+  for (auto& a : ctx->attn) {
+    if (a.e0) cudaEventDestroy(a.e0);
+    if (a.e1) cudaEventDestroy(a.e1);
+  }
   delete ctx;
   return FB_OK;
 }
@@ -915,6 +928,68 @@ fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* even
 }
 
 int32_t fb_max_pairs(const fb_ctx* ctx) { return ctx ? ctx->max_pairs : 0; }
+
+fb_status fb_attention_begin(fb_ctx* ctx, int32_t layer_id, int32_t attn_type, fb_stream stream_) {
+  if (!ctx || attn_type < 0 || attn_type >= FB_MAX_ATTENTION_TYPES || layer_id < 0) return FB_ERR_INVALID_ARG;
+  fb_ctx::AttnSlot& a = ctx->attn[attn_type];
+  if (a.layer >= 0) return FB_OK;                      // this type already has its r(l)
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  if (!a.e0 && cudaEventCreate(&a.e0) != cudaSuccess) return FB_ERR_CUDA;
+  if (!a.e1 && cudaEventCreate(&a.e1) != cudaSuccess) return FB_ERR_CUDA;
+  if (cudaEventRecord(a.e0, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return FB_ERR_CUDA;
+  a.layer = layer_id;
+  a.open = true;
+  return FB_OK;
+}
+
+fb_status fb_attention_end(fb_ctx* ctx, int32_t layer_id, int32_t attn_type, fb_stream stream_) {
+  if (!ctx || attn_type < 0 || attn_type >= FB_MAX_ATTENTION_TYPES || layer_id < 0) return FB_ERR_INVALID_ARG;
+  fb_ctx::AttnSlot& a = ctx->attn[attn_type];
+  if (!a.open || a.layer != layer_id) return FB_OK;    // not the layer being measured
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  if (cudaEventRecord(a.e1, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return FB_ERR_CUDA;
+  a.open = false;
+  a.pending = true;
+  return FB_OK;
+}
+
+fb_status fb_layer_budget_ns(fb_ctx* ctx, int32_t attn_type, uint64_t delta_ns, uint64_t* budget_ns,
+                             int32_t* profiled_layer) {
+  if (!ctx || !budget_ns || attn_type < 0 || attn_type >= FB_MAX_ATTENTION_TYPES) return FB_ERR_INVALID_ARG;
+  fb_ctx::AttnSlot& a = ctx->attn[attn_type];
+  if (a.pending) {
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FB_ERR_CUDA;
+    float ms = 0.0f;
+    if (cudaEventSynchronize(a.e1) != cudaSuccess || cudaEventElapsedTime(&ms, a.e0, a.e1) != cudaSuccess)
+      return FB_ERR_CUDA;
+    a.t_ns = static_cast<uint64_t>(static_cast<double>(ms) * 1e6 + 0.5);
+    a.pending = false;
+    a.has_time = true;
+  }
+  if (!a.has_time) return FB_ERR_INVALID_ARG;          // never profiled (or the region is still open)
+  *budget_ns = fb_budget_ns(a.t_ns, delta_ns);         // Eq. 10
+  if (profiled_layer) *profiled_layer = a.layer;
+  return FB_OK;
+}
+
+fb_status fb_attention_set_time_ns(fb_ctx* ctx, int32_t attn_type, int32_t layer_id, uint64_t t_attn_ns) {
+  if (!ctx || attn_type < 0 || attn_type >= FB_MAX_ATTENTION_TYPES || layer_id < 0) return FB_ERR_INVALID_ARG;
+  fb_ctx::AttnSlot& a = ctx->attn[attn_type];
+  a.layer = layer_id;
+  a.t_ns = t_attn_ns;
+  a.open = a.pending = false;
+  a.has_time = true;
+  return FB_OK;
+}
+
+fb_status fb_attention_reset(fb_ctx* ctx) {
+  if (!ctx) return FB_ERR_INVALID_ARG;
+  for (auto& a : ctx->attn) { a.layer = -1; a.open = a.pending = a.has_time = false; a.t_ns = 0; }
+  return FB_OK;
+}
 
 fb_status fb_clock_probe(uint64_t* samples, int32_t n, uint32_t period_ns, fb_stream stream_) {
   // bounded by construction: at most 65536 samples, at most 100 us apart

@@ -34,26 +34,6 @@ def make_budget_for(wl: I.Workload, T: int, **override) -> B.FbBudget:
     return B.make_budget(**kw)
 
 
-class AttentionProfile:
-    """Budgets of Eq. 10 with one measured attention time per attention type: the first layer
-    of each type is the one whose time is kept and reused for later layers of that type."""
-
-    def __init__(self, delta_ns: int):
-        self.delta_ns = delta_ns
-        self._first: Dict[str, int] = {}          # attention type -> first layer seen
-        self._time_ns: Dict[int, int] = {}        # that layer -> measured attention time
-
-    def needs_profile(self, layer: int, attn_type: str) -> bool:
-        return self._first.setdefault(attn_type, layer) == layer and layer not in self._time_ns
-
-    def record(self, layer: int, attn_type: str, t_attn_ns: int) -> None:
-        if self._first.setdefault(attn_type, layer) == layer:
-            self._time_ns[layer] = int(t_attn_ns)
-
-    def budget_ns(self, attn_type: str) -> int:
-        return B.fb_budget_ns(self._time_ns[self._first[attn_type]], self.delta_ns)
-
-
 class ServingLoop:
     """Per-layer placement state plus the output buffers of one layer step."""
 

@@ -5,7 +5,6 @@ import pytest
 
 from oracle import freebalance_oracle as O
 from paper_2608_14205_b200 import binding as B
-from paper_2608_14205_b200.serving import AttentionProfile
 
 
 def test_fit_matches_the_oracle_on_random_timings():
@@ -27,17 +26,3 @@ def test_fit_rejects_what_the_oracle_rejects():
             B.fb_fit_cost_model(*args)
         with pytest.raises(ValueError):
             O.fit_cost_model(*args)
-
-
-def test_attention_profile_reuses_the_first_layer_of_each_type():
-    types = ["full", "linear", "linear", "full", "sparse", "full"]
-    times = {0: 700_000, 1: 150_000, 4: 90_000}
-    prof = AttentionProfile(delta_ns=100_000)
-    got = []
-    for l, t in enumerate(types):
-        if prof.needs_profile(l, t):
-            prof.record(l, t, times[l])
-        else:
-            prof.record(l, t, 123)                 # later measurements of a known type are ignored
-        got.append(prof.budget_ns(t))
-    assert got == O.budgets_by_attention_type(types, times, 100_000) == [600_000, 50_000, 50_000, 600_000, 0, 600_000]

@@ -229,6 +229,32 @@ fb_status fb_route_dispatch(fb_ctx* ctx, const fb_router* router, const void* x,
                             int32_t* perm, int32_t* inv_perm, uint32_t* rank_load,
                             float* logits, fb_stream stream);
 
+/* ---- the path on several GPUs (token-sharded; "Budgeted Expert-Swap Planning": the ranks
+ * exchange only the compact load statistics and then reproduce the same plan locally) ----
+ * Every GPU holds a contiguous token range, in rank order.  Prediction and planning need one
+ * exchange: fb_predict_load on the local tokens, a sum all-reduce of the E counts among the
+ * ranks (the caller's collective, e.g. NCCL), fb_plan_swaps on the summed counts - every rank
+ * arrives at the same plan.  The dispatch index needs one more: fb_route_dispatch on the local
+ * tokens gives local positions; fb_dispatch_slot_counts turns the local slot_offsets into the E
+ * per-slot counts; the ranks all-gather them (world x E words); fb_dispatch_globalize then
+ * rewrites the local inv_perm into positions in the dispatch order of the WHOLE batch (by slot,
+ * then by token, earlier ranks' tokens first) and writes the whole batch's slot_offsets,
+ * rank_offsets and rank_load, identical on every rank.  An assignment at whole-batch position
+ * pos goes to the rank r with rank_offsets[r] <= pos < rank_offsets[r+1], to row
+ * pos - rank_offsets[r] of its receive buffer.
+ *   slot_counts_all     dev u32 [world][E]  the gathered counts, row r from rank r
+ *   slot_offsets_local  dev u32 [E+1]       as written by fb_route_dispatch on the local tokens
+ *   topk_ids            dev i32 [T_local][k], expert_to_slot dev i32 [E]: as given to / written by that call
+ *   inv_perm            dev i32 [T_local*k] in: local positions; out: whole-batch positions
+ * Errors: FB_ERR_INVALID_ARG (NULL pointer, rank outside [0, world), world outside [1, 4096]),
+ * FB_ERR_UNSUPPORTED_SHAPE (T_local > T_max).  The whole batch must stay below 2^31 assignments. */
+fb_status fb_dispatch_slot_counts(fb_ctx* ctx, const uint32_t* slot_offsets, uint32_t* slot_counts, fb_stream stream);
+fb_status fb_dispatch_globalize(fb_ctx* ctx, int32_t T_local, int32_t world, int32_t rank,
+                                const uint32_t* slot_counts_all, const uint32_t* slot_offsets_local,
+                                const int32_t* topk_ids, const int32_t* expert_to_slot, int32_t* inv_perm,
+                                uint32_t* slot_offsets, uint32_t* rank_offsets, uint32_t* rank_load,
+                                fb_stream stream);
+
 /* One whole layer with device buffers: stages 1, 2 and 4 in one call.  Same results, bit for
  * bit, as fb_predict_and_plan followed by fb_route_dispatch under the new placement, but
  * both router passes (the early one on h_prev, the normal one on H) run in ONE kernel

@@ -37,6 +37,9 @@ itself live in ``tests/test_oracle_*.py``):
                           width 1.
 * ``dispatch_index``     pinned: brute-force ``sorted`` on tiny inputs, a
                           hand-worked example, permutation/offset invariants.
+* ``globalize_dispatch`` pinned: the whole batch's ``dispatch_index`` cut into the shards' token
+                          ranges (positions, offsets and loads must coincide), on random cases
+                          with uneven and empty shards.
 * ``budget_ns``          pinned: Eq. 10 special cases.
 * ``row_cosine_mean``    pinned: closed forms (equal, opposite, orthogonal rows,
                           a 45-degree pair, scale invariance, the zero-row rule).
@@ -541,6 +544,38 @@ def dispatch_index(ids: np.ndarray, expert_to_slot: Sequence[int], R: int):
     rank_load = [rank_offsets[r + 1] - rank_offsets[r] for r in range(R)]
     return (np.array(slot_offsets, dtype=np.int64), np.array(rank_offsets, dtype=np.int64),
             perm, inv_perm, np.array(rank_load, dtype=np.int64))
+
+
+def globalize_dispatch(slot_counts_all: Sequence[Sequence[int]], rank: int, slot_offsets_local: Sequence[int],
+                       inv_perm_local: Sequence[int], R: int):
+    """Token-sharded dispatch: from a shard's own dispatch index to positions in the dispatch
+    order of the whole batch.
+
+    The ranks hold contiguous token ranges in rank order, and the order of the whole batch is by
+    (slot, token), so inside slot p the assignments of earlier ranks come first.  With
+    ``slot_counts_all[r][p]`` the number of assignments rank r sends to slot p (the exchange
+    step: an all-gather of E counts per rank), the position of a local assignment whose local
+    position is ``q`` in slot p is  G[p] + sum_{r' < rank} slot_counts_all[r'][p] + (q -
+    slot_offsets_local[p]),  where G is the exclusive prefix over the slots of the counts summed
+    over all ranks.  Returns (slot_offsets [E+1], rank_offsets [R+1], rank_load [R]) of the whole
+    batch and the shard's inv_perm in whole-batch positions."""
+    world = len(slot_counts_all)
+    E = len(slot_counts_all[0])
+    m = E // R
+    total = [sum(int(slot_counts_all[r][p]) for r in range(world)) for p in range(E)]
+    G = [0] * (E + 1)
+    for p in range(E):
+        G[p + 1] = G[p] + total[p]
+    before = [sum(int(slot_counts_all[r][p]) for r in range(rank)) for p in range(E)]
+    out = []
+    for q in inv_perm_local:
+        q = int(q)
+        p = max(s for s in range(E) if int(slot_offsets_local[s]) <= q and int(slot_offsets_local[s + 1]) > q)
+        out.append(G[p] + before[p] + q - int(slot_offsets_local[p]))
+    rank_offsets = [G[r * m] for r in range(R)] + [G[E]]
+    rank_load = [rank_offsets[r + 1] - rank_offsets[r] for r in range(R)]
+    return (np.array(G, dtype=np.int64), np.array(rank_offsets, dtype=np.int64),
+            np.array(rank_load, dtype=np.int64), np.array(out, dtype=np.int64))
 
 
 # ----------------------------------------------------------------------------

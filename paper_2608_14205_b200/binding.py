@@ -57,7 +57,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
            "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
            "fb_set_stamp_buffer", "fb_clock_probe", "fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns",
-           "fb_attention_set_time_ns", "fb_attention_reset"]
+           "fb_attention_set_time_ns", "fb_attention_reset", "fb_dispatch_slot_counts", "fb_dispatch_globalize"]
 
 _lib = None
 
@@ -105,6 +105,10 @@ def lib() -> ctypes.CDLL:
     L.fb_set_pair_limit.restype = ctypes.c_int
     L.fb_max_pairs.argtypes = [vp]
     L.fb_max_pairs.restype = i32
+    L.fb_dispatch_slot_counts.argtypes = [vp, vp, vp, vp]
+    L.fb_dispatch_slot_counts.restype = ctypes.c_int
+    L.fb_dispatch_globalize.argtypes = [vp, i32, i32, i32] + [vp] * 9
+    L.fb_dispatch_globalize.restype = ctypes.c_int
     L.fb_attention_begin.argtypes = [vp, i32, i32, vp]
     L.fb_attention_end.argtypes = [vp, i32, i32, vp]
     L.fb_layer_budget_ns.argtypes = [vp, i32, u64, ctypes.POINTER(u64), ctypes.POINTER(i32)]
@@ -334,6 +338,17 @@ class Context:
 
     def fb_max_pairs(self) -> int:
         return int(lib().fb_max_pairs(self._h))
+
+    def fb_dispatch_slot_counts(self, slot_offsets, slot_counts, stream=None) -> None:
+        _check(lib().fb_dispatch_slot_counts(self._h, _ptr(slot_offsets), _ptr(slot_counts), _stream(stream)),
+               "fb_dispatch_slot_counts")
+
+    def fb_dispatch_globalize(self, T_local, world, rank, slot_counts_all, slot_offsets_local, topk_ids,
+                              expert_to_slot, inv_perm, slot_offsets, rank_offsets, rank_load, stream=None) -> None:
+        _check(lib().fb_dispatch_globalize(self._h, T_local, world, rank, _ptr(slot_counts_all),
+                                           _ptr(slot_offsets_local), _ptr(topk_ids), _ptr(expert_to_slot),
+                                           _ptr(inv_perm), _ptr(slot_offsets), _ptr(rank_offsets), _ptr(rank_load),
+                                           _stream(stream)), "fb_dispatch_globalize")
 
     def fb_attention_begin(self, layer_id: int, attn_type: int = 0, stream=None) -> None:
         _check(lib().fb_attention_begin(self._h, layer_id, attn_type, _stream(stream)), "fb_attention_begin")

@@ -929,6 +929,43 @@ fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* even
 
 int32_t fb_max_pairs(const fb_ctx* ctx) { return ctx ? ctx->max_pairs : 0; }
 
+fb_status fb_dispatch_slot_counts(fb_ctx* ctx, const uint32_t* slot_offsets, uint32_t* slot_counts, fb_stream stream_) {
+  if (!ctx || !slot_offsets || !slot_counts) return FB_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  fb::fb_slot_counts_kernel<<<1, FB_MAX_EXPERTS, 0, static_cast<cudaStream_t>(stream_)>>>(slot_offsets, ctx->cfg.E,
+                                                                                          slot_counts);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status fb_dispatch_globalize(fb_ctx* ctx, int32_t T_local, int32_t world, int32_t rank,
+                                const uint32_t* slot_counts_all, const uint32_t* slot_offsets_local,
+                                const int32_t* topk_ids, const int32_t* expert_to_slot, int32_t* inv_perm,
+                                uint32_t* slot_offsets, uint32_t* rank_offsets, uint32_t* rank_load,
+                                fb_stream stream_) {
+  if (!ctx || T_local < 0 || world < 1 || world > 4096 || rank < 0 || rank >= world || !slot_counts_all ||
+      !slot_offsets_local || !expert_to_slot || !slot_offsets || !rank_offsets || !rank_load)
+    return FB_ERR_INVALID_ARG;
+  if (T_local > ctx->cfg.T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  if (T_local > 0 && (!topk_ids || !inv_perm)) return FB_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  fb::GlobalizeParams gp;
+  gp.T = T_local; gp.k = ctx->cfg.k; gp.E = ctx->cfg.E; gp.R = ctx->cfg.R; gp.world = world; gp.rank = rank;
+  gp.counts_all = slot_counts_all; gp.local_offsets = slot_offsets_local; gp.topk_ids = topk_ids;
+  gp.expert_to_slot = expert_to_slot; gp.inv_perm = inv_perm;
+  gp.slot_offsets = slot_offsets; gp.rank_offsets = rank_offsets; gp.rank_load = rank_load;
+  const long long n = static_cast<long long>(T_local) * ctx->cfg.k;
+  long long blocks = (n + fb::kGlobalizeThreads - 1) / fb::kGlobalizeThreads;
+  if (blocks < 1) blocks = 1;
+  if (blocks > 2 * ctx->dispatch_blocks_max) blocks = 2 * ctx->dispatch_blocks_max;
+  fb::fb_dispatch_globalize_kernel<<<static_cast<unsigned>(blocks), fb::kGlobalizeThreads, 0,
+                                     static_cast<cudaStream_t>(stream_)>>>(gp);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
 fb_status fb_attention_begin(fb_ctx* ctx, int32_t layer_id, int32_t attn_type, fb_stream stream_) {
   if (!ctx || attn_type < 0 || attn_type >= FB_MAX_ATTENTION_TYPES || layer_id < 0) return FB_ERR_INVALID_ARG;
   fb_ctx::AttnSlot& a = ctx->attn[attn_type];

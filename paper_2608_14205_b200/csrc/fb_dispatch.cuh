@@ -211,4 +211,74 @@ fb_tile_sums_kernel(const uint32_t* __restrict__ tile_counts, uint32_t* __restri
   super_counts[static_cast<size_t>(sb) * E + e] = s;
 }
 
+// ---- token-sharded dispatch (several GPUs, each with a contiguous token range in rank order)
+// A shard's dispatch index is local.  The order of the whole batch is by (slot, token), so in
+// slot p the assignments of earlier ranks come first: the whole-batch position of a local
+// assignment at local position q in slot p is
+//     G[p] + sum_{r' < rank} counts[r'][p] + (q - local_offsets[p]),
+// G = exclusive prefix over slots of the counts summed over all ranks.  counts[r][p] is what the
+// ranks exchange (an all-gather of E words per rank).
+
+// counts[p] = number of local assignments in slot p
+__global__ void fb_slot_counts_kernel(const uint32_t* __restrict__ slot_offsets, int E, uint32_t* __restrict__ counts) {
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  if (p < E) counts[p] = slot_offsets[p + 1] - slot_offsets[p];
+}
+
+constexpr int kGlobalizeThreads = 256;   // >= FB_MAX_EXPERTS: one thread per slot for the shifts
+
+struct GlobalizeParams {
+  int32_t T, k, E, R, world, rank;
+  const uint32_t* counts_all;        // [world][E]
+  const uint32_t* local_offsets;     // [E+1]
+  const int32_t* topk_ids;           // [T][k] (local)
+  const int32_t* expert_to_slot;     // [E]
+  int32_t* inv_perm;                 // [T*k] in: local positions, out: whole-batch positions
+  uint32_t* slot_offsets;            // [E+1] out (whole batch)
+  uint32_t* rank_offsets;            // [R+1] out
+  uint32_t* rank_load;               // [R]   out
+};
+
+__global__ void __launch_bounds__(kGlobalizeThreads)
+fb_dispatch_globalize_kernel(const __grid_constant__ GlobalizeParams p) {
+  __shared__ uint32_t total[FB_MAX_EXPERTS];
+  __shared__ uint32_t shift[FB_MAX_EXPERTS];
+  __shared__ uint32_t G[FB_MAX_EXPERTS + 1];
+  __shared__ int32_t slot_of[FB_MAX_EXPERTS];
+  const int t = threadIdx.x;
+  uint32_t before = 0;
+  if (t < p.E) {
+    uint32_t sum = 0;
+    for (int r = 0; r < p.world; ++r) {
+      const uint32_t c = p.counts_all[static_cast<size_t>(r) * p.E + t];
+      if (r < p.rank) before += c;
+      sum += c;
+    }
+    total[t] = sum;
+    slot_of[t] = p.expert_to_slot[t];
+  }
+  __syncthreads();
+  if (t == 0) {                                 // at most 256 slots: a serial prefix is cheapest here
+    uint32_t run = 0;
+    for (int s = 0; s < p.E; ++s) { G[s] = run; run += total[s]; }
+    G[p.E] = run;
+  }
+  __syncthreads();
+  if (t < p.E) shift[t] = G[t] + before - p.local_offsets[t];
+  if (blockIdx.x == 0) {
+    const int m = p.E / p.R;
+    for (int s = t; s <= p.E; s += kGlobalizeThreads) p.slot_offsets[s] = G[s];
+    for (int r = t; r <= p.R; r += kGlobalizeThreads) p.rank_offsets[r] = G[r == p.R ? p.E : r * m];
+    for (int r = t; r < p.R; r += kGlobalizeThreads) p.rank_load[r] = G[(r + 1) * m] - G[r * m];
+  }
+  __syncthreads();
+  const long long n = static_cast<long long>(p.T) * p.k;
+  for (long long q = static_cast<long long>(blockIdx.x) * kGlobalizeThreads + t; q < n;
+       q += static_cast<long long>(gridDim.x) * kGlobalizeThreads) {
+    const int e = p.topk_ids[q];
+    const int s = (e >= 0 && e < p.E) ? slot_of[e] : -1;
+    if (s >= 0 && s < p.E) p.inv_perm[q] = static_cast<int32_t>(static_cast<uint32_t>(p.inv_perm[q]) + shift[s]);
+  }
+}
+
 }  // namespace fb

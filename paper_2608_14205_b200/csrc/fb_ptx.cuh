@@ -217,13 +217,14 @@ __device__ __forceinline__ void umma_commit_1cta(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
-// Pair version: signal the barrier at this offset in the CTAs selected by cta_mask.
-// (A commit multicast is a barrier arrival, not a data load.)
-__device__ __forceinline__ void umma_commit_2cta(uint32_t bar, uint16_t cta_mask) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-      "h"(cta_mask)
-      : "memory");
+// Pair version: make the barrier at this offset complete in BOTH blocks of the pair once all
+// MMAs issued so far by this thread are done.  Two plain commits - one to this block's
+// barrier, one to the partner's (its shared::cluster address) - rather than one commit with a
+// cluster-wide destination mask.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint32_t my_cta_rank) {
+  const uint32_t peer = map_to_cta(bar, my_cta_rank ^ 1u);
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer) : "memory");
 }
 
 // 32 lanes x 32 columns of 32-bit accumulators: thread t of the warp receives row

@@ -496,12 +496,12 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
         // frees the stage (in both blocks of a pair) when these MMAs retire
         if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.empty_bar[s]));
-        else umma_commit_2cta(smem_u32(&sh.empty_bar[s]), 0x3);
+        else umma_commit_pair(smem_u32(&sh.empty_bar[s]), cta_rank);
       }
       if (warp == 1) FB_STAMP(17, 32);
       // this issuer's accumulator is complete
       if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.accum_bar));
-      else umma_commit_2cta(smem_u32(&sh.accum_bar), 0x3);
+      else umma_commit_pair(smem_u32(&sh.accum_bar), cta_rank);
     }
     if (warp == 1) {
     // One thread polls for the finished accumulator on behalf of the 16 epilogue warps,

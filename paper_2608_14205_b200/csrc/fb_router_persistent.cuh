@@ -187,11 +187,11 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
 #pragma unroll
             for (int kk = 0; kk < kBlockK / kUmmaK; ++kk)
               umma_bf16<2>(acc, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb != first_kb || kk != 0) ? 1u : 0u);
-            umma_commit_2cta(smem_u32(&sh.empty_bar[s]), 0x3);   // frees the stage in both blocks
+            umma_commit_pair(smem_u32(&sh.empty_bar[s]), cta_rank);   // frees the stage in both blocks
           }
           ring_advance(s, phase, p.stages);
         }
-        if (ok) umma_commit_2cta(smem_u32(&sh.accum_bar[set]), 0x3);   // this issuer's accumulator is complete
+        if (ok) umma_commit_pair(smem_u32(&sh.accum_bar[set]), cta_rank);   // this issuer's accumulator is complete
       }
     }
   } else {

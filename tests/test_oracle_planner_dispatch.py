@@ -420,6 +420,28 @@ def test_dispatch_matches_lexsort_and_invariants(seed):
     assert rl.tolist() == O.rank_loads(counts, pi, R)
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_sharded_dispatch_equals_the_whole_batch_cut_into_shards(seed):
+    rng = random.Random(70 + seed)
+    R = rng.choice([2, 4])
+    E = R * rng.choice([1, 2, 4])
+    k = rng.choice([1, 2, min(3, E)])
+    world = rng.choice([1, 2, 3, 5])
+    T = rng.choice([0, 1, 7, 40])
+    ids = np.array([rng.sample(range(E), k) for _ in range(T)], dtype=np.int64).reshape(T, k)
+    pi = list(range(E))
+    rng.shuffle(pi)
+    so, ro, perm, inv, rl = O.dispatch_index(ids, pi, R)
+    cuts = sorted(rng.randrange(0, T + 1) for _ in range(world - 1))
+    bounds = [0] + cuts + [T]                                     # uneven, possibly empty shards
+    local = [O.dispatch_index(ids[bounds[r]:bounds[r + 1]], pi, R) for r in range(world)]
+    counts_all = [np.diff(loc[0]).tolist() for loc in local]
+    for r in range(world):
+        g_so, g_ro, g_rl, g_inv = O.globalize_dispatch(counts_all, r, local[r][0], local[r][3], R)
+        assert g_so.tolist() == so.tolist() and g_ro.tolist() == ro.tolist() and g_rl.tolist() == rl.tolist()
+        assert g_inv.tolist() == inv[bounds[r] * k:bounds[r + 1] * k].tolist()
+
+
 def test_dispatch_empty():
     so, ro, perm, inv, rl = O.dispatch_index(np.zeros((0, 2), dtype=np.int32), [0, 1, 2, 3], 2)
     assert so.tolist() == [0] * 5 and ro.tolist() == [0] * 3 and perm.size == 0 and rl.tolist() == [0, 0]

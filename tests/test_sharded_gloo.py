@@ -1,6 +1,7 @@
-"""Token-sharded prediction + planning: the rank bookkeeping and the one exchange step, run as
-gloo processes on CPU.  The library's two calls are replaced by the oracle's functions (test
-infrastructure) so that the sharding logic itself can run without a GPU."""
+"""The token-sharded layer: the rank bookkeeping and the two exchange steps (count all-reduce,
+slot-count all-gather), run as gloo processes on CPU.  The library's calls are replaced by the
+oracle's functions (test infrastructure) so that the sharding logic itself can run without a
+GPU; the same module drives the CUDA library in tests/test_gpu_sharded.py."""
 import os
 import socket
 import sys
@@ -32,6 +33,35 @@ class OracleContext:
         ids, _ = self.O.select_topk(z, self.gate, None)
         counts.copy_(torch.from_numpy(self.O.expert_histogram(ids, self.gate.E).astype(np.int32)))
 
+    def fb_route_dispatch(self, router, x, T, expert_to_slot, ids_out, w_out, so, ro, perm, inv, rl, logits=None,
+                          stream=None):
+        bits = x.contiguous().view(torch.int16).numpy().view(np.uint16)[:T]
+        z = self.O.router_logits(bits, self.W_bits, None)
+        ids, w = self.O.select_topk(z, self.gate, None)
+        s, r, p, i, l = self.O.dispatch_index(ids, expert_to_slot.tolist(), self.R)
+        k = self.gate.k
+        ids_out[:T * k] = torch.from_numpy(ids.reshape(-1).astype(np.int32))
+        w_out[:T * k] = torch.from_numpy(w.reshape(-1).astype(np.float32))
+        so.copy_(torch.from_numpy(s.astype(np.int32)))
+        ro.copy_(torch.from_numpy(r.astype(np.int32)))
+        perm[:T * k] = torch.from_numpy(p.astype(np.int32))
+        inv[:T * k] = torch.from_numpy(i.astype(np.int32))
+        rl.copy_(torch.from_numpy(l.astype(np.int32)))
+
+    def fb_dispatch_slot_counts(self, slot_offsets, slot_counts, stream=None):
+        E = self.gate.E
+        slot_counts.view(-1)[:E] = slot_offsets[1:E + 1] - slot_offsets[:E]
+
+    def fb_dispatch_globalize(self, T, world, rank, counts_all, local_offsets, ids, expert_to_slot, inv, so, ro, rl,
+                              stream=None):
+        k, E = self.gate.k, self.gate.E
+        g_so, g_ro, g_rl, g_inv = self.O.globalize_dispatch(counts_all.view(world, E).tolist(), rank,
+                                                            local_offsets.tolist(), inv[:T * k].tolist(), self.R)
+        so.copy_(torch.from_numpy(g_so.astype(np.int32)))
+        ro.copy_(torch.from_numpy(g_ro.astype(np.int32)))
+        rl.copy_(torch.from_numpy(g_rl.astype(np.int32)))
+        inv[:T * k] = torch.from_numpy(g_inv.astype(np.int32))
+
     def fb_plan_swaps(self, counts, expert_to_slot, budget, layer_id, pi_out, swaps, n_swaps, lb, la, stream=None):
         sw, pi_new, before, after = self.O.plan_swaps(counts.tolist(), expert_to_slot.tolist(), self.R, self.bud, layer_id)
         pi_out.copy_(torch.tensor(pi_new, dtype=torch.int32))
@@ -56,10 +86,15 @@ def _worker(rank, world, port, T, out):
     ctx = OracleContext(O, _gate(wl), bits(li.W), wl.R, _budget(wl, T))
     sp = ShardedPredictor(ctx)
     i32 = lambda n: torch.zeros(n, dtype=torch.int32)
-    counts, pi_out, swaps, n_swaps, lb, la = i32(wl.E), i32(wl.E), i32(4 * 8), i32(1), i32(wl.R), i32(wl.R)
-    sp.predict_and_plan(None, li.h_prev[lo:hi], hi - lo, li.expert_to_slot, None, 0, counts, pi_out, swaps, n_swaps, lb, la)
+    Tl, k = hi - lo, wl.k
+    o = dict(counts=i32(wl.E), pi_out=i32(wl.E), swaps=i32(4 * 8), n_swaps=i32(1), load_before=i32(wl.R),
+             load_after=i32(wl.R), ids=i32(max(1, Tl * k)), w=torch.zeros(max(1, Tl * k)), slot_offsets=i32(wl.E + 1),
+             rank_offsets=i32(wl.R + 1), perm=i32(max(1, Tl * k)), inv_perm=i32(max(1, Tl * k)), rank_load=i32(wl.R))
+    sp.layer_step(None, li.h_prev[lo:hi], li.H[lo:hi], Tl, li.expert_to_slot, None, 0, o, i32(world * wl.E))
     dist.barrier()
-    out.put((rank, lo, hi, counts.tolist(), pi_out.tolist(), swaps[:4 * int(n_swaps)].tolist(), la.tolist()))
+    out.put((rank, lo, hi, o["counts"].tolist(), o["pi_out"].tolist(), o["swaps"][:4 * int(o["n_swaps"])].tolist(),
+             o["load_after"].tolist(), o["inv_perm"][:Tl * k].tolist(), o["slot_offsets"].tolist(),
+             o["rank_offsets"].tolist(), o["rank_load"].tolist(), o["ids"][:Tl * k].tolist()))
     dist.destroy_process_group()
 
 
@@ -83,11 +118,17 @@ def test_all_ranks_reach_the_plan_of_the_whole_batch(world, T):
     li = I.make_layer(wl, 0, 0, T=T)
     ref = O.layer_step(bits(li.h_prev), bits(li.H), bits(li.W), _gate(wl), wl.R, li.expert_to_slot.tolist(), _budget(wl, T))
     covered = []
-    for rank, lo, hi, counts, pi_out, swaps, la in got:
+    k = wl.k
+    d_so, d_ro, _, d_inv, d_rl = ref["dispatch"]
+    for rank, lo, hi, counts, pi_out, swaps, la, inv, so, ro, rl, ids in got:
         covered += list(range(lo, hi))
         assert counts == ref["counts"].tolist(), "every rank holds the global histogram after the exchange"
         assert pi_out == ref["pi_new"] and la == ref["load_after"]
         assert [tuple(swaps[i:i + 4]) for i in range(0, len(swaps), 4)] == ref["swaps"]
+        # the dispatch index of the whole batch, cut to this rank's tokens
+        assert ids == ref["ids"][lo:hi].reshape(-1).tolist()
+        assert inv == d_inv[lo * k:hi * k].tolist(), "whole-batch positions of the shard's assignments"
+        assert so == d_so.tolist() and ro == d_ro.tolist() and rl == d_rl.tolist()
     assert covered == list(range(T)), "the shards tile the batch"
 
 

@@ -211,6 +211,83 @@ def run_reference(args, wl, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_sharded(args, wl, B, dist, dev, rank, local_rank, world, sampler):
+    """Strong-scaling leg: one batch of wl.T tokens split over the ranks.  Per step and rank: early
+    pass on the local tokens, all-reduce of the E counts, planner, normal pass + local dispatch
+    index, all-gather of the E slot counts, whole-batch positions (sharded.ShardedPredictor)."""
+    from paper_2608_14205_b200.sharded import ShardedPredictor, shard_bounds
+    T, E, R, k, d = wl.T, wl.E, wl.R, wl.k, wl.d
+    lo, hi = shard_bounds(T, world, rank)
+    Tl = hi - lo
+    bkw = budget_kwargs(wl, T)                                  # gamma from the whole batch, same on every rank
+    budget = B.make_budget(**bkw)
+    ctx = B.Context(max(Tl, 1), d, E, k, R, wl.gate, wl.n_group, wl.topk_group, wl.renorm, wl.route_scale,
+                    device=local_rank)
+    ring = max(1, args.ring)
+    layers = []
+    for l in range(ring):
+        li = I.make_layer(wl, layer=l, seed=0)                  # the same batch on every rank; each keeps its shard
+        sb = li.select_bias.to(dev) if li.select_bias is not None else None
+        W = li.W.to(dev)
+        layers.append(dict(W=W, sb=sb, router=B.make_router(W, None, sb), h_prev=li.h_prev[lo:hi].contiguous().to(dev),
+                           H=li.H[lo:hi].contiguous().to(dev), pi=li.expert_to_slot.to(dev)))
+    i32 = lambda n: torch.zeros(max(1, n), dtype=torch.int32, device=dev)
+    out = dict(counts=i32(E), pi_out=i32(E), swaps=i32(4 * max(1, bkw["max_swaps"])), n_swaps=i32(1),
+               load_before=i32(R), load_after=i32(R), ids=i32(Tl * k), w=torch.zeros(max(1, Tl * k), device=dev),
+               slot_offsets=i32(E + 1), rank_offsets=i32(R + 1), perm=i32(Tl * k), inv_perm=i32(Tl * k),
+               rank_load=i32(R))
+    counts_all = i32(world * E)
+    sp = ShardedPredictor(ctx)
+
+    def step(L):
+        sp.layer_step(L["router"], L["h_prev"], L["H"], Tl, L["pi"], budget, 0, out, counts_all)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for i in range(args.warmup):
+        step(layers[i % ring])
+    barrier()
+    K = args.steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.fb_launch_count()
+    sampler.start()
+    sampler.window[0] = time.perf_counter()
+    e0.record()
+    for i in range(K):
+        step(layers[i % ring])
+    e1.record()
+    barrier()
+    sampler.window[1] = time.perf_counter()
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    launches = ctx.fb_launch_count() - launches0
+    status = ctx.fb_device_status()
+    if rank == 0:
+        mom = lambda L: (max(L) * len(L) / sum(L)) if sum(L) else 1.0
+        line = {"metric": METRIC, "value": T * K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+                "warmup": args.warmup, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "strong",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": wl.name, "T": T, "T_per_rank": Tl, "d": d, "E": E, "k": k, "R": R,
+                           "api": "sharded.ShardedPredictor.layer_step (fb_predict_load, all-reduce, fb_plan_swaps, "
+                                  "fb_route_dispatch, all-gather, fb_dispatch_globalize)",
+                           "parallelism": f"token shards x{world}", "layers_in_ring": ring,
+                           "l2": "inputs larger than L2" if Tl * d * 2 > L2_BYTES else
+                                 "ring of layers; inputs may be L2-resident"},
+                "clocks": clocks, "e2e": None, "gpu_launches": int(launches), "device_status": status,
+                "collectives_per_step": 0 if world == 1 else 2,
+                "load_balance": {"predicted_max_over_mean": [mom(out["load_before"].tolist()),
+                                                             mom(out["load_after"].tolist())],
+                                 "realized_max_over_mean_after": mom(out["rank_load"].tolist()),
+                                 "n_swaps": int(out["n_swaps"].item())}}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -221,6 +298,9 @@ def main():
     ap.add_argument("--ring", type=int, default=2, help="distinct layers cycled through")
     ap.add_argument("--api", default="layer", choices=["layer", "separate"],
                     help="layer: fb_layer_step (default); separate: fb_predict_and_plan + fb_route_dispatch")
+    ap.add_argument("--sharded", action="store_true",
+                    help="strong scaling: the workload's T tokens are split over the ranks (contiguous ranges); "
+                         "two small collectives per step (count all-reduce, slot-count all-gather)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     ap.add_argument("--no-probe", action="store_true",
@@ -250,6 +330,9 @@ def main():
 
     # the clock sampler's process starts now (it needs a second to load NVML) and waits for start()
     sampler = ClockSampler(physical_gpu_index(local_rank))
+    T_global = wl.T
+    if args.sharded:
+        return run_sharded(args, wl, B, dist, dev, rank, local_rank, world, sampler)
     T, E, R, k, d = wl.T, wl.E, wl.R, wl.k, wl.d
     bkw = budget_kwargs(wl, T)
     budget = B.make_budget(**bkw)

@@ -211,6 +211,116 @@ def run_reference(args, wl, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_overlap(wl, B, dev, window_us, reps=10, pair_limits=(8, 16, 24, 32, 48), T=None, expert_bytes=None,
+                n_sm=None):
+    """The method's two-stream schedule on one GPU ("Overlap Analysis"): the target layer's
+    attention on one stream, and on a side stream the work it is meant to hide - early router
+    pass + planner (fb_predict_and_plan), then the weight exchange of the accepted swaps
+    (fb_apply_swaps, or the host-issued copies of fb_apply_swaps_staged).
+
+    Attention is a compute-bound stand-in (fb_standin_attention) on n_sm - 2 p SMs; the router
+    kernel is confined to the other p SM pairs (fb_set_pair_limit).  The window B of Eq. 10 comes
+    from the library's own attention profile (fb_attention_begin / _end around the stand-in,
+    fb_layer_budget_ns with a 10 % margin) and is what the planner's time budgets are set to.
+    For every p: attention alone, auxiliary work alone, both together, exposed = together -
+    attention alone, and whether the auxiliary work fitted into the window."""
+    T = T or wl.T
+    E, R, k = wl.E, wl.R, wl.k
+    n_sm = n_sm or torch.cuda.get_device_properties(dev).multi_processor_count
+    S = ((expert_bytes if expert_bytes is not None else wl.expert_bytes) or 16 * 2**20) // 16 * 16
+    li = I.make_layer(wl, 0, 0, T=T)
+    ctx = B.Context(T, wl.d, E, k, R, wl.gate, wl.n_group, wl.topk_group, wl.renorm, wl.route_scale,
+                    device=dev.index or 0)
+    sb = li.select_bias.to(dev) if li.select_bias is not None else None
+    W = li.W.to(dev)
+    router = B.make_router(W, None, sb)
+    h_prev, pi = li.h_prev.to(dev), li.expert_to_slot.to(dev)
+    i32 = lambda n: torch.zeros(max(1, n), dtype=torch.int32, device=dev)
+    cap = max(1, min(wl.max_swaps, E // 2))
+    counts, pi_out, swaps, n_swaps, lb, la = i32(E), i32(E), i32(4 * cap), i32(1), i32(R), i32(R)
+    weights = torch.empty(E * S, dtype=torch.uint8, device=dev)          # content is irrelevant for timing
+    sink = torch.zeros(1024 * 1024, device=dev)
+    side = torch.cuda.Stream(device=dev)
+    main = torch.cuda.current_stream(dev)
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize(dev)
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize(dev)
+            ts.append(a.elapsed_time(b) * 1e3)
+        return statistics.median(ts)
+
+    # stand-in length: iterations per microsecond from two probes
+    t1 = timed(lambda: B.fb_standin_attention(sink, n_sm, 2000))
+    t2 = timed(lambda: B.fb_standin_attention(sink, n_sm, 12000))
+    iters = max(1, int(2000 + (window_us - t1) * 10000 / max(t2 - t1, 1e-3)))
+    rows = []
+    for p_lim in pair_limits:
+        if 2 * p_lim >= n_sm:
+            continue
+        blocks = n_sm - 2 * p_lim
+        ctx.fb_set_pair_limit(p_lim)
+        attention = lambda: B.fb_standin_attention(sink, blocks, iters)
+        # the window of Eq. 10 from the library's attention profile, 10 % margin
+        ctx.fb_attention_reset()
+        attention()
+        ctx.fb_attention_begin(0, 0)
+        attention()
+        ctx.fb_attention_end(0, 0)
+        window_ns, _ = ctx.fb_layer_budget_ns(0, 0)
+        budget_ns, _ = ctx.fb_layer_budget_ns(0, window_ns // 10)
+        bkw = budget_kwargs(wl, T)
+        bkw.update(max_swaps=cap)
+        if wl.global_ns != 2**64 - 1:                         # workloads with a time budget take the measured one
+            bkw.update(global_ns=budget_ns, rank_ns=budget_ns, link_ns=budget_ns)
+        budget = B.make_budget(**bkw)
+
+        def predict_plan(stream=None):
+            ctx.fb_predict_and_plan(router, h_prev, T, pi, budget, 0, counts, pi_out, swaps, n_swaps, lb, la,
+                                    stream=stream)
+
+        def aux_kernel(stream=None):
+            predict_plan(stream)
+            B.fb_apply_swaps(weights, S, E, pi, swaps, n_swaps, cap, stream=stream)
+
+        def aux_copies(stream=None):
+            predict_plan(stream)
+            ctx.fb_apply_swaps_staged(weights, S, pi, swaps, n_swaps, cap, 0, plan_stream=stream, copy_stream=stream)
+
+        def beside(work):
+            def run():
+                side.wait_stream(main)
+                attention()                                   # main stream
+                work(side)                                    # side stream, started at the same time
+                main.wait_stream(side)
+            return run
+
+        row = dict(router_pairs=p_lim, attention_sms=blocks, window_us=window_ns / 1e3, budget_us=budget_ns / 1e3,
+                   attention_us=timed(attention), predict_plan_us=timed(predict_plan))
+        for name, work in (("exchange_kernel", aux_kernel), ("exchange_copies", aux_copies)):
+            alone, both = timed(work), timed(beside(work))
+            row[name] = dict(auxiliary_alone_us=alone, together_us=both,
+                             exposed_us=max(0.0, both - row["attention_us"]),
+                             hidden_fraction=1.0 - max(0.0, both - row["attention_us"]) / alone if alone > 0 else None,
+                             fits_window=both <= row["attention_us"] * 1.05)
+        row["swaps"] = int(n_swaps.item())
+        row["exchange_bytes"] = 4 * S * row["swaps"]
+        rows.append(row)
+    ctx.fb_set_pair_limit(0)
+    status = ctx.fb_device_status()
+    ctx.close()
+    return {"experiment": "two-stream overlap on one GPU", "workload": wl.name, "T": T, "expert_bytes": S,
+            "stand_in": f"fb_standin_attention, {iters} iterations, one block per SM", "sms": n_sm,
+            "device_status": status, "rows": rows}
+
+
 def run_sharded(args, wl, B, dist, dev, rank, local_rank, world, sampler):
     """Strong-scaling leg: one batch of wl.T tokens split over the ranks.  Per step and rank: early
     pass on the local tokens, all-reduce of the E counts, planner, normal pass + local dispatch
@@ -301,6 +411,10 @@ def main():
     ap.add_argument("--sharded", action="store_true",
                     help="strong scaling: the workload's T tokens are split over the ranks (contiguous ranges); "
                          "two small collectives per step (count all-reduce, slot-count all-gather)")
+    ap.add_argument("--overlap", action="store_true",
+                    help="the two-stream schedule on one GPU: prediction, planning and the weight exchange on a "
+                         "side stream beside a stand-in attention; sweeps the SM pairs left to the router kernel")
+    ap.add_argument("--window-us", type=float, default=500.0, help="--overlap: length of the stand-in attention")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     ap.add_argument("--no-probe", action="store_true",
@@ -333,6 +447,10 @@ def main():
     T_global = wl.T
     if args.sharded:
         return run_sharded(args, wl, B, dist, dev, rank, local_rank, world, sampler)
+    if args.overlap:
+        sampler.stop()
+        print(json.dumps(run_overlap(wl, B, dev, args.window_us, reps=max(3, min(args.steps, 10)))), flush=True)
+        return
     T, E, R, k, d = wl.T, wl.E, wl.R, wl.k, wl.d
     bkw = budget_kwargs(wl, T)
     budget = B.make_budget(**bkw)

@@ -27,6 +27,15 @@ uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
  * alone inside a call that launches several kernels. */
 fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
 
+/* Stand-in for an attention kernel, for overlap experiments on one GPU (the method hides
+ * prediction, planning and weight transfer behind the target layer's attention; "Overlap
+ * Analysis").  A compute-bound kernel of `blocks` blocks, one per SM (1024 threads and 120 KB
+ * of shared memory each), each running iters x 32 dependent FMAs per thread: it occupies
+ * exactly `blocks` SMs for a time proportional to iters and leaves the other SMs - and room
+ * beside it for small memory-bound blocks - to other streams.  out: dev f32 [blocks * 1024]
+ * (receives meaningless values).  blocks 1..1024, iters 0..2^24. */
+fb_status fb_standin_attention(float* out, int32_t blocks, int32_t iters, fb_stream stream);
+
 /* SM clock probe.  A one-thread kernel on `stream` writes n pairs (global nanosecond timer,
  * SM cycle counter) into samples (dev u64 [2 n]), about period_ns apart, and ends by itself
  * (n <= 65536, period_ns <= 100000: at most a few seconds).  Between two samples the SMs ran

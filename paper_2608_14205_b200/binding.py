@@ -57,7 +57,8 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
            "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
            "fb_set_stamp_buffer", "fb_clock_probe", "fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns",
-           "fb_attention_set_time_ns", "fb_attention_reset", "fb_dispatch_slot_counts", "fb_dispatch_globalize"]
+           "fb_attention_set_time_ns", "fb_attention_reset", "fb_dispatch_slot_counts", "fb_dispatch_globalize",
+           "fb_standin_attention"]
 
 _lib = None
 
@@ -117,6 +118,8 @@ def lib() -> ctypes.CDLL:
     for name in ("fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns", "fb_attention_set_time_ns",
                  "fb_attention_reset"):
         getattr(L, name).restype = ctypes.c_int
+    L.fb_standin_attention.argtypes = [vp, i32, i32, vp]
+    L.fb_standin_attention.restype = ctypes.c_int
     L.fb_clock_probe.argtypes = [vp, i32, ctypes.c_uint32, vp]
     L.fb_clock_probe.restype = ctypes.c_int
     L.fb_set_stamp_buffer.argtypes = [vp, vp]
@@ -251,6 +254,11 @@ def fb_predict_load_static(cfg: FbConfig, device: int, router: FbRouter, x, T: i
     _check(lib().fb_predict_load_static(ctypes.byref(cfg), device, ctypes.byref(router), _ptr(x), T, _ptr(counts),
                                         _ptr(topk_ids), _ptr(status_word), _stream(stream)),
            "fb_predict_load_static")
+
+
+def fb_standin_attention(out, blocks: int, iters: int, stream=None) -> None:
+    """Compute-bound stand-in for attention on exactly `blocks` SMs (out: float32 [blocks * 1024])."""
+    _check(lib().fb_standin_attention(_ptr(out), blocks, iters, _stream(stream)), "fb_standin_attention")
 
 
 def fb_clock_probe(samples, n: int, period_ns: int, stream=None) -> None:

@@ -1028,6 +1028,24 @@ fb_status fb_attention_reset(fb_ctx* ctx) {
   return FB_OK;
 }
 
+fb_status fb_standin_attention(float* out, int32_t blocks, int32_t iters, fb_stream stream_) {
+  if (!out || blocks < 1 || blocks > 1024 || iters < 0 || iters > (1 << 24)) return FB_ERR_INVALID_ARG;
+  const int device = device_of(out);
+  if (device < 0) return FB_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  static bool raised[64] = {};
+  if (device < 64 && !raised[device]) {
+    if (cudaFuncSetAttribute(reinterpret_cast<const void*>(fb::fb_standin_attention_kernel),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, fb::kStandinSmemBytes) != cudaSuccess)
+      return FB_ERR_CUDA;
+    raised[device] = true;
+  }
+  fb::fb_standin_attention_kernel<<<static_cast<unsigned>(blocks), fb::kStandinThreads, fb::kStandinSmemBytes,
+                                    static_cast<cudaStream_t>(stream_)>>>(out, iters);
+  return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
 fb_status fb_clock_probe(uint64_t* samples, int32_t n, uint32_t period_ns, fb_stream stream_) {
   // bounded by construction: at most 65536 samples, at most 100 us apart
   if (!samples || n < 1 || n > 65536 || period_ns > 100000) return FB_ERR_INVALID_ARG;

@@ -55,7 +55,9 @@ typedef enum {
   FB_ERR_CUDA = 3,                         /* a CUDA runtime / driver call failed             */
   FB_ERR_BAD_PLACEMENT = 4,                /* device: expert_to_slot is not a bijection       */
   FB_ERR_TIMEOUT = 5,                      /* device: a bounded wait inside a kernel expired  */
-  FB_ERR_RANGE = 6                         /* device: sum of counts exceeds FB_MAX_COUNT_SUM  */
+  FB_ERR_RANGE = 6,                        /* device: sum of counts exceeds FB_MAX_COUNT_SUM  */
+  FB_ERR_INTERNAL = 7                      /* device, builds with -DFB_DEBUG only: an index the */
+                                           /* kernels were about to write was out of range      */
 } fb_status;
 
 /* The model's "original top-k rule" applied to the router logits (text after Eq. 4). */

@@ -49,6 +49,7 @@ FB_ERR_CUDA = 3
 FB_ERR_BAD_PLACEMENT = 4
 FB_ERR_TIMEOUT = 5
 FB_ERR_RANGE = 6
+FB_ERR_INTERNAL = 7
 
 EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_predict_load",
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",

@@ -440,6 +440,7 @@ const char* fb_status_string(fb_status s) {
     case FB_ERR_BAD_PLACEMENT: return "expert_to_slot is not a bijection";
     case FB_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case FB_ERR_RANGE: return "sum of counts beyond the planner's range";
+    case FB_ERR_INTERNAL: return "debug build: an output index was out of range";
   }
   return "unknown status";
 }

@@ -161,6 +161,9 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
     const long long i = static_cast<long long>(tile) * kDispatchTile + row;
     if (tile >= tile_end || j >= k || i >= p.T) return -1;
     const int e = p.topk_ids[i * k + j];
+#ifdef FB_DEBUG
+    if (e < 0 || e >= E) atomicCAS(p.status, 0, FB_ERR_INTERNAL);       // an expert id outside [0, E)
+#endif
     return (e < 0 || e >= E) ? 0 : e;
   };
   int e_cur = load_id(tile_begin);
@@ -178,6 +181,10 @@ fb_dispatch_kernel(const __grid_constant__ DispatchParams p) {
       for (int w = 0; w < (row >> 5); ++w) ahead += __popc(mask[mb][my_slot][w]);
       const long long pos = static_cast<long long>(offs[my_slot]) + before[par][my_slot] + ahead;
       const long long flat = (static_cast<long long>(tile) * kDispatchTile + row) * k + j;
+#ifdef FB_DEBUG
+      if (pos < 0 || pos >= n_assign || flat >= n_assign || my_slot < 0 || my_slot >= E)
+        atomicCAS(p.status, 0, FB_ERR_INTERNAL);                          // a position outside [0, T k) or a slot outside [0, E)
+#endif
       if (pos < n_assign) {
         p.perm[pos] = static_cast<int32_t>(flat);
         p.inv_perm[flat] = static_cast<int32_t>(pos);

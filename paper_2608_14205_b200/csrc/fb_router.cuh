@@ -281,6 +281,21 @@ __device__ __forceinline__ void write_row_outputs(const TopK& top, const RouterP
                                                   float sm_max, float sm_sum) {
   const int k = p.k;
   const bool sigmoid_gate = p.gate != FB_GATE_SOFTMAX_TOPK;
+#ifdef FB_DEBUG
+  // what the sanitizer would catch: a chosen expert outside [0, E), a repeated expert, a row outside [0, T)
+  {
+    bool bad = row < 0 || row >= p.T;
+#pragma unroll
+    for (int j = 0; j < FB_MAX_TOPK; ++j) {
+      if (j < k) {
+        bad = bad || top.i[j] < 0 || top.i[j] >= p.E;
+#pragma unroll
+        for (int h = 0; h < FB_MAX_TOPK; ++h) bad = bad || (h < j && top.i[h] == top.i[j]);
+      }
+    }
+    if (bad) atomicCAS(p.status, 0, FB_ERR_INTERNAL);
+  }
+#endif
   if (out_ids != nullptr) {
 #pragma unroll
     for (int j = 0; j < FB_MAX_TOPK; ++j)

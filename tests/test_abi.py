@@ -55,8 +55,8 @@ def test_cost_helper_reports_overflow():
 
 def test_status_strings():
     L = B.lib()
-    seen = {L.fb_status_string(s).decode() for s in range(7)}
-    assert len(seen) == 7 and all(seen)
+    seen = {L.fb_status_string(s).decode() for s in range(8)}
+    assert len(seen) == 8 and all(seen)
 
 
 def test_create_rejects_bad_shapes_before_touching_a_device():

@@ -407,6 +407,18 @@ fb_status fb_topk_hits(const int32_t* ids_a, const int32_t* ids_b, int32_t T, in
  * weights are renormalised); other shapes ignore it.  Returns FB_ERR_INVALID_ARG for a
  * negative limit. */
 fb_status fb_set_pair_limit(fb_ctx* ctx, int32_t pairs);
+/* k-range split of the router kernel (on by default).  When a call has fewer 256-row tile pairs
+ * than block pairs fit on the GPU (and the persistent kernel is not used), the spare pairs sum
+ * the tail of every tile's k-range into partial tiles that the tiles' owners add before their
+ * epilogue, so that every SM's tensor core works through the whole main loop (128 tiles leave
+ * 20 of 148 SMs idle otherwise; the smaller shapes leave more than half).  The schedule is a
+ * function of the shape and of the number of pairs only: a call is reproducible, but its logits
+ * differ from an unsplit call's in the order of the fp32 additions (both stay within the
+ * library's tolerance of the fp64 product), so a token whose k-th and (k+1)-th keys are closer
+ * than that rounding may be routed differently by the two.  mode 0 switches the split off, 1 on;
+ * owner_bias_kblocks tunes how many k-blocks more than an even share a tile's owner keeps
+ * (-1: built-in choice).  FB_ERR_INVALID_ARG for other values. */
+fb_status fb_set_split(fb_ctx* ctx, int32_t mode, int32_t owner_bias_kblocks);
 /* Block pairs of the persistent router kernel that fit on the GPU at once (0 when the
  * configuration does not support that kernel). */
 int32_t fb_max_pairs(const fb_ctx* ctx);

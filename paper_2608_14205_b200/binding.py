@@ -59,7 +59,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
            "fb_set_stamp_buffer", "fb_clock_probe", "fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns",
            "fb_attention_set_time_ns", "fb_attention_reset", "fb_dispatch_slot_counts", "fb_dispatch_globalize",
-           "fb_standin_attention"]
+           "fb_standin_attention", "fb_set_split"]
 
 _lib = None
 
@@ -119,6 +119,8 @@ def lib() -> ctypes.CDLL:
     for name in ("fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns", "fb_attention_set_time_ns",
                  "fb_attention_reset"):
         getattr(L, name).restype = ctypes.c_int
+    L.fb_set_split.argtypes = [vp, i32, i32]
+    L.fb_set_split.restype = ctypes.c_int
     L.fb_standin_attention.argtypes = [vp, i32, i32, vp]
     L.fb_standin_attention.restype = ctypes.c_int
     L.fb_clock_probe.argtypes = [vp, i32, ctypes.c_uint32, vp]
@@ -344,6 +346,9 @@ class Context:
 
     def fb_set_pair_limit(self, pairs: int) -> None:
         _check(lib().fb_set_pair_limit(self._h, pairs), "fb_set_pair_limit")
+
+    def fb_set_split(self, mode: int, owner_bias_kblocks: int = -1) -> None:
+        _check(lib().fb_set_split(self._h, mode, owner_bias_kblocks), "fb_set_split")
 
     def fb_max_pairs(self) -> int:
         return int(lib().fb_max_pairs(self._h))

@@ -50,6 +50,15 @@ struct fb_ctx {
   int max_pairs = 0;
   int pair_limit = 0;
   int dispatch_blocks_max = 296;       // resident blocks of the dispatch-index kernel (2 per SM)
+  // k-range split of the one-tile pair kernel: block pairs that fit on the GPU at once, the
+  // partial tiles and their flags (one slot per helper item), a launch counter for the flags'
+  // epoch, and the caller's switch / tuning value
+  int split_pairs = 0;
+  float* split_partial = nullptr;
+  uint32_t* split_flags = nullptr;
+  uint32_t split_epoch = 0;
+  int split_mode = 1;                  // 0 off, 1 on
+  int split_bias = -1;                 // extra k-blocks an owner keeps (-1: the built-in choice)
   EncodeTiledFn encode = nullptr;
   // device scratch
   uint32_t* counts_scratch = nullptr;   // [256], zero between calls
@@ -205,6 +214,16 @@ static RouterKernelFn router_kernel_fn(int sel, bool lb) {
     default: return fb::fb_router_kernel<kCtas, fb::kSelectSoftmaxRank, true>;
   }
 }
+static RouterKernelFn router_split_kernel_fn(int sel, bool lb) {
+  switch (sel * 2 + (lb ? 1 : 0)) {
+    case 0: return fb::fb_router_kernel<2, fb::kSelectGeneral, false, true>;
+    case 1: return fb::fb_router_kernel<2, fb::kSelectGeneral, true, true>;
+    case 2: return fb::fb_router_kernel<2, fb::kSelectSigmoidRank, false, true>;
+    case 3: return fb::fb_router_kernel<2, fb::kSelectSigmoidRank, true, true>;
+    case 4: return fb::fb_router_kernel<2, fb::kSelectSoftmaxRank, false, true>;
+    default: return fb::fb_router_kernel<2, fb::kSelectSoftmaxRank, true, true>;
+  }
+}
 static RouterKernelFn persistent_kernel_fn(bool sigmoid, bool lb) {
   if (sigmoid) return lb ? fb::fb_router_persistent_kernel<true, true> : fb::fb_router_persistent_kernel<true, false>;
   return lb ? fb::fb_router_persistent_kernel<false, true> : fb::fb_router_persistent_kernel<false, false>;
@@ -281,6 +300,40 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
       p.stages = ctx->persist_stages;
     }
   }
+  // Fewer tile pairs than block pairs fit on the GPU: the spare pairs become helpers that sum
+  // the tail of every tile's k-range (see RouterParams).  The schedule depends on the shape and
+  // on the number of pairs only.
+  bool split = false;
+  if (pair && !persistent && mode != fb::kModeLayer && ctx->split_partial != nullptr && ctx->split_mode != 0) {
+    const int tile_pairs = tiles_pad / 2;
+    int pairs_avail = ctx->split_pairs;
+    if (ctx->pair_limit > 0 && ctx->pair_limit < pairs_avail) pairs_avail = ctx->pair_limit;
+    const int spare = pairs_avail - tile_pairs;
+    // Worth it only where at least half of the pairs would idle: with 64 tile pairs on 74 block
+    // pairs (the 16k-token DeepSeek-V3 shape) the main loop is bound by HBM, not by the tensor
+    // cores of the busy SMs, and helpers only add their copy-outs (measured: 60 -> 68 us).
+    if (spare >= tile_pairs && p.num_kb >= 32) {
+      int J = spare / tile_pairs;                      // helpers per tile: J pieces each
+      if (J > 3) J = 3;
+      const int helpers = tile_pairs * J;
+      int ko = (p.num_kb + J) / (J + 1);
+      // a helper pays for the copy-out of its partial, the owner for reading it: owners keep a
+      // few k-blocks more than an even share
+      ko += ctx->split_bias >= 0 ? ctx->split_bias : 2;
+      if (ko > p.num_kb - 2 * J) ko = p.num_kb - 2 * J;     // every piece has at least two k-blocks
+      if (ko >= 2) {
+        split = true;
+        p.split_helpers = helpers;
+        p.split_ko = ko;
+        p.split_j = J;
+        if (++ctx->split_epoch == 0) ctx->split_epoch = 1;
+        p.split_epoch = ctx->split_epoch;
+        p.split_partial = ctx->split_partial;
+        p.split_flags = ctx->split_flags;
+        blocks += 2 * helpers;
+      }
+    }
+  }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.blockDim = dim3(fb::kRouterThreads, 1, 1);
@@ -306,6 +359,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
     cfg.numAttrs = 2;
     const bool lb = router->logit_bias != nullptr;
     err = cudaLaunchKernelEx(&cfg, persistent ? persistent_kernel_fn(c.gate == FB_GATE_SIGMOID_GROUP_TOPK, lb)
+                                   : split    ? router_split_kernel_fn(sel, lb)
                                               : router_kernel_fn<2>(sel, lb), *mx, *mx2, *mw, p);
   } else {
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
@@ -421,6 +475,7 @@ static fb_status ensure_kernel_attributes(int device, const cudaDeviceProp& prop
     for (int lb = 0; lb < 2; ++lb) {
       raise(router_kernel_fn<1>(sel, lb != 0));
       raise(router_kernel_fn<2>(sel, lb != 0));
+      raise(router_split_kernel_fn(sel, lb != 0));
     }
   for (int sg = 0; sg < 2; ++sg)
     for (int lb = 0; lb < 2; ++lb) raise(persistent_kernel_fn(sg != 0, lb != 0));
@@ -518,6 +573,29 @@ fb_status fb_create(fb_ctx** out, const fb_config* cfg, int device) {
       ctx->persist_stages = 0;                           // not usable here: the one-tile kernel serves every call
     cudaGetLastError();
   }
+  if (ctx->stages[1] >= 2) {
+    // block pairs of the one-tile pair kernel that the GPU holds at once: the grid of a split launch
+    cudaLaunchConfig_t occ;
+    memset(&occ, 0, sizeof(occ));
+    occ.gridDim = dim3(2 * static_cast<unsigned>(prop.multiProcessorCount), 1, 1);
+    occ.blockDim = dim3(fb::kRouterThreads, 1, 1);
+    occ.dynamicSmemBytes = ctx->smem_bytes[1];
+    cudaLaunchAttribute cl[1];
+    cl[0].id = cudaLaunchAttributeClusterDimension;
+    cl[0].val.clusterDim.x = 2; cl[0].val.clusterDim.y = 1; cl[0].val.clusterDim.z = 1;
+    occ.attrs = cl;
+    occ.numAttrs = 1;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, router_split_kernel_fn(0, false), &occ) == cudaSuccess &&
+        n_clusters >= 2) {
+      ctx->split_pairs = n_clusters;
+      const size_t slots = static_cast<size_t>(n_clusters);          // one partial per helper item, at most
+      ok = ok && dev_alloc(&ctx->split_partial, slots * 2 * ctx->N * fb::kTileM) &&
+           dev_alloc(&ctx->split_flags, slots * 2) &&
+           cudaMemset(ctx->split_flags, 0, slots * 2 * sizeof(uint32_t)) == cudaSuccess;
+    }
+    cudaGetLastError();
+  }
   ok = ok && dev_alloc(&ctx->counts_scratch, FB_MAX_EXPERTS) && dev_alloc(&ctx->ticket, 1) &&
        dev_alloc(&ctx->status, 1) &&
        dev_alloc(&ctx->tile_counts, static_cast<size_t>(ctx->max_tiles) * cfg->E) &&
@@ -535,7 +613,8 @@ fb_status fb_destroy(fb_ctx* ctx) {
   if (!ctx) return FB_OK;
   DeviceGuard guard(ctx->device);
   cudaDeviceSynchronize();
-  void* ptrs[] = {ctx->counts_scratch, ctx->ticket, ctx->status, ctx->tile_counts, ctx->super_counts, ctx->st_hprev, ctx->st_H,
+  void* ptrs[] = {ctx->split_partial, ctx->split_flags,
+                  ctx->counts_scratch, ctx->ticket, ctx->status, ctx->tile_counts, ctx->super_counts, ctx->st_hprev, ctx->st_H,
                   ctx->st_pi, ctx->st_pi_out, ctx->st_counts, ctx->st_swaps, ctx->st_nswaps, ctx->st_load_before,
                   ctx->st_load_after, ctx->st_ids, ctx->st_w, ctx->st_slot_offsets, ctx->st_rank_offsets,
                   ctx->st_perm, ctx->st_inv_perm, ctx->st_rank_load};
@@ -913,6 +992,13 @@ fb_status fb_topk_hits(const int32_t* ids_a, const int32_t* ids_b, int32_t T, in
   if (cudaMemsetAsync(hits_out, 0, sizeof(uint32_t), stream) != cudaSuccess) return FB_ERR_CUDA;
   if (T > 0) fb::fb_topk_hits_kernel<<<(T + 255) / 256, 256, 0, stream>>>(ids_a, ids_b, T, k, hits_out);
   return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+}
+
+fb_status fb_set_split(fb_ctx* ctx, int32_t mode, int32_t owner_bias_kblocks) {
+  if (!ctx || (mode != 0 && mode != 1) || owner_bias_kblocks < -1 || owner_bias_kblocks > 1024) return FB_ERR_INVALID_ARG;
+  ctx->split_mode = mode;
+  ctx->split_bias = owner_bias_kblocks;
+  return FB_OK;
 }
 
 fb_status fb_set_pair_limit(fb_ctx* ctx, int32_t pairs) {

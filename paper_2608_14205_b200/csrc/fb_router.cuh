@@ -97,6 +97,17 @@ struct RouterParams {
   float* logits;                     // [T][E] or nullptr
   uint32_t* tile_counts;             // [tiles][E]    (dispatch mode)
   unsigned long long* stamps;        // [blocks][64] phase time stamps (FB_TIMING builds) or nullptr
+  // k-range split (kSplit instances): the first 2 * split_helpers blocks are helper pairs, the
+  // tiles' owners follow.  An owner accumulates k-blocks [0, split_ko) of its tile; the rest,
+  // [split_ko, num_kb), is cut into split_j pieces, each summed by one helper pair (helper
+  // t * split_j + j for piece j of tile pair t) into a partial tile in global memory that the
+  // owner adds before its epilogue.
+  int32_t split_helpers;             // helper pairs in the grid (0: no split)
+  int32_t split_ko;                  // k-blocks an owner keeps
+  int32_t split_j;                   // pieces per tile = helper pairs per tile pair
+  uint32_t split_epoch;              // value a partial's flag takes when the partial of THIS launch is complete
+  float* split_partial;              // [slot][2 blocks][N columns][128 rows]
+  uint32_t* split_flags;             // [slot][2 blocks]
   PlanParams plan;
 };
 
@@ -380,6 +391,28 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32
   tmem_ld_wait();
 }
 
+// Wait until a partial's flag carries this launch's epoch (bounded like every other wait).
+__device__ __forceinline__ bool flag_wait(const uint32_t* flag, uint32_t epoch, volatile int* abort_flag) {
+  uint32_t polls = 0;
+  uint64_t t0 = 0;
+  for (;;) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v == epoch) return true;
+    if ((++polls & 0x3Fu) == 0) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
+// Offset (in floats) of column `col`, row 0 of the partial tile that block `cta` of a pair owns in `slot`.
+__device__ __forceinline__ size_t partial_offset(int slot, uint32_t cta, int N, int col) {
+  return ((static_cast<size_t>(slot) * 2 + cta) * static_cast<size_t>(N) + static_cast<size_t>(col)) * kTileM;
+}
+
 // kCtas == 1: every block computes its 128 x N tile alone.
 // kCtas == 2: launched in clusters of two; the pair shares one 256 x N MMA
 // (tcgen05 cta_group::2).  Each block still loads its own 128 rows of x, but only half
@@ -390,7 +423,13 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32
 // the registers its gate needs; the host picks it with select_kind().
 // kLogitBias: whether a logit bias (Eq. 2's "+ b") is given; without it the key computation
 // shrinks to one variant.
-template <int kCtas, int kSel, bool kLogitBias>
+// kSplit (pairs only): the grid has more block pairs than the call has tile pairs, and the spare
+// pairs take the tail of every tile's k-range (see RouterParams).  A tile that fills one SM
+// pair for the whole main loop leaves the spare SMs' tensor cores idle otherwise (128 tiles on
+// 148 SMs; 64 tiles on 148 SMs for the smaller shapes).  The split is a function of the shape
+// and of the number of pairs only, so a call's result is reproducible; its logits differ from
+// the unsplit kernel's in the order of the fp32 additions.
+template <int kCtas, int kSel, bool kLogitBias, bool kSplit = false>
 __global__ void __launch_bounds__(kRouterThreads, 1)
 fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x2,
                  const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ RouterParams p) {
@@ -402,7 +441,10 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   // kModeLayer: which pass this block belongs to, its tile there and its input
   const bool second_pass = p.mode == kModeLayer && static_cast<int>(blockIdx.x) >= p.tiles_first;
   const int mode = p.mode == kModeLayer ? (second_pass ? kModeDispatch : kModePredictPlan) : p.mode;
-  const int tile = second_pass ? static_cast<int>(blockIdx.x) - p.tiles_first : static_cast<int>(blockIdx.x);
+  const bool is_helper = kSplit && static_cast<int>(blockIdx.x) < 2 * p.split_helpers;
+  const int owner_block = kSplit ? static_cast<int>(blockIdx.x) - 2 * p.split_helpers : static_cast<int>(blockIdx.x);
+  const int tile = second_pass ? owner_block - p.tiles_first : owner_block;
+  const int kb_end = kSplit ? p.split_ko : p.num_kb;        // k-blocks this block accumulates for its own tile
   const CUtensorMap* xmap = second_pass ? &tmap_x2 : &tmap_x;
   // outputs of the normal pass are not written by blocks of the early pass
   int32_t* const out_ids = (p.mode == kModeLayer && !second_pass) ? nullptr : p.topk_ids;
@@ -455,511 +497,628 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   const uint32_t tmem_base = sh.tmem_base;
   FB_STAMP(1, 64);
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      const uint64_t pol_x = l2_policy_evict_first();   // x is streamed once
-      const uint64_t pol_w = l2_policy_evict_last();    // W is re-read by every block
-      for (int kb = 0; kb < p.num_kb; ++kb) {
-        const int s = kb % p.stages;
-        const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
-        if (!mbar_wait<kCtas == 2>(smem_u32(&sh.empty_bar[s]), phase ^ 1u, abort_flag)) break;
-        if (kb == 0) FB_STAMP(14, 0);
-        if (kb == p.num_kb - 1) FB_STAMP(15, 0);
-        const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
-        if (kCtas == 1) {
-          const uint32_t full = smem_u32(&sh.full_bar[s]);
-          mbar_arrive_expect_tx(full, stage_bytes);
-          tma_load_2d(a_dst, xmap, full, kb * kBlockK, tile * kTileM, pol_x);
-          tma_load_2d(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK, 0, pol_w);
-        } else {
-          // both blocks report their bytes to the even block's barrier, which expects
-          // the bytes of the whole pair
+  if (is_helper) {
+    // ============================================================ helper pair (kSplit instances)
+    // Helper pair hp sums piece j = hp % split_j of the remaining k-blocks [split_ko, num_kb) of
+    // tile pair t = hp / split_j into the partial tile of slot hp.  Even / odd k-blocks of the
+    // piece go to the two issuers' accumulators as in an owner.
+    const int hp = static_cast<int>(blockIdx.x) >> 1;
+    const int rest = p.num_kb - p.split_ko;
+    const int tp = hp / p.split_j, piece = hp % p.split_j;
+    const int kb0 = p.split_ko + rest * piece / p.split_j, kb1 = p.split_ko + rest * (piece + 1) / p.split_j;
+    const int my_tile = 2 * tp + static_cast<int>(cta_rank);
+    if (warp == 0) {
+      // ---------------------------------------------------------- TMA producer
+      if (lane == 0) {
+        const uint64_t pol_x = l2_policy_evict_first();
+        const uint64_t pol_w = l2_policy_evict_last();
+        for (int kb = kb0; kb < kb1; ++kb) {
+          const int s = (kb - kb0) % p.stages;
+          const uint32_t phase = static_cast<uint32_t>((kb - kb0) / p.stages) & 1u;
+          if (!mbar_wait<true>(smem_u32(&sh.empty_bar[s]), phase ^ 1u, abort_flag)) break;
+          const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
           const uint32_t full = map_to_cta(smem_u32(&sh.full_bar[s]), 0u);
           if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&sh.full_bar[s]), 2u * stage_bytes);
-          tma_load_2d_pair(a_dst, xmap, full, kb * kBlockK, tile * kTileM, pol_x);
+          tma_load_2d_pair(a_dst, &tmap_x, full, kb * kBlockK, my_tile * kTileM, pol_x);
           tma_load_2d_pair(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK,
                            static_cast<int32_t>(cta_rank) * (p.N / 2), pol_w);
         }
       }
-    }
-    __syncwarp();
-    if (kCtas == 2) cluster_arrive();          // this warp is done with the pair's shared state (see the teardown)
-  } else if (warp == 1 || warp == kSecondIssuerWarp) {
-    // ------------------------------------------------------------ MMA issuers
-    // warp 1: k-blocks 0, 2, 4, ... into accumulator 0; the last warp: 1, 3, 5, ... into
-    // accumulator 1 (N columns further).  In a pair only the even block issues.
-    if (lane == 0 && cta_rank == 0) {
-      const int first_kb = warp == 1 ? 0 : 1;
-      const uint32_t acc = tmem_base + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
-      const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.N));
-      bool ok = true;
-      for (int kb = first_kb; kb < p.num_kb && ok; kb += 2) {
-        const int s = kb % p.stages;
-        const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
-        ok = mbar_wait<kCtas == 2>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
-        if (!ok) break;
+      __syncwarp();
+      cluster_arrive();
+    } else if (warp == 1 || warp == kSecondIssuerWarp) {
+      // ---------------------------------------------------------- MMA issuers (even block only)
+      if (lane == 0 && cta_rank == 0) {
+        const int first_kb = kb0 + (warp == 1 ? 0 : 1);
+        const uint32_t acc = tmem_base + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
+        const uint32_t idesc = umma_idesc_bf16_f32(kTileM * 2, static_cast<uint32_t>(p.N));
+        bool ok = true;
+        for (int kb = first_kb; kb < kb1 && ok; kb += 2) {
+          const int s = (kb - kb0) % p.stages;
+          const uint32_t phase = static_cast<uint32_t>((kb - kb0) / p.stages) & 1u;
+          ok = mbar_wait<true>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
+          if (!ok) break;
+          tcgen05_fence_after();
+          const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
+          const uint64_t adesc = umma_smem_desc_sw128(a_addr);
+          const uint64_t bdesc = umma_smem_desc_sw128(a_addr + kATileBytes);
+#pragma unroll
+          for (int kk = 0; kk < kBlockK / kUmmaK; ++kk)
+            umma_bf16<2>(acc, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb != first_kb || kk != 0) ? 1u : 0u);
+          umma_commit_pair(smem_u32(&sh.empty_bar[s]), cta_rank);
+        }
+        umma_commit_pair(smem_u32(&sh.accum_bar), cta_rank);      // this issuer's share of the piece is complete
+      }
+      __syncwarp();
+      cluster_arrive();
+    } else {
+      // ---------------------------------------------------------- copy-out warps
+      const int et = threadIdx.x - 64;
+      const int quarter = warp & 3;
+      const int sub = (warp - 2) >> 2;
+      const int row_in_tile = quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+      const int N = p.N;
+      const int n_chunks = (N + 31) >> 5;
+      if (et == 0) sh.accum_ok = mbar_wait<true>(smem_u32(&sh.accum_bar), 0u, abort_flag) ? 1 : 0;
+      named_bar_sync(kAccumBarrierId, kEpilogueThreads);
+      if (sh.accum_ok != 0) {
         tcgen05_fence_after();
-        if (kb == 0) FB_STAMP(16, 32);
-        const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
-        const uint64_t adesc = umma_smem_desc_sw128(a_addr);
-        const uint64_t bdesc = umma_smem_desc_sw128(a_addr + kATileBytes);
-#pragma unroll
-        for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
-          // advance 16 elements = 32 bytes inside the swizzled row: +2 in the address field
-          umma_bf16<kCtas>(acc, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb != first_kb || kk != 0) ? 1u : 0u);
-        }
-        // frees the stage (in both blocks of a pair) when these MMAs retire
-        if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.empty_bar[s]));
-        else umma_commit_pair(smem_u32(&sh.empty_bar[s]), cta_rank);
-      }
-      if (warp == 1) FB_STAMP(17, 32);
-      // this issuer's accumulator is complete
-      if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.accum_bar));
-      else umma_commit_pair(smem_u32(&sh.accum_bar), cta_rank);
-    }
-    if (warp == 1) {
-    // One thread polls for the finished accumulator on behalf of the 16 epilogue warps,
-    // which sleep at a hardware barrier meanwhile (no issue slots, no power).
-    if (lane == 0) sh.accum_ok = mbar_wait<kCtas == 2>(smem_u32(&sh.accum_bar), 0u, abort_flag) ? 1 : 0;
-    __syncwarp();
-    named_bar_arrive(kAccumBarrierId, kEpilogueThreads + 32);
-    }
-    __syncwarp();
-    if (kCtas == 2) cluster_arrive();
-  } else {
-    // ------------------------------------------------------------ epilogue
-    const int et = threadIdx.x - 64;                       // 0 .. kEpilogueThreads-1
-    const int quarter = warp & 3;                          // TMEM lanes this warp may touch
-    const int sub = (warp - 2) >> 2;                       // which share of the columns
-    const int row_in_tile = quarter * 32 + lane;
-    const long long row = static_cast<long long>(tile) * kTileM + row_in_tile;
-    const bool valid = row < p.T;
-    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-    const int E = p.E, N = p.N, k = p.k;
-    const bool sigmoid_gate = kSel == kSelectSigmoidRank ? true
-                              : kSel == kSelectSoftmaxRank ? false : p.gate != FB_GATE_SOFTMAX_TOPK;
-    const int gs = kSel == kSelectSigmoidRank ? 32 : (sigmoid_gate ? E / p.n_group : E);   // experts per group
-    // Which sub owns chunk c: whole groups must stay with one sub.
-    const int n_chunks = (N + 31) >> 5;
-    const int chunks_per_group = (sigmoid_gate && gs % 32 == 0) ? gs / 32 : 1;
-    const bool splittable = !sigmoid_gate || gs % 32 == 0 || 32 % gs == 0;
-    const bool want_sum = kSel == kSelectGeneral && out_w != nullptr && !p.renorm && !sigmoid_gate;
-    // Selection by ranking a short candidate list instead of insertion (see select_kind).
-    constexpr bool fast_select = kSel != kSelectGeneral;
-
-    // Chunk bookkeeping, worked out while the main loop runs (integer divisions by run-time
-    // values are slow and would otherwise sit between the chunks of the epilogue):
-    // which chunks this warp owns, which of them end a group, and each chunk's group.
-    uint32_t owned_chunks = 0, group_end_chunks = 0, chunk_group = 0;     // bit c / nibble c
-    for (int c = 0; c < n_chunks; ++c) {
-      const int owner = splittable ? (c / chunks_per_group) % kEpiSubs : 0;
-      if (owner == sub) owned_chunks |= 1u << c;
-      if (sigmoid_gate && gs % 32 == 0) {
-        if ((c * 32 + 32) % gs == 0) group_end_chunks |= 1u << c;
-        chunk_group |= static_cast<uint32_t>((c * 32) / gs) << (4 * c);   // at most 8 groups here
-      }
-    }
-    // While the main loop runs, stage the biases (read by these warps only, after the barrier
-    // below) and the placement for the planner (any block may turn out to be the last one).
-    for (int e = et; e < FB_MAX_EXPERTS + 32; e += kEpilogueThreads) {
-      sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
-      sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
-    }
-    if (mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
-    named_bar_sync(kAccumBarrierId, kEpilogueThreads + 32);
-    const bool got = sh.accum_ok != 0;
-    tcgen05_fence_after();
-    FB_STAMP(2, 64);
-
-    // scratch carved out of the (now idle) pipeline stages
-    float* key_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // [N][128]
-    float* gscore_s = key_s + static_cast<size_t>(N) * kTileM;                               // [32][128]
-    float* glow_s = gscore_s + FB_MAX_GROUPS * kTileM;                                       // [32][128]
-    float* merge_v = glow_s + FB_MAX_GROUPS * kTileM;                                        // [subs-1][8][128]
-    int32_t* merge_i = reinterpret_cast<int32_t*>(merge_v + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);
-    float* part_s = reinterpret_cast<float*>(merge_i + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);   // [subs][2][128]
-
-    TopK top;
-    top.init();
-    float sm_max = -INFINITY, sm_sum = 0.0f;               // softmax denominator (weights without renorm)
-    constexpr bool has_lb = kLogitBias;
-    if (got) {
-      // ---------------- pass 1
-      float m1 = -INFINITY, m2 = -INFINITY;
-      for (int c = 0; c < n_chunks; ++c) {
-        if (((owned_chunks >> c) & 1u) == 0) continue;
-        const int c0 = c * 32;
-        uint32_t r[32];
-        float q[32];
-        load_chunk(taddr, c0, N, r);
-        if (p.num_kb > 1) {                                  // add the odd k-blocks' accumulator
-          const int halves = (N - c0 >= 32) ? 2 : 1;         // 16 columns at a time keeps registers low
-          for (int h = 0; h < halves; ++h) {
-            uint32_t r2[32];
-            tmem_ld_32x32b_x16(taddr + N + c0 + 16 * h, r2);
-            tmem_ld_wait();
-            if (h == 0) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) r[16 + j] = __float_as_uint(__uint_as_float(r[16 + j]) + __uint_as_float(r2[j]));
-            }
-          }
-        }
-        if (p.logits != nullptr && valid) {
+        // every piece has at least two k-blocks (the host sees to it): both accumulators are live
+        float* part = p.split_partial + partial_offset(hp, cta_rank, N, 0) + row_in_tile;
+        for (int c = sub; c < n_chunks; c += kEpiSubs) {
+          const int c0 = c * 32;
+          uint32_t r[32], r2[32];
+          load_chunk(taddr, c0, N, r);
+          load_chunk(taddr + N, c0, N, r2);
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (c0 + j < E)
-              p.logits[row * E + c0 + j] = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
+            if (c0 + j < N) __stcg(part + static_cast<size_t>(c0 + j) * kTileM, __uint_as_float(r[j]) + __uint_as_float(r2[j]));
         }
-        if (sigmoid_gate && c0 + 32 <= E && !has_lb) {
-          // whole chunk valid, no logit bias (the common case).  Every key goes through the
-          // same two hardware approximations, so equal logits give equal keys in every column
-          // (an FMA-pipe reciprocal on alternate columns was no faster and broke exact ties).
-          const float4* sb4 = reinterpret_cast<const float4*>(&sh.select_bias[c0]);
-#pragma unroll
-          for (int j4 = 0; j4 < 8; ++j4) {
-            const float4 b = sb4[j4];
-            q[4 * j4 + 0] = fb_sigmoid(__uint_as_float(r[4 * j4 + 0])) + b.x;
-            q[4 * j4 + 1] = fb_sigmoid(__uint_as_float(r[4 * j4 + 1])) + b.y;
-            q[4 * j4 + 2] = fb_sigmoid(__uint_as_float(r[4 * j4 + 2])) + b.z;
-            q[4 * j4 + 3] = fb_sigmoid(__uint_as_float(r[4 * j4 + 3])) + b.w;
-          }
-        } else if (sigmoid_gate) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float z = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
-            q[j] = (c0 + j < E) ? fb_sigmoid(z) + sh.select_bias[c0 + j] : -INFINITY;
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float z = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
-            q[j] = (c0 + j < E) ? z : -INFINITY;
+        tcgen05_fence_before();
+        // publish the partial: every thread's stores, then one release of the flag
+        named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+        if (et == 0) {
+          __threadfence();
+          uint32_t* flag = p.split_flags + static_cast<size_t>(hp) * 2 + cta_rank;
+          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(p.split_epoch) : "memory");
+        }
+      }
+      __syncwarp();
+      cluster_arrive();
+    }
+  } else {
+    if (warp == 0) {
+      // ------------------------------------------------------------ TMA producer
+      if (lane == 0) {
+        const uint64_t pol_x = l2_policy_evict_first();   // x is streamed once
+        const uint64_t pol_w = l2_policy_evict_last();    // W is re-read by every block
+        for (int kb = 0; kb < kb_end; ++kb) {
+          const int s = kb % p.stages;
+          const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
+          if (!mbar_wait<kCtas == 2>(smem_u32(&sh.empty_bar[s]), phase ^ 1u, abort_flag)) break;
+          if (kb == 0) FB_STAMP(14, 0);
+          if (kb == kb_end - 1) FB_STAMP(15, 0);
+          const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
+          if (kCtas == 1) {
+            const uint32_t full = smem_u32(&sh.full_bar[s]);
+            mbar_arrive_expect_tx(full, stage_bytes);
+            tma_load_2d(a_dst, xmap, full, kb * kBlockK, tile * kTileM, pol_x);
+            tma_load_2d(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK, 0, pol_w);
+          } else {
+            // both blocks report their bytes to the even block's barrier, which expects
+            // the bytes of the whole pair
+            const uint32_t full = map_to_cta(smem_u32(&sh.full_bar[s]), 0u);
+            if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&sh.full_bar[s]), 2u * stage_bytes);
+            tma_load_2d_pair(a_dst, xmap, full, kb * kBlockK, tile * kTileM, pol_x);
+            tma_load_2d_pair(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK,
+                             static_cast<int32_t>(cta_rank) * (p.N / 2), pol_w);
           }
         }
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (c0 + j < N) key_s[(c0 + j) * kTileM + row_in_tile] = q[j];
-        if (want_sum) {
-          float cmax = q[0];
-#pragma unroll
-          for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, q[j]);
-          const float nmax = fmaxf(sm_max, cmax);
-          float part = 0.0f;
-#pragma unroll
-          for (int j = 0; j < 32; ++j) part += __expf(q[j] - nmax);     // exp(-inf) = 0 for padding
-          sm_sum = sm_sum * __expf(sm_max - nmax) + part;
-          sm_max = nmax;
+      }
+      __syncwarp();
+      if (kCtas == 2) cluster_arrive();          // this warp is done with the pair's shared state (see the teardown)
+    } else if (warp == 1 || warp == kSecondIssuerWarp) {
+      // ------------------------------------------------------------ MMA issuers
+      // warp 1: k-blocks 0, 2, 4, ... into accumulator 0; the last warp: 1, 3, 5, ... into
+      // accumulator 1 (N columns further).  In a pair only the even block issues.
+      if (lane == 0 && cta_rank == 0) {
+        const int first_kb = warp == 1 ? 0 : 1;
+        const uint32_t acc = tmem_base + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
+        const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.N));
+        bool ok = true;
+        for (int kb = first_kb; kb < kb_end && ok; kb += 2) {
+          const int s = kb % p.stages;
+          const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
+          ok = mbar_wait<kCtas == 2>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
+          if (!ok) break;
+          tcgen05_fence_after();
+          if (kb == 0) FB_STAMP(16, 32);
+          const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
+          const uint64_t adesc = umma_smem_desc_sw128(a_addr);
+          const uint64_t bdesc = umma_smem_desc_sw128(a_addr + kATileBytes);
+  #pragma unroll
+          for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
+            // advance 16 elements = 32 bytes inside the swizzled row: +2 in the address field
+            umma_bf16<kCtas>(acc, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb != first_kb || kk != 0) ? 1u : 0u);
+          }
+          // frees the stage (in both blocks of a pair) when these MMAs retire
+          if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.empty_bar[s]));
+          else umma_commit_pair(smem_u32(&sh.empty_bar[s]), cta_rank);
         }
+        if (warp == 1) FB_STAMP(17, 32);
+        // this issuer's accumulator is complete
+        if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.accum_bar));
+        else umma_commit_pair(smem_u32(&sh.accum_bar), cta_rank);
+      }
+      if (warp == 1) {
+      // One thread polls for the finished accumulator on behalf of the 16 epilogue warps,
+      // which sleep at a hardware barrier meanwhile (no issue slots, no power).
+      if (lane == 0) {
+        bool ok = mbar_wait<kCtas == 2>(smem_u32(&sh.accum_bar), 0u, abort_flag);
+        if (kSplit) {
+          // ... and for the helpers' partial sums of this tile's remaining k-blocks
+          const int tp = tile >> 1;
+          for (int j = 0; j < p.split_j && ok; ++j)
+            ok = flag_wait(p.split_flags + (static_cast<size_t>(tp) * p.split_j + j) * 2 + cta_rank, p.split_epoch, abort_flag);
+        }
+        sh.accum_ok = ok ? 1 : 0;
+      }
+      __syncwarp();
+      named_bar_arrive(kAccumBarrierId, kEpilogueThreads + 32);
+      }
+      __syncwarp();
+      if (kCtas == 2) cluster_arrive();
+    } else {
+      // ------------------------------------------------------------ epilogue
+      const int et = threadIdx.x - 64;                       // 0 .. kEpilogueThreads-1
+      const int quarter = warp & 3;                          // TMEM lanes this warp may touch
+      const int sub = (warp - 2) >> 2;                       // which share of the columns
+      const int row_in_tile = quarter * 32 + lane;
+      const long long row = static_cast<long long>(tile) * kTileM + row_in_tile;
+      const bool valid = row < p.T;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+      const int E = p.E, N = p.N, k = p.k;
+      const bool sigmoid_gate = kSel == kSelectSigmoidRank ? true
+                                : kSel == kSelectSoftmaxRank ? false : p.gate != FB_GATE_SOFTMAX_TOPK;
+      const int gs = kSel == kSelectSigmoidRank ? 32 : (sigmoid_gate ? E / p.n_group : E);   // experts per group
+      // Which sub owns chunk c: whole groups must stay with one sub.
+      const int n_chunks = (N + 31) >> 5;
+      const int chunks_per_group = (sigmoid_gate && gs % 32 == 0) ? gs / 32 : 1;
+      const bool splittable = !sigmoid_gate || gs % 32 == 0 || 32 % gs == 0;
+      const bool want_sum = kSel == kSelectGeneral && out_w != nullptr && !p.renorm && !sigmoid_gate;
+      // Selection by ranking a short candidate list instead of insertion (see select_kind).
+      constexpr bool fast_select = kSel != kSelectGeneral;
+
+      // Chunk bookkeeping, worked out while the main loop runs (integer divisions by run-time
+      // values are slow and would otherwise sit between the chunks of the epilogue):
+      // which chunks this warp owns, which of them end a group, and each chunk's group.
+      uint32_t owned_chunks = 0, group_end_chunks = 0, chunk_group = 0;     // bit c / nibble c
+      for (int c = 0; c < n_chunks; ++c) {
+        const int owner = splittable ? (c / chunks_per_group) % kEpiSubs : 0;
+        if (owner == sub) owned_chunks |= 1u << c;
         if (sigmoid_gate && gs % 32 == 0) {
-          // the chunk lies inside one group: branch-free top-2 of its 32 keys by a merge tree
-          float a1[16], a2[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) { a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); }
-#pragma unroll
-          for (int w = 8; w >= 1; w >>= 1) {
-#pragma unroll
-            for (int j = 0; j < w; ++j) {
-              const float hi = fmaxf(a1[j], a1[j + w]);
-              a2[j] = fmaxf(fminf(a1[j], a1[j + w]), fmaxf(a2[j], a2[j + w]));
-              a1[j] = hi;
+          if ((c * 32 + 32) % gs == 0) group_end_chunks |= 1u << c;
+          chunk_group |= static_cast<uint32_t>((c * 32) / gs) << (4 * c);   // at most 8 groups here
+        }
+      }
+      // While the main loop runs, stage the biases (read by these warps only, after the barrier
+      // below) and the placement for the planner (any block may turn out to be the last one).
+      for (int e = et; e < FB_MAX_EXPERTS + 32; e += kEpilogueThreads) {
+        sh.logit_bias[e] = (p.logit_bias != nullptr && e < p.E) ? p.logit_bias[e] : 0.0f;
+        sh.select_bias[e] = (p.select_bias != nullptr && e < p.E) ? p.select_bias[e] : 0.0f;
+      }
+      if (mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
+      named_bar_sync(kAccumBarrierId, kEpilogueThreads + 32);
+      const bool got = sh.accum_ok != 0;
+      tcgen05_fence_after();
+      FB_STAMP(2, 64);
+
+      // scratch carved out of the (now idle) pipeline stages
+      float* key_s = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // [N][128]
+      float* gscore_s = key_s + static_cast<size_t>(N) * kTileM;                               // [32][128]
+      float* glow_s = gscore_s + FB_MAX_GROUPS * kTileM;                                       // [32][128]
+      float* merge_v = glow_s + FB_MAX_GROUPS * kTileM;                                        // [subs-1][8][128]
+      int32_t* merge_i = reinterpret_cast<int32_t*>(merge_v + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);
+      float* part_s = reinterpret_cast<float*>(merge_i + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);   // [subs][2][128]
+
+      TopK top;
+      top.init();
+      float sm_max = -INFINITY, sm_sum = 0.0f;               // softmax denominator (weights without renorm)
+      constexpr bool has_lb = kLogitBias;
+      if (got) {
+        // ---------------- pass 1
+        float m1 = -INFINITY, m2 = -INFINITY;
+        for (int c = 0; c < n_chunks; ++c) {
+          if (((owned_chunks >> c) & 1u) == 0) continue;
+          const int c0 = c * 32;
+          uint32_t r[32];
+          float q[32];
+          load_chunk(taddr, c0, N, r);
+          if (kb_end > 1) {                                    // add the odd k-blocks' accumulator
+            const int halves = (N - c0 >= 32) ? 2 : 1;         // 16 columns at a time keeps registers low
+            for (int h = 0; h < halves; ++h) {
+              uint32_t r2[32];
+              tmem_ld_32x32b_x16(taddr + N + c0 + 16 * h, r2);
+              tmem_ld_wait();
+              if (h == 0) {
+  #pragma unroll
+                for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+              } else {
+  #pragma unroll
+                for (int j = 0; j < 16; ++j) r[16 + j] = __float_as_uint(__uint_as_float(r[16 + j]) + __uint_as_float(r2[j]));
+              }
             }
           }
-          m2 = fmaxf(fminf(m1, a1[0]), fmaxf(m2, a2[0]));
-          m1 = fmaxf(m1, a1[0]);
-          if ((group_end_chunks >> c) & 1u) {                 // last chunk of the group
-            const int g = static_cast<int>((chunk_group >> (4 * c)) & 15u);
-            gscore_s[g * kTileM + row_in_tile] = m1 + m2;
-            glow_s[g * kTileM + row_in_tile] = m2;
-            m1 = -INFINITY; m2 = -INFINITY;
-          }
-        } else if (!sigmoid_gate && fast_select) {
-          // softmax gate, fast selection: the chunk's three best keys (sorted) feed the bound
-          float a1[16], a2[16], a3[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); a3[j] = -INFINITY;
-          }
-#pragma unroll
-          for (int w = 8; w >= 1; w >>= 1) {
-#pragma unroll
-            for (int j = 0; j < w; ++j) {
-              // best three of two sorted triples
-              const float lo1 = fminf(a1[j], a1[j + w]), hi2 = fmaxf(a2[j], a2[j + w]);
-              a1[j] = fmaxf(a1[j], a1[j + w]);
-              a2[j] = fmaxf(lo1, hi2);
-              a3[j] = fmaxf(fminf(lo1, hi2), fmaxf(a3[j], a3[j + w]));
+          if (kSplit) {
+            // add the helpers' partial sums of the remaining k-blocks, piece by piece in a fixed order;
+            // a partial tile is stored column by column, so the warp's 32 rows read 128 contiguous bytes
+            const int tp = tile >> 1;
+            for (int pj = 0; pj < p.split_j; ++pj) {
+              const float* part = p.split_partial + partial_offset(tp * p.split_j + pj, cta_rank, N, c0) + row_in_tile;
+  #pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                float pv[16];
+  #pragma unroll
+                for (int j = 0; j < 16; ++j) pv[j] = (c0 + 16 * h + j < N) ? __ldcg(part + (16 * h + j) * kTileM) : 0.0f;
+  #pragma unroll
+                for (int j = 0; j < 16; ++j) r[16 * h + j] = __float_as_uint(__uint_as_float(r[16 * h + j]) + pv[j]);
+              }
             }
           }
-          gscore_s[c * kTileM + row_in_tile] = a1[0];
-          gscore_s[(kBoundRows + c) * kTileM + row_in_tile] = a2[0];
-          gscore_s[(2 * kBoundRows + c) * kTileM + row_in_tile] = a3[0];
-        } else if (sigmoid_gate) {
-          int g = c0 / gs, pos = c0 % gs;
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (c0 + j < E) {
-              m2 = fmaxf(m2, fminf(m1, q[j]));
-              m1 = fmaxf(m1, q[j]);
-              if (++pos == gs) {                              // group complete (uniform branch)
-                gscore_s[g * kTileM + row_in_tile] = gs >= 2 ? m1 + m2 : m1;
-                glow_s[g * kTileM + row_in_tile] = gs >= 2 ? m2 : m1;
-                ++g; pos = 0; m1 = -INFINITY; m2 = -INFINITY;
+          if (p.logits != nullptr && valid) {
+  #pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c0 + j < E)
+                p.logits[row * E + c0 + j] = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
+          }
+          if (sigmoid_gate && c0 + 32 <= E && !has_lb) {
+            // whole chunk valid, no logit bias (the common case).  Every key goes through the
+            // same two hardware approximations, so equal logits give equal keys in every column
+            // (an FMA-pipe reciprocal on alternate columns was no faster and broke exact ties).
+            const float4* sb4 = reinterpret_cast<const float4*>(&sh.select_bias[c0]);
+  #pragma unroll
+            for (int j4 = 0; j4 < 8; ++j4) {
+              const float4 b = sb4[j4];
+              q[4 * j4 + 0] = fb_sigmoid(__uint_as_float(r[4 * j4 + 0])) + b.x;
+              q[4 * j4 + 1] = fb_sigmoid(__uint_as_float(r[4 * j4 + 1])) + b.y;
+              q[4 * j4 + 2] = fb_sigmoid(__uint_as_float(r[4 * j4 + 2])) + b.z;
+              q[4 * j4 + 3] = fb_sigmoid(__uint_as_float(r[4 * j4 + 3])) + b.w;
+            }
+          } else if (sigmoid_gate) {
+  #pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float z = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
+              q[j] = (c0 + j < E) ? fb_sigmoid(z) + sh.select_bias[c0 + j] : -INFINITY;
+            }
+          } else {
+  #pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float z = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
+              q[j] = (c0 + j < E) ? z : -INFINITY;
+            }
+          }
+  #pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < N) key_s[(c0 + j) * kTileM + row_in_tile] = q[j];
+          if (want_sum) {
+            float cmax = q[0];
+  #pragma unroll
+            for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, q[j]);
+            const float nmax = fmaxf(sm_max, cmax);
+            float part = 0.0f;
+  #pragma unroll
+            for (int j = 0; j < 32; ++j) part += __expf(q[j] - nmax);     // exp(-inf) = 0 for padding
+            sm_sum = sm_sum * __expf(sm_max - nmax) + part;
+            sm_max = nmax;
+          }
+          if (sigmoid_gate && gs % 32 == 0) {
+            // the chunk lies inside one group: branch-free top-2 of its 32 keys by a merge tree
+            float a1[16], a2[16];
+  #pragma unroll
+            for (int j = 0; j < 16; ++j) { a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); }
+  #pragma unroll
+            for (int w = 8; w >= 1; w >>= 1) {
+  #pragma unroll
+              for (int j = 0; j < w; ++j) {
+                const float hi = fmaxf(a1[j], a1[j + w]);
+                a2[j] = fmaxf(fminf(a1[j], a1[j + w]), fmaxf(a2[j], a2[j + w]));
+                a1[j] = hi;
+              }
+            }
+            m2 = fmaxf(fminf(m1, a1[0]), fmaxf(m2, a2[0]));
+            m1 = fmaxf(m1, a1[0]);
+            if ((group_end_chunks >> c) & 1u) {                 // last chunk of the group
+              const int g = static_cast<int>((chunk_group >> (4 * c)) & 15u);
+              gscore_s[g * kTileM + row_in_tile] = m1 + m2;
+              glow_s[g * kTileM + row_in_tile] = m2;
+              m1 = -INFINITY; m2 = -INFINITY;
+            }
+          } else if (!sigmoid_gate && fast_select) {
+            // softmax gate, fast selection: the chunk's three best keys (sorted) feed the bound
+            float a1[16], a2[16], a3[16];
+  #pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              a1[j] = fmaxf(q[2 * j], q[2 * j + 1]); a2[j] = fminf(q[2 * j], q[2 * j + 1]); a3[j] = -INFINITY;
+            }
+  #pragma unroll
+            for (int w = 8; w >= 1; w >>= 1) {
+  #pragma unroll
+              for (int j = 0; j < w; ++j) {
+                // best three of two sorted triples
+                const float lo1 = fminf(a1[j], a1[j + w]), hi2 = fmaxf(a2[j], a2[j + w]);
+                a1[j] = fmaxf(a1[j], a1[j + w]);
+                a2[j] = fmaxf(lo1, hi2);
+                a3[j] = fmaxf(fminf(lo1, hi2), fmaxf(a3[j], a3[j + w]));
+              }
+            }
+            gscore_s[c * kTileM + row_in_tile] = a1[0];
+            gscore_s[(kBoundRows + c) * kTileM + row_in_tile] = a2[0];
+            gscore_s[(2 * kBoundRows + c) * kTileM + row_in_tile] = a3[0];
+          } else if (sigmoid_gate) {
+            int g = c0 / gs, pos = c0 % gs;
+  #pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (c0 + j < E) {
+                m2 = fmaxf(m2, fminf(m1, q[j]));
+                m1 = fmaxf(m1, q[j]);
+                if (++pos == gs) {                              // group complete (uniform branch)
+                  gscore_s[g * kTileM + row_in_tile] = gs >= 2 ? m1 + m2 : m1;
+                  glow_s[g * kTileM + row_in_tile] = gs >= 2 ? m2 : m1;
+                  ++g; pos = 0; m1 = -INFINITY; m2 = -INFINITY;
+                }
               }
             }
           }
         }
       }
-    }
-    FB_STAMP(3, 64);
-    tcgen05_fence_before();
-    // This warp has read its part of tensor memory: its share of the pair's closing barrier
-    // is delivered now, so that nobody waits for it at the end (see the teardown).
-    if (kCtas == 2) cluster_arrive();
-    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-    FB_STAMP(4, 64);
-    if (got && fast_select) {
-      // ---------------- choose: rank the (at most 8) group scores of this row
-      unsigned long long* cand = reinterpret_cast<unsigned long long*>(merge_v);   // [kCandCap][128], see rank_candidates
-      int my_groups[2] = {-1, -1};                        // the 32-column groups this sub scans
-      float floor_key = INFINITY;
-      if (sigmoid_gate) {
-        float sc[8];
-#pragma unroll
-        for (int g = 0; g < 8; ++g) sc[g] = g < p.n_group ? gscore_s[g * kTileM + row_in_tile] : -INFINITY;
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          int rank = 0;
-#pragma unroll
-          for (int h = 0; h < 8; ++h)          // a lower-numbered group wins ties
-            if (h != g) rank += (h < g ? sc[h] >= sc[g] : sc[h] > sc[g]) ? 1 : 0;
-          if (g < p.n_group && rank < p.topk_group) {
-            floor_key = fminf(floor_key, glow_s[g * kTileM + row_in_tile]);
-            if (rank == sub) my_groups[0] = g;   // sub s scans the row's s-th best group
-          }
-        }
-      } else {
-        // bound for the k-th key: the k-th largest of the chunks' three best keys (3 n_chunks >= k of them)
-        floor_key = kth_largest_known(gscore_s, n_chunks, k, row_in_tile);
-        if (sub < n_chunks) my_groups[0] = sub;
-        if (sub + kEpiSubs < n_chunks) my_groups[1] = sub + kEpiSubs;
-      }
-      FB_STAMP(5, 64);
-      // ---------------- collect the keys >= floor (at least k keys qualify: the bound is one of k known keys)
-#pragma unroll 1
-      for (int gi = 0; gi < 2; ++gi) {
-        if (my_groups[gi] < 0) continue;                  // no such group: true for the whole warp at once
-        const int base = my_groups[gi] * 32;              // (which group may differ from row to row)
-        uint32_t mask = 0;
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          mask |= (key_s[(base + j) * kTileM + row_in_tile] >= floor_key) ? (1u << j) : 0u;
-        const uint32_t mine = __popc(mask);
-        const uint32_t first = atomicAdd(&sh.cand_count[row_in_tile], mine);
-        const uint32_t most = __reduce_max_sync(0xffffffffu, mine);
-#pragma unroll 1
-        for (uint32_t i = 0; i < most; ++i) {
-          if (mask != 0 && first + i < kCandCap) {
-            const int j = __ffs(mask) - 1;
-            mask &= mask - 1;
-            cand[(first + i) * kTileM + row_in_tile] =
-                (static_cast<unsigned long long>(ordered_bits(key_s[(base + j) * kTileM + row_in_tile])) << 32) |
-                ~static_cast<uint32_t>(base + j);
-          }
-        }
-      }
-    }
-    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-    FB_STAMP(7, 64);
-    uint32_t* out_hi = reinterpret_cast<uint32_t*>(gscore_s);               // [8][128], group scores are dead now
-    uint32_t* out_lo = out_hi + FB_MAX_TOPK * kTileM;
-    bool overflow = false;
-    if (got && fast_select) {
-      overflow = rank_candidates(reinterpret_cast<const unsigned long long*>(merge_v), sh.cand_count[row_in_tile], sub,
-                                 row_in_tile, out_hi, out_lo);
-    }
-    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-    FB_STAMP(8, 64);
-    if (got && fast_select && sub == 0) {
-      if (!overflow) read_ranked(top, k, out_hi, out_lo, row_in_tile);
-      if (__any_sync(0xffffffffu, overflow)) {
-        // More than kCandCap keys reached the floor (many equal keys): plain scan of the
-        // kept groups for the rows concerned.
-        if (overflow && !sigmoid_gate) {
-          top.init();
-          for (int e = 0; e < E; ++e) {
-            const float x = key_s[e * kTileM + row_in_tile];
-            if (x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
-          }
-        } else if (overflow) {
+      FB_STAMP(3, 64);
+      tcgen05_fence_before();
+      // This warp has read its part of tensor memory: its share of the pair's closing barrier
+      // is delivered now, so that nobody waits for it at the end (see the teardown).
+      if (kCtas == 2) cluster_arrive();
+      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      FB_STAMP(4, 64);
+      if (got && fast_select) {
+        // ---------------- choose: rank the (at most 8) group scores of this row
+        unsigned long long* cand = reinterpret_cast<unsigned long long*>(merge_v);   // [kCandCap][128], see rank_candidates
+        int my_groups[2] = {-1, -1};                        // the 32-column groups this sub scans
+        float floor_key = INFINITY;
+        if (sigmoid_gate) {
           float sc[8];
-#pragma unroll
-          for (int g = 0; g < 8; ++g) sc[g] = -INFINITY;
-          // group scores were overwritten by the output area: recompute them from the keys
-          for (int g = 0; g < p.n_group; ++g) {
-            float a1 = -INFINITY, a2 = -INFINITY;
-            for (int j = 0; j < 32; ++j) {
-              const float x = key_s[(g * 32 + j) * kTileM + row_in_tile];
-              a2 = fmaxf(a2, fminf(a1, x));
-              a1 = fmaxf(a1, x);
-            }
-#pragma unroll
-            for (int h = 0; h < 8; ++h) if (h == g) sc[h] = a1 + a2;
-          }
-          top.init();
-#pragma unroll
+  #pragma unroll
+          for (int g = 0; g < 8; ++g) sc[g] = g < p.n_group ? gscore_s[g * kTileM + row_in_tile] : -INFINITY;
+  #pragma unroll
           for (int g = 0; g < 8; ++g) {
             int rank = 0;
-#pragma unroll
-            for (int h = 0; h < 8; ++h)
+  #pragma unroll
+            for (int h = 0; h < 8; ++h)          // a lower-numbered group wins ties
               if (h != g) rank += (h < g ? sc[h] >= sc[g] : sc[h] > sc[g]) ? 1 : 0;
             if (g < p.n_group && rank < p.topk_group) {
+              floor_key = fminf(floor_key, glow_s[g * kTileM + row_in_tile]);
+              if (rank == sub) my_groups[0] = g;   // sub s scans the row's s-th best group
+            }
+          }
+        } else {
+          // bound for the k-th key: the k-th largest of the chunks' three best keys (3 n_chunks >= k of them)
+          floor_key = kth_largest_known(gscore_s, n_chunks, k, row_in_tile);
+          if (sub < n_chunks) my_groups[0] = sub;
+          if (sub + kEpiSubs < n_chunks) my_groups[1] = sub + kEpiSubs;
+        }
+        FB_STAMP(5, 64);
+        // ---------------- collect the keys >= floor (at least k keys qualify: the bound is one of k known keys)
+  #pragma unroll 1
+        for (int gi = 0; gi < 2; ++gi) {
+          if (my_groups[gi] < 0) continue;                  // no such group: true for the whole warp at once
+          const int base = my_groups[gi] * 32;              // (which group may differ from row to row)
+          uint32_t mask = 0;
+  #pragma unroll
+          for (int j = 0; j < 32; ++j)
+            mask |= (key_s[(base + j) * kTileM + row_in_tile] >= floor_key) ? (1u << j) : 0u;
+          const uint32_t mine = __popc(mask);
+          const uint32_t first = atomicAdd(&sh.cand_count[row_in_tile], mine);
+          const uint32_t most = __reduce_max_sync(0xffffffffu, mine);
+  #pragma unroll 1
+          for (uint32_t i = 0; i < most; ++i) {
+            if (mask != 0 && first + i < kCandCap) {
+              const int j = __ffs(mask) - 1;
+              mask &= mask - 1;
+              cand[(first + i) * kTileM + row_in_tile] =
+                  (static_cast<unsigned long long>(ordered_bits(key_s[(base + j) * kTileM + row_in_tile])) << 32) |
+                  ~static_cast<uint32_t>(base + j);
+            }
+          }
+        }
+      }
+      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      FB_STAMP(7, 64);
+      uint32_t* out_hi = reinterpret_cast<uint32_t*>(gscore_s);               // [8][128], group scores are dead now
+      uint32_t* out_lo = out_hi + FB_MAX_TOPK * kTileM;
+      bool overflow = false;
+      if (got && fast_select) {
+        overflow = rank_candidates(reinterpret_cast<const unsigned long long*>(merge_v), sh.cand_count[row_in_tile], sub,
+                                   row_in_tile, out_hi, out_lo);
+      }
+      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      FB_STAMP(8, 64);
+      if (got && fast_select && sub == 0) {
+        if (!overflow) read_ranked(top, k, out_hi, out_lo, row_in_tile);
+        if (__any_sync(0xffffffffu, overflow)) {
+          // More than kCandCap keys reached the floor (many equal keys): plain scan of the
+          // kept groups for the rows concerned.
+          if (overflow && !sigmoid_gate) {
+            top.init();
+            for (int e = 0; e < E; ++e) {
+              const float x = key_s[e * kTileM + row_in_tile];
+              if (x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+            }
+          } else if (overflow) {
+            float sc[8];
+  #pragma unroll
+            for (int g = 0; g < 8; ++g) sc[g] = -INFINITY;
+            // group scores were overwritten by the output area: recompute them from the keys
+            for (int g = 0; g < p.n_group; ++g) {
+              float a1 = -INFINITY, a2 = -INFINITY;
               for (int j = 0; j < 32; ++j) {
                 const float x = key_s[(g * 32 + j) * kTileM + row_in_tile];
-                if (x > top.v[FB_MAX_TOPK - 1] || x == top.v[FB_MAX_TOPK - 1]) top.insert_any_order(x, g * 32 + j);
+                a2 = fmaxf(a2, fminf(a1, x));
+                a1 = fmaxf(a1, x);
+              }
+  #pragma unroll
+              for (int h = 0; h < 8; ++h) if (h == g) sc[h] = a1 + a2;
+            }
+            top.init();
+  #pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              int rank = 0;
+  #pragma unroll
+              for (int h = 0; h < 8; ++h)
+                if (h != g) rank += (h < g ? sc[h] >= sc[g] : sc[h] > sc[g]) ? 1 : 0;
+              if (g < p.n_group && rank < p.topk_group) {
+                for (int j = 0; j < 32; ++j) {
+                  const float x = key_s[(g * 32 + j) * kTileM + row_in_tile];
+                  if (x > top.v[FB_MAX_TOPK - 1] || x == top.v[FB_MAX_TOPK - 1]) top.insert_any_order(x, g * 32 + j);
+                }
               }
             }
           }
         }
       }
-    }
-    if (got && !fast_select) {
-      // ---------------- choose the groups; lower bound for the k-th key
-      uint32_t keep = 1u;
-      float floor_key = -INFINITY;
-      if (sigmoid_gate) {
-        TopK gtop;                                          // FB_MAX_TOPK >= topk_group
-        gtop.init();
-        for (int g = 0; g < p.n_group; ++g) {
-          const float sc = gscore_s[g * kTileM + row_in_tile];
-          if (sc > gtop.v[FB_MAX_TOPK - 1]) gtop.insert(sc, g);
-        }
-        keep = 0;
-        float low = INFINITY;
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j) {
-          if (j < p.topk_group) {
-            keep |= 1u << gtop.i[j];
-            low = fminf(low, glow_s[gtop.i[j] * kTileM + row_in_tile]);
+      if (got && !fast_select) {
+        // ---------------- choose the groups; lower bound for the k-th key
+        uint32_t keep = 1u;
+        float floor_key = -INFINITY;
+        if (sigmoid_gate) {
+          TopK gtop;                                          // FB_MAX_TOPK >= topk_group
+          gtop.init();
+          for (int g = 0; g < p.n_group; ++g) {
+            const float sc = gscore_s[g * kTileM + row_in_tile];
+            if (sc > gtop.v[FB_MAX_TOPK - 1]) gtop.insert(sc, g);
           }
-        }
-        // The kept groups' best (two) keys are eligible; if there are at least k of
-        // them, the smallest is a lower bound for the k-th largest eligible key.
-        if (p.topk_group * (gs >= 2 ? 2 : 1) >= k) floor_key = low;
-      }
-      // ---------------- pass 2
-      for (int c = 0; c < n_chunks; ++c) {
-        if (((owned_chunks >> c) & 1u) == 0) continue;
-        const int c0 = c * 32;
-        int g = sigmoid_gate ? c0 / gs : 0, pos = sigmoid_gate ? c0 % gs : 0;
-        const int g_start = g, pos_start = pos;
-        uint32_t cnt = 0;
-        unsigned long long packed = 0;                      // up to 8 column offsets, one byte each
-#pragma unroll 4
-        for (int j = 0; j < 32; ++j) {
-          const int e = c0 + j;
-          if (e < E) {
-            const float x = key_s[e * kTileM + row_in_tile];
-            if (((keep >> g) & 1u) && x >= floor_key && x > top.v[FB_MAX_TOPK - 1]) {
-              if (cnt < 8) packed |= static_cast<unsigned long long>(j) << (8 * cnt);
-              ++cnt;
+          keep = 0;
+          float low = INFINITY;
+  #pragma unroll
+          for (int j = 0; j < FB_MAX_TOPK; ++j) {
+            if (j < p.topk_group) {
+              keep |= 1u << gtop.i[j];
+              low = fminf(low, glow_s[gtop.i[j] * kTileM + row_in_tile]);
             }
-            if (++pos == gs) { ++g; pos = 0; }
           }
+          // The kept groups' best (two) keys are eligible; if there are at least k of
+          // them, the smallest is a lower bound for the k-th largest eligible key.
+          if (p.topk_group * (gs >= 2 ? 2 : 1) >= k) floor_key = low;
         }
-        const uint32_t most = __reduce_max_sync(0xffffffffu, cnt);
-        if (most > 8) {
-          // too many candidates for the packed list somewhere in the warp: plain scan
-          g = g_start; pos = pos_start;
-#pragma unroll 1
+        // ---------------- pass 2
+        for (int c = 0; c < n_chunks; ++c) {
+          if (((owned_chunks >> c) & 1u) == 0) continue;
+          const int c0 = c * 32;
+          int g = sigmoid_gate ? c0 / gs : 0, pos = sigmoid_gate ? c0 % gs : 0;
+          const int g_start = g, pos_start = pos;
+          uint32_t cnt = 0;
+          unsigned long long packed = 0;                      // up to 8 column offsets, one byte each
+  #pragma unroll 4
           for (int j = 0; j < 32; ++j) {
             const int e = c0 + j;
             if (e < E) {
               const float x = key_s[e * kTileM + row_in_tile];
-              if (((keep >> g) & 1u) && x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+              if (((keep >> g) & 1u) && x >= floor_key && x > top.v[FB_MAX_TOPK - 1]) {
+                if (cnt < 8) packed |= static_cast<unsigned long long>(j) << (8 * cnt);
+                ++cnt;
+              }
               if (++pos == gs) { ++g; pos = 0; }
             }
           }
+          const uint32_t most = __reduce_max_sync(0xffffffffu, cnt);
+          if (most > 8) {
+            // too many candidates for the packed list somewhere in the warp: plain scan
+            g = g_start; pos = pos_start;
+  #pragma unroll 1
+            for (int j = 0; j < 32; ++j) {
+              const int e = c0 + j;
+              if (e < E) {
+                const float x = key_s[e * kTileM + row_in_tile];
+                if (((keep >> g) & 1u) && x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+                if (++pos == gs) { ++g; pos = 0; }
+              }
+            }
+          } else {
+  #pragma unroll 1
+            for (uint32_t i = 0; i < most; ++i) {
+              if (i < cnt) {
+                const int e = c0 + static_cast<int>((packed >> (8 * i)) & 0xffu);
+                const float x = key_s[e * kTileM + row_in_tile];
+                if (x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+              }
+            }
+          }
+        }
+        // ---------------- hand the partial lists to sub 0
+        if (sub != 0) {
+  #pragma unroll
+          for (int j = 0; j < FB_MAX_TOPK; ++j) {
+            merge_v[((sub - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile] = top.v[j];
+            merge_i[((sub - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile] = top.i[j];
+          }
+        }
+        if (want_sum) {
+          part_s[(sub * 2 + 0) * kTileM + row_in_tile] = sm_max;
+          part_s[(sub * 2 + 1) * kTileM + row_in_tile] = sm_sum;
+        }
+      }
+      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      const bool writer = got && valid && sub == 0;
+      if (got && sub == 0 && !fast_select) {
+  #pragma unroll 1
+        for (int s2 = 1; s2 < kEpiSubs; ++s2) {
+  #pragma unroll 1
+          for (int j = 0; j < FB_MAX_TOPK; ++j) {
+            const float x = merge_v[((s2 - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile];
+            if (x > -INFINITY) top.insert_any_order(x, merge_i[((s2 - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile]);
+          }
+        }
+        if (want_sum) {
+          float mx = -INFINITY;
+          for (int s2 = 0; s2 < kEpiSubs; ++s2) mx = fmaxf(mx, part_s[(s2 * 2 + 0) * kTileM + row_in_tile]);
+          float sum = 0.0f;
+          for (int s2 = 0; s2 < kEpiSubs; ++s2)
+            sum += part_s[(s2 * 2 + 1) * kTileM + row_in_tile] * __expf(part_s[(s2 * 2 + 0) * kTileM + row_in_tile] - mx);
+          sm_max = mx; sm_sum = sum;
+        }
+      }
+
+      FB_STAMP(9, 64);
+      // ---- outputs per row
+      if (writer) write_row_outputs(top, p, row, out_ids, out_w, sh.select_bias, sm_max, sm_sum);
+      FB_STAMP(10, 64);
+      // ---- histogram: one shared-memory atomic per distinct expert per warp (Eq. 5)
+      if (sub == 0) {
+        if (E > 32) {
+          // many bins: lanes rarely collide, plain shared-memory atomics are cheapest
+  #pragma unroll
+          for (int j = 0; j < FB_MAX_TOPK; ++j)
+            if (j < k && writer) atomicAdd(&sh.hist[top.i[j]], 1u);
         } else {
-#pragma unroll 1
-          for (uint32_t i = 0; i < most; ++i) {
-            if (i < cnt) {
-              const int e = c0 + static_cast<int>((packed >> (8 * i)) & 0xffu);
-              const float x = key_s[e * kTileM + row_in_tile];
-              if (x > top.v[FB_MAX_TOPK - 1]) top.insert(x, e);
+          // few bins: add once per distinct expert per warp
+  #pragma unroll
+          for (int j = 0; j < FB_MAX_TOPK; ++j) {
+            if (j < k) {
+              const int e = writer ? top.i[j] : -1;
+              const uint32_t same = __match_any_sync(0xffffffffu, e);
+              if (e >= 0 && lane == __ffs(same) - 1) atomicAdd(&sh.hist[e], __popc(same));
             }
           }
         }
       }
-      // ---------------- hand the partial lists to sub 0
-      if (sub != 0) {
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j) {
-          merge_v[((sub - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile] = top.v[j];
-          merge_i[((sub - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile] = top.i[j];
-        }
-      }
-      if (want_sum) {
-        part_s[(sub * 2 + 0) * kTileM + row_in_tile] = sm_max;
-        part_s[(sub * 2 + 1) * kTileM + row_in_tile] = sm_sum;
-      }
-    }
-    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-    const bool writer = got && valid && sub == 0;
-    if (got && sub == 0 && !fast_select) {
-#pragma unroll 1
-      for (int s2 = 1; s2 < kEpiSubs; ++s2) {
-#pragma unroll 1
-        for (int j = 0; j < FB_MAX_TOPK; ++j) {
-          const float x = merge_v[((s2 - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile];
-          if (x > -INFINITY) top.insert_any_order(x, merge_i[((s2 - 1) * FB_MAX_TOPK + j) * kTileM + row_in_tile]);
-        }
-      }
-      if (want_sum) {
-        float mx = -INFINITY;
-        for (int s2 = 0; s2 < kEpiSubs; ++s2) mx = fmaxf(mx, part_s[(s2 * 2 + 0) * kTileM + row_in_tile]);
-        float sum = 0.0f;
-        for (int s2 = 0; s2 < kEpiSubs; ++s2)
-          sum += part_s[(s2 * 2 + 1) * kTileM + row_in_tile] * __expf(part_s[(s2 * 2 + 0) * kTileM + row_in_tile] - mx);
-        sm_max = mx; sm_sum = sum;
-      }
-    }
-
-    FB_STAMP(9, 64);
-    // ---- outputs per row
-    if (writer) write_row_outputs(top, p, row, out_ids, out_w, sh.select_bias, sm_max, sm_sum);
-    FB_STAMP(10, 64);
-    // ---- histogram: one shared-memory atomic per distinct expert per warp (Eq. 5)
-    if (sub == 0) {
-      if (E > 32) {
-        // many bins: lanes rarely collide, plain shared-memory atomics are cheapest
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j)
-          if (j < k && writer) atomicAdd(&sh.hist[top.i[j]], 1u);
+      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      if (mode == kModeDispatch) {
+        if (static_cast<long long>(tile) * kTileM < p.T)       // the padding block of an odd pair owns no tile
+          for (int e = et; e < E; e += kEpilogueThreads)
+            p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
       } else {
-        // few bins: add once per distinct expert per warp
-#pragma unroll
-        for (int j = 0; j < FB_MAX_TOPK; ++j) {
-          if (j < k) {
-            const int e = writer ? top.i[j] : -1;
-            const uint32_t same = __match_any_sync(0xffffffffu, e);
-            if (e >= 0 && lane == __ffs(same) - 1) atomicAdd(&sh.hist[e], __popc(same));
-          }
-        }
+        publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
       }
+      FB_STAMP(12, 64);
     }
-    named_bar_sync(kPlanBarrierId, kEpilogueThreads);
-    if (mode == kModeDispatch) {
-      if (static_cast<long long>(tile) * kTileM < p.T)       // the padding block of an odd pair owns no tile
-        for (int e = et; e < E; e += kEpilogueThreads)
-          p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
-    } else {
-      publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
-    }
-    FB_STAMP(12, 64);
   }
 
   // ---------------------------------------------------------------- teardown

@@ -12,6 +12,8 @@ Comparison rules
 * everything integer (counts, plan, placement, loads, dispatch index) is rechecked
   bit-exactly by feeding the GPU's own top-k to the oracle, and must additionally equal
   the oracle's own pipeline when no token differed.
+* the one-call layer step is checked the same way, on its own outputs (not against the
+  separate calls: the kernel variants differ in the order of their fp32 sums).
 """
 from __future__ import annotations
 
@@ -278,17 +280,30 @@ def compare_layer(wl: I.Workload, li: I.LayerInputs, bkw: dict, gpu: dict, place
     assert gpu["rank_load"].tolist() == rl.tolist()
     assert np.array_equal(gpu["perm"], perm), "perm differs"
     assert np.array_equal(gpu["inv_perm"], inv), "inv_perm differs"
-    # ---- the one-call layer step: the same kernels on the same inputs, so every output is
-    # bit-identical to the separate entry points (which the oracle has just checked)
+    # ---- the one-call layer step, checked on its own against the oracle.  Its router passes may
+    # run another kernel variant than the separate calls (persistent kernel, k-range split), whose
+    # fp32 sums are formed in another order: logits agree to rounding, so a token at a near tie
+    # may be routed differently by the two and everything downstream follows the call's own top-k.
     ly = gpu["layer"]
-    assert ly["counts"].tolist() == gpu["counts"].tolist(), "layer step: counts differ"
-    assert ly["swaps"] == swaps and ly["pi_out"] == pi_new, "layer step: plan differs"
-    assert ly["load_before"] == before and ly["load_after"] == after
-    assert np.array_equal(ly["ids"], gpu["ids"]), "layer step: top-k ids differ"
-    assert np.array_equal(ly["w"], gpu["w"]), "layer step: routing weights differ"
-    assert ly["slot_offsets"].tolist() == so.tolist() and ly["rank_offsets"].tolist() == ro.tolist()
-    assert ly["rank_load"].tolist() == rl.tolist()
-    assert np.array_equal(ly["perm"], perm) and np.array_equal(ly["inv_perm"], inv), "layer step: dispatch index"
+    T_all = li.h_prev.shape[0]
+    assert int(ly["counts"].sum()) == T_all * k
+    moved = int(np.abs(ly["counts"] - gpu["counts"]).sum()) // 2
+    if full:
+        assert moved <= k * report["early_flagged_tight"], "layer step: counts differ beyond the near-tie tokens"
+    report["layer_counts_moved"] = moved
+    l_swaps, l_pi, l_before, l_after = O.plan_swaps(ly["counts"].tolist(), pi0, R, bud)
+    assert ly["swaps"] == l_swaps and ly["pi_out"] == l_pi, "layer step: plan differs from the oracle's on its counts"
+    assert ly["load_before"] == l_before and ly["load_after"] == l_after
+    mism_l = compare_routing("layer", None, ly["ids"][rows], z, ids, gate, sb, report)
+    if T:
+        same = ~mism_l
+        wg = np.take_along_axis(ly["w"][rows], np.argsort(ly["ids"][rows], axis=1), axis=1)[same]
+        wr = np.take_along_axis(w, np.argsort(ids, axis=1), axis=1)[same]
+        assert (float(np.abs(wg - wr).max()) if wg.size else 0.0) <= WEIGHT_TOL, "layer step: routing weights"
+    l_so, l_ro, l_perm, l_inv, l_rl = O.dispatch_index(ly["ids"], l_pi, R)
+    assert ly["slot_offsets"].tolist() == l_so.tolist() and ly["rank_offsets"].tolist() == l_ro.tolist()
+    assert ly["rank_load"].tolist() == l_rl.tolist()
+    assert np.array_equal(ly["perm"], l_perm) and np.array_equal(ly["inv_perm"], l_inv), "layer step: dispatch index"
     realized = O.expert_histogram(gpu["ids"], E)
     report["real_max_over_mean_before"] = O.max_over_mean(O.rank_loads(realized, pi0, R))
     report["real_max_over_mean_after"] = O.max_over_mean(O.rank_loads(realized, pi_new, R))

@@ -50,8 +50,10 @@ def test_static_entry_matches_context_entry_twice(name, T):
     B.fb_predict_load_static(cfg, 0, router, x, T, got_counts, got_ids, status)
     torch.cuda.synchronize(dev)
     assert torch.cuda.mem_get_info(dev)[0] >= free_before
-    # the reference results, through a context
+    # the reference results, through a context running the same kernel (the static entry has no
+    # room for the partial tiles of the k-range split, so the context switches its split off)
     ctx = P.make_context(wl, T)
+    ctx.fb_set_split(0)
     for router, x, want_counts, want_ids, _, _, _ in prepared:
         ctx.fb_predict_load(router, x, T, want_counts, want_ids)
     assert ctx.fb_device_status() == 0
@@ -90,6 +92,7 @@ def test_static_entry_beside_contexts_of_other_shapes():
     dev = torch.device("cuda", 0)
     T = 600
     big = P.make_context(I.WORKLOADS["dsv3"], T)                       # alive throughout
+    big.fb_set_split(0)                                                # like with like: see the test above
     big_li = I.make_layer(I.WORKLOADS["dsv3"], 0, 0, T=T)
     big_router = B.make_router(big_li.W.to(dev), None, big_li.select_bias.to(dev))
     big_x = big_li.h_prev.to(dev)
@@ -102,6 +105,7 @@ def test_static_entry_beside_contexts_of_other_shapes():
         router = B.make_router(li.W.to(dev), None, li.select_bias.to(dev) if li.select_bias is not None else None)
         x = li.h_prev.to(dev)
         ctx = P.make_context(wl, T)
+        ctx.fb_set_split(0)
         want = torch.full((wl.E,), -1, dtype=torch.int32, device=dev)
         ctx.fb_predict_load(router, x, T, want)
         got = torch.full((wl.E,), -2, dtype=torch.int32, device=dev)

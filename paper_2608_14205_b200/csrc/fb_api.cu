@@ -272,6 +272,11 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.tile_counts = ctx->tile_counts;
   p.stamps = ctx->stamps;
   if (plan) p.plan = *plan;
+  // The fused tail serves the common plans; a plan that needs the general loop (per-expert sizes,
+  // more than 16 experts per rank, a planner variant) gets the stand-alone planner kernel behind
+  // the router kernel instead.
+  const bool plan_wanted = plan != nullptr && (mode == fb::kModePredictPlan || mode == fb::kModeLayer);
+  p.fuse_planner = (plan_wanted && !fb::plan_needs_general_loop(*plan)) ? 1 : 0;
   const int tiles_pad = pair ? (tiles + 1) / 2 * 2 : tiles;       // a pair never straddles the two passes
   int blocks = mode == fb::kModeLayer ? 2 * tiles_pad : tiles_pad;
   p.tiles_first = tiles_pad;
@@ -369,7 +374,13 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   ctx->ev_before = ctx->ev_after = nullptr;
   ++ctx->launches;
   if (persistent) ++ctx->persistent_launches;
-  return err == cudaSuccess ? FB_OK : FB_ERR_CUDA;
+  if (err != cudaSuccess) return FB_ERR_CUDA;
+  if (plan_wanted && !p.fuse_planner) {
+    fb::fb_plan_kernel<<<1, fb::kPlanThreads, 0, stream>>>(*plan, counts_out, ctx->status);
+    ++ctx->launches;
+    if (cudaGetLastError() != cudaSuccess) return FB_ERR_CUDA;
+  }
+  return FB_OK;
 }
 
 // Dispatch index from the router kernel's top-k ids and per-tile histograms.

@@ -338,77 +338,19 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
   return n;
 }
 
-// The planner, run by ONE warp (all 32 lanes) once plan_load_placement has filled the
-// placement arrays, sh.cnt holds the count vector and plan_scatter_counts has turned it into
-// counts per slot.  A single warp keeps the rank loads in registers (lane r holds ranks r and
-// r + 32) and needs no block barrier.  Writes the swaps, their number and the rank loads
-// before and after; the new placement is written afterwards by plan_write_placement.
-__device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh, int lane, int* status) {
+// Which plans the fast loop cannot serve (host and device agree on this test).
+__host__ __device__ inline bool plan_needs_general_loop(const PlanParams& p) {
+  return p.expert_bytes_table != nullptr || p.E / p.R > 16 || p.mode != FB_PLAN_LOOP;
+}
+
+// The general greedy loop: per-expert sizes, more than 16 experts per rank, or a planner
+// variant (the one-pass sweep of the ordering paragraph, a widened frontier).  Plain and slow;
+// a function of its own so that its registers and spills stay out of the common path.
+// L0 / L1: this lane's rank loads (ranks lane and lane + 32, -1 if absent).
+__device__ __noinline__ void plan_loop_general(const PlanParams& p, PlanShared& sh, int lane, long long L0,
+                                               long long L1) {
   const int E = p.E, R = p.R, m = E / R;
   const uint32_t full = 0xffffffffu;
-  __syncwarp();
-  FB_PLAN_STAMP(18);
-  // ---- rank loads (Algorithm 1 line 2), formed by plan_put_count: lane holds L[lane] and
-  // L[lane + 32]; their sum is checked against the planner's range
-  const unsigned long long s0 = lane < R ? sh.load[lane] : 0u, s1 = lane + 32 < R ? sh.load[lane + 32] : 0u;
-  const uint32_t total = __reduce_add_sync(full, static_cast<uint32_t>(s0 + s1));   // at most 256 counts of <= 2^21 each
-  int bad = sh.bad ? 1 : ((sh.bad_range || total > FB_MAX_COUNT_SUM) ? 2 : 0);
-  if (bad) {
-    // Unusable input: report it, keep the placement as given, empty plan.
-    if (lane == 0) {
-      atomicCAS(status, 0, bad == 1 ? FB_ERR_BAD_PLACEMENT : FB_ERR_RANGE);
-      *p.n_swaps = 0;
-      sh.bad_range = 1;                          // plan_write_placement copies the input placement
-    }
-    for (int r = lane; r < R; r += 32) { p.load_before[r] = 0; p.load_after[r] = 0; }
-    return;
-  }
-  long long L0 = -1, L1 = -1;                  // -1 marks "no such rank"
-  if (lane < R) {
-    L0 = static_cast<long long>(s0);
-    p.load_before[lane] = static_cast<uint32_t>(s0);
-    sh.rank_spent[lane] = 0;
-  }
-  if (lane + 32 < R) {
-    L1 = static_cast<long long>(s1);
-    p.load_before[lane + 32] = static_cast<uint32_t>(s1);
-    sh.rank_spent[lane + 32] = 0;
-  }
-  __syncwarp();
-  FB_PLAN_STAMP(19);
-
-  if (p.expert_bytes_table == nullptr && m <= 16 && p.mode == FB_PLAN_LOOP) {
-    int l0 = static_cast<int>(L0), l1 = static_cast<int>(L1);
-    const int mm = m * m;
-    // largest benefit any swap of this call can have (rank loads never exceed the initial maximum)
-    const unsigned long long lmax = __reduce_max_sync(full, static_cast<uint32_t>(s0 > s1 ? s0 : s1));
-    const unsigned long long bound = static_cast<unsigned long long>(p.gamma_den ? p.gamma_den : 1u) * lmax +
-                                     (p.gamma_den ? 2ull * p.gamma_num : 0ull) * ((lmax * lmax) >> 2);
-    const bool narrow = bound < (1ull << 32);
-    // can the per-rank or the per-link budget stop a swap that the global budget admits?
-    const bool side = (p.rank_ns != FB_BUDGET_OFF && !(p.global_ns != FB_BUDGET_OFF && p.rank_ns >= p.global_ns)) ||
-                      (p.link_ns != FB_BUDGET_OFF && !(p.global_ns != FB_BUDGET_OFF && p.link_ns >= p.global_ns));
-    uint32_t n_fast;
-    if (lane == 0) sh.fast = 1;
-    if (narrow && !side)
-      n_fast = mm <= 32 ? plan_loop_uniform<1, true, false>(p, sh, lane, l0, l1)
-               : mm <= 64 ? plan_loop_uniform<2, true, false>(p, sh, lane, l0, l1)
-               : mm <= 128 ? plan_loop_uniform<4, true, false>(p, sh, lane, l0, l1)
-                           : plan_loop_uniform<8, true, false>(p, sh, lane, l0, l1);
-    else if (narrow)
-      n_fast = mm <= 64 ? plan_loop_uniform<2, true, true>(p, sh, lane, l0, l1)
-                        : plan_loop_uniform<8, true, true>(p, sh, lane, l0, l1);
-    else
-      n_fast = mm <= 64 ? plan_loop_uniform<2, false, true>(p, sh, lane, l0, l1)
-                        : plan_loop_uniform<8, false, true>(p, sh, lane, l0, l1);
-    FB_PLAN_STAMP(20);
-    if (lane == 0) *p.n_swaps = static_cast<int32_t>(n_fast);
-    if (lane < R) p.load_after[lane] = static_cast<uint32_t>(l0);
-    if (lane + 32 < R) p.load_after[lane + 32] = static_cast<uint32_t>(l1);
-    return;
-  }
-  // ---- general loop: per-expert sizes, more than 16 experts per rank, or a planner variant
-  // (the one-pass sweep of the ordering paragraph, a widened frontier).  Plain and slow.
   const long long gnum = p.gamma_den ? p.gamma_num : 0;
   const long long gden = p.gamma_den ? p.gamma_den : 1;
   const int rpn = p.ranks_per_node;
@@ -549,5 +491,90 @@ __device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh
   if (lane < R) p.load_after[lane] = static_cast<uint32_t>(L0);
   if (lane + 32 < R) p.load_after[lane + 32] = static_cast<uint32_t>(L1);
 }
+
+// The planner, run by ONE warp (all 32 lanes) once plan_load_placement has filled the
+// placement arrays, sh.cnt holds the count vector and plan_scatter_counts has turned it into
+// counts per slot.  A single warp keeps the rank loads in registers (lane r holds ranks r and
+// r + 32) and needs no block barrier.  Writes the swaps, their number and the rank loads
+// before and after; the new placement is written afterwards by plan_write_placement.
+// kGeneral: the instance carries the general loop as well.  The router kernels' fused tail uses
+// the instance without it (the host launches the stand-alone planner kernel behind the router
+// kernel when a plan needs the general loop - see plan_needs_general_loop): the general loop's
+// registers and code would otherwise weigh on every router kernel.
+template <bool kGeneral>
+__device__ __noinline__ void plan_swaps_warp(const PlanParams& p, PlanShared& sh, int lane, int* status) {
+  const int E = p.E, R = p.R, m = E / R;
+  const uint32_t full = 0xffffffffu;
+  __syncwarp();
+  FB_PLAN_STAMP(18);
+  // ---- rank loads (Algorithm 1 line 2), formed by plan_put_count: lane holds L[lane] and
+  // L[lane + 32]; their sum is checked against the planner's range
+  const unsigned long long s0 = lane < R ? sh.load[lane] : 0u, s1 = lane + 32 < R ? sh.load[lane + 32] : 0u;
+  const uint32_t total = __reduce_add_sync(full, static_cast<uint32_t>(s0 + s1));   // at most 256 counts of <= 2^21 each
+  int bad = sh.bad ? 1 : ((sh.bad_range || total > FB_MAX_COUNT_SUM) ? 2 : 0);
+  if (bad) {
+    // Unusable input: report it, keep the placement as given, empty plan.
+    if (lane == 0) {
+      atomicCAS(status, 0, bad == 1 ? FB_ERR_BAD_PLACEMENT : FB_ERR_RANGE);
+      *p.n_swaps = 0;
+      sh.bad_range = 1;                          // plan_write_placement copies the input placement
+    }
+    for (int r = lane; r < R; r += 32) { p.load_before[r] = 0; p.load_after[r] = 0; }
+    return;
+  }
+  long long L0 = -1, L1 = -1;                  // -1 marks "no such rank"
+  if (lane < R) {
+    L0 = static_cast<long long>(s0);
+    p.load_before[lane] = static_cast<uint32_t>(s0);
+    sh.rank_spent[lane] = 0;
+  }
+  if (lane + 32 < R) {
+    L1 = static_cast<long long>(s1);
+    p.load_before[lane + 32] = static_cast<uint32_t>(s1);
+    sh.rank_spent[lane + 32] = 0;
+  }
+  __syncwarp();
+  FB_PLAN_STAMP(19);
+
+  if (!plan_needs_general_loop(p)) {
+    int l0 = static_cast<int>(L0), l1 = static_cast<int>(L1);
+    const int mm = m * m;
+    // largest benefit any swap of this call can have (rank loads never exceed the initial maximum)
+    const unsigned long long lmax = __reduce_max_sync(full, static_cast<uint32_t>(s0 > s1 ? s0 : s1));
+    const unsigned long long bound = static_cast<unsigned long long>(p.gamma_den ? p.gamma_den : 1u) * lmax +
+                                     (p.gamma_den ? 2ull * p.gamma_num : 0ull) * ((lmax * lmax) >> 2);
+    const bool narrow = bound < (1ull << 32);
+    // can the per-rank or the per-link budget stop a swap that the global budget admits?
+    const bool side = (p.rank_ns != FB_BUDGET_OFF && !(p.global_ns != FB_BUDGET_OFF && p.rank_ns >= p.global_ns)) ||
+                      (p.link_ns != FB_BUDGET_OFF && !(p.global_ns != FB_BUDGET_OFF && p.link_ns >= p.global_ns));
+    uint32_t n_fast;
+    if (lane == 0) sh.fast = 1;
+    if (narrow && !side)
+      n_fast = mm <= 32 ? plan_loop_uniform<1, true, false>(p, sh, lane, l0, l1)
+               : mm <= 64 ? plan_loop_uniform<2, true, false>(p, sh, lane, l0, l1)
+               : mm <= 128 ? plan_loop_uniform<4, true, false>(p, sh, lane, l0, l1)
+                           : plan_loop_uniform<8, true, false>(p, sh, lane, l0, l1);
+    else if (narrow)
+      n_fast = mm <= 64 ? plan_loop_uniform<2, true, true>(p, sh, lane, l0, l1)
+                        : plan_loop_uniform<8, true, true>(p, sh, lane, l0, l1);
+    else
+      n_fast = mm <= 64 ? plan_loop_uniform<2, false, true>(p, sh, lane, l0, l1)
+                        : plan_loop_uniform<8, false, true>(p, sh, lane, l0, l1);
+    FB_PLAN_STAMP(20);
+    if (lane == 0) *p.n_swaps = static_cast<int32_t>(n_fast);
+    if (lane < R) p.load_after[lane] = static_cast<uint32_t>(l0);
+    if (lane + 32 < R) p.load_after[lane + 32] = static_cast<uint32_t>(l1);
+    return;
+  }
+  if constexpr (kGeneral) {
+    plan_loop_general(p, sh, lane, L0, L1);
+  } else {
+    // not reachable when the host follows plan_needs_general_loop; an empty plan otherwise
+    if (lane == 0) *p.n_swaps = 0;
+    if (lane < R) p.load_after[lane] = static_cast<uint32_t>(L0);
+    if (lane + 32 < R) p.load_after[lane + 32] = static_cast<uint32_t>(L1);
+  }
+}
+
 
 }  // namespace fb

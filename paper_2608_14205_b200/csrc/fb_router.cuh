@@ -86,6 +86,7 @@ struct RouterParams {
   int32_t mode;
   int32_t tiles_first;               // kModeLayer: blocks below this index (even) belong to the early pass
   int32_t ticket_target;             // number of blocks that take a ticket (those that publish counts)
+  int32_t fuse_planner;              // prediction modes: the block that finishes last runs the planner
   const float* logit_bias;           // [E] or nullptr
   const float* select_bias;          // [E] or nullptr
   uint32_t* counts_scratch;          // [E] zero on entry, zero again on exit
@@ -373,9 +374,9 @@ __device__ __forceinline__ void publish_counts(Shared& sh, const RouterParams& p
 #ifdef FB_TIMING
         PlanParams pt = p.plan;
         pt.stamps = p.stamps != nullptr ? p.stamps + static_cast<size_t>(blockIdx.x) * 64 : nullptr;
-        plan_swaps_warp(pt, sh.plan, lane, p.status);
+        plan_swaps_warp<false>(pt, sh.plan, lane, p.status);
 #else
-        plan_swaps_warp(p.plan, sh.plan, lane, p.status);
+        plan_swaps_warp<false>(p.plan, sh.plan, lane, p.status);
 #endif
       }
       named_bar_sync(kPlanBarrierId, kEpilogueThreads);
@@ -1115,7 +1116,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           for (int e = et; e < E; e += kEpilogueThreads)
             p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
       } else {
-        publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
+        publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan && p.fuse_planner != 0);
       }
       FB_STAMP(12, 64);
     }
@@ -1166,7 +1167,7 @@ fb_plan_kernel(const __grid_constant__ PlanParams p, const uint32_t* __restrict_
   plan_load_placement(p, sh, t, kPlanThreads);
   __syncwarp();
   for (int e = t; e < p.E; e += kPlanThreads) plan_put_count(sh, e, counts[e]);
-  plan_swaps_warp(p, sh, t, status);
+  plan_swaps_warp<true>(p, sh, t, status);
   __syncwarp();
   plan_write_placement(p, sh, t, kPlanThreads);
 }

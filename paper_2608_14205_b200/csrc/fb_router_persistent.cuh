@@ -450,7 +450,7 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
       } else if (pt + pair_stride >= pairs_per_pass) {
         // The histogram keeps accumulating over this block's tiles of the pass and is published
         // once, after the last of them (one fence and one ticket per block, not per tile).
-        publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan);
+        publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan && p.fuse_planner != 0);
       }
     }
   }

@@ -418,7 +418,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     ap.add_argument("--no-probe", action="store_true",
-                    help="skip the per-kernel timing passes after the bracketed region (for profiler captures)")
+                    help="skip the per-kernel timing passes after the bracketed region and the in-kernel clock "
+                         "probe (for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -523,13 +524,15 @@ def main():
     barrier()
     sampler.start()
     sampler.window[0] = time.perf_counter()
-    B.fb_clock_probe(probe, probe_n, probe_period_ns, stream=side)
-    B.fb_clock_probe(marks[0:2], 1, 0)
+    if not args.no_probe:                    # (under a profiler the probe kernel would be serialised with the steps)
+        B.fb_clock_probe(probe, probe_n, probe_period_ns, stream=side)
+        B.fb_clock_probe(marks[0:2], 1, 0)
     ev_begin.record()
     for i in range(K):
         step(layers[i % ring])
     ev_end.record()
-    B.fb_clock_probe(marks[2:4], 1, 0)
+    if not args.no_probe:
+        B.fb_clock_probe(marks[2:4], 1, 0)
     barrier()
     sampler.window[1] = time.perf_counter()
     launches = ctx.fb_launch_count() - launches0

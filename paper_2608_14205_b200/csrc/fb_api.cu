@@ -1151,6 +1151,16 @@ fb_status fb_clock_probe(uint64_t* samples, int32_t n, uint32_t period_ns, fb_st
   if (device < 0) return FB_ERR_INVALID_ARG;
   DeviceGuard guard(device);
   if (!guard.ok) return FB_ERR_CUDA;
+  // The split between L1 and shared memory is a per-SM setting that only changes while the SM is
+  // idle: a resident block of a kernel that prefers a small shared-memory share would keep the
+  // router kernel's blocks (over 200 KB of shared memory each) off its SM for as long as it runs.
+  static bool carveout_set[64] = {};
+  if (device < 64 && !carveout_set[device]) {
+    if (cudaFuncSetAttribute(reinterpret_cast<const void*>(fb::fb_clock_probe_kernel),
+                             cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+      return FB_ERR_CUDA;
+    carveout_set[device] = true;
+  }
   fb::fb_clock_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream_)>>>(
       reinterpret_cast<unsigned long long*>(samples), n, period_ns);
   return cudaGetLastError() == cudaSuccess ? FB_OK : FB_ERR_CUDA;

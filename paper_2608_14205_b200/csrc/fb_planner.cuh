@@ -254,45 +254,64 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
       stop = stop || used >= (cls ? link_cap1 : link_cap0);
     }
     // ---- candidates of this lane: largest benefit, ties -> smallest (expert on a, expert on b)
-    unsigned long long best_ben = 0;
-    uint32_t best_pair = 0xffffffffu, best_slots = 0, best_wa = 0, best_wb = 0;
+    int src, ea, eb, sa, sb;
+    uint32_t wwa, wwb;                                            // slot words of the accepted pair
+    if (k32) {
+      // One 64-bit key per candidate: benefit, then the complement of the pair (so that the
+      // larger key is the better candidate), then the candidate's index in this lane.  The
+      // candidates of a lane are independent of each other; only the maximum chains them.
+      unsigned long long best_key = 0;
 #pragma unroll
-    for (int t = 0; t < kPerLane; ++t) {
-      const int dlt = static_cast<int>(wa[t] & kSlotCountMask) - static_cast<int>(wb[t] & kSlotCountMask);   // tokens moved a -> b
-      int Mn = La - dlt;                                          // Eq. 6
-      if (Lb + dlt > Mn) Mn = Lb + dlt;                           // Eq. 7
-      if (M2 > Mn) Mn = M2;
-      // gamma_den * (Phi(L) - Phi(L')), variance term 2 dlt (La - Lb - dlt).  It is positive only
-      // for 0 < dlt < D, and inside that range both terms are non-negative.
-      const bool usable = cand_ok[t] && ((wa[t] | wb[t]) >> 31) == 0 && dlt > 0 && dlt < D;   // neither expert moved yet
-      unsigned long long ub;
-      if (k32) {
+      for (int t = 0; t < kPerLane; ++t) {
+        const int dlt = static_cast<int>(wa[t] & kSlotCountMask) - static_cast<int>(wb[t] & kSlotCountMask);   // tokens moved a -> b
+        int Mn = La - dlt;                                        // Eq. 6
+        if (Lb + dlt > Mn) Mn = Lb + dlt;                         // Eq. 7
+        if (M2 > Mn) Mn = M2;
+        // gamma_den * (Phi(L) - Phi(L')), variance term 2 dlt (La - Lb - dlt).  It is positive only
+        // for 0 < dlt < D, and inside that range both terms are non-negative.
+        const bool usable = cand_ok[t] && ((wa[t] | wb[t]) >> 31) == 0 && dlt > 0 && dlt < D;   // neither expert moved yet
         const uint32_t b32 = gden * static_cast<uint32_t>(La - Mn) +
                              gnum2 * (static_cast<uint32_t>(dlt) * static_cast<uint32_t>(D - dlt));
-        ub = usable ? b32 : 0u;
-      } else {
-        const long long ben = static_cast<long long>(gden) * (La - Mn) +
-                              static_cast<long long>(gnum2) * (static_cast<long long>(dlt) * (D - dlt));
-        ub = usable ? static_cast<unsigned long long>(ben) : 0ull;
+        const uint32_t pair = ((wa[t] >> 22) & 0xffu) << 8 | ((wb[t] >> 22) & 0xffu);
+        const unsigned long long key = static_cast<unsigned long long>(usable ? b32 : 0u) << 32 |
+                                       static_cast<unsigned long long>(0xffffu - pair) << 8 | static_cast<unsigned>(t);
+        best_key = key > best_key ? key : best_key;
       }
-      const uint32_t pair = ((wa[t] >> 22) & 0xffu) << 16 | ((wb[t] >> 22) & 0xffu);
-      if (ub > best_ben || (ub == best_ben && ub > 0 && pair < best_pair)) {
-        best_ben = ub; best_pair = pair; best_wa = wa[t]; best_wb = wb[t];
-        best_slots = static_cast<uint32_t>(base_a + cand_sa[t]) << 16 | static_cast<uint32_t>(base_b + cand_sb[t]);
-      }
-    }
-    int src, ea, eb;
-    if (k32) {
-      const uint32_t mine = static_cast<uint32_t>(best_ben);
+      const uint32_t mine = static_cast<uint32_t>(best_key >> 32);
       const uint32_t top = __reduce_max_sync(full, mine);
       if (stop || top == 0) break;                                // Algorithm 1 lines 6-7
-      // expert ids are below 256: (expert on a, expert on b, lane) packs into 21 bits
-      const uint32_t tag = (best_pair >> 16) << 13 | (best_pair & 0xffu) << 5 | static_cast<uint32_t>(lane);
-      const uint32_t win = __reduce_min_sync(full, mine == top ? tag : 0xffffffffu);
-      src = static_cast<int>(win & 31u);
-      ea = static_cast<int>(win >> 13);
-      eb = static_cast<int>((win >> 5) & 0xffu);
+      // among the lanes that hold the top benefit: smallest pair, i.e. largest complement; the lane rides along
+      const uint32_t low = static_cast<uint32_t>(best_key);      // complement of the pair << 8 | index
+      const uint32_t win = __reduce_max_sync(full, mine == top ? ((low >> 8) << 5 | static_cast<uint32_t>(31 - lane)) : 0u);
+      src = 31 - static_cast<int>(win & 31u);
+      const uint32_t pair = 0xffffu - (win >> 5);
+      ea = static_cast<int>(pair >> 8);
+      eb = static_cast<int>(pair & 0xffu);
+      // the winning lane's candidate index gives the slots; their words come from shared memory
+      const int t_win = __shfl_sync(full, static_cast<int>(low & 0xffu), src);
+      sa = base_a + sh.cand_a[src + 32 * t_win];
+      sb = base_b + sh.cand_b[src + 32 * t_win];
+      wwa = sh.slot_cnt[sa];
+      wwb = sh.slot_cnt[sb];
     } else {
+      unsigned long long best_ben = 0;
+      uint32_t best_pair = 0xffffffffu, best_slots = 0, best_wa = 0, best_wb = 0;
+#pragma unroll
+      for (int t = 0; t < kPerLane; ++t) {
+        const int dlt = static_cast<int>(wa[t] & kSlotCountMask) - static_cast<int>(wb[t] & kSlotCountMask);
+        int Mn = La - dlt;
+        if (Lb + dlt > Mn) Mn = Lb + dlt;
+        if (M2 > Mn) Mn = M2;
+        const bool usable = cand_ok[t] && ((wa[t] | wb[t]) >> 31) == 0 && dlt > 0 && dlt < D;
+        const long long ben = static_cast<long long>(gden) * (La - Mn) +
+                              static_cast<long long>(gnum2) * (static_cast<long long>(dlt) * (D - dlt));
+        const unsigned long long ub = usable ? static_cast<unsigned long long>(ben) : 0ull;
+        const uint32_t pair = ((wa[t] >> 22) & 0xffu) << 16 | ((wb[t] >> 22) & 0xffu);
+        if (ub > best_ben || (ub == best_ben && ub > 0 && pair < best_pair)) {
+          best_ben = ub; best_pair = pair; best_wa = wa[t]; best_wb = wb[t];
+          best_slots = static_cast<uint32_t>(base_a + cand_sa[t]) << 16 | static_cast<uint32_t>(base_b + cand_sb[t]);
+        }
+      }
       const uint32_t top_hi = __reduce_max_sync(full, static_cast<uint32_t>(best_ben >> 32));
       const uint32_t top_lo = __reduce_max_sync(full, static_cast<uint32_t>(best_ben >> 32) == top_hi ? static_cast<uint32_t>(best_ben) : 0u);
       const unsigned long long top_ben = static_cast<unsigned long long>(top_hi) << 32 | top_lo;
@@ -301,11 +320,13 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
       src = __ffs(__ballot_sync(full, best_ben == top_ben && best_pair == win)) - 1;
       ea = static_cast<int>(win >> 16);
       eb = static_cast<int>(win & 0xffffu);
+      // the lane that holds the accepted pair hands out its slots and slot words
+      const uint32_t slots = __shfl_sync(full, best_slots, src);
+      wwa = __shfl_sync(full, best_wa, src);
+      wwb = __shfl_sync(full, best_wb, src);
+      sa = static_cast<int>(slots >> 16);
+      sb = static_cast<int>(slots & 0xffffu);
     }
-    // the lane that holds the accepted pair hands out its slots and slot words
-    const uint32_t slots = __shfl_sync(full, best_slots, src);
-    const uint32_t wwa = __shfl_sync(full, best_wa, src), wwb = __shfl_sync(full, best_wb, src);
-    const int sa = static_cast<int>(slots >> 16), sb = static_cast<int>(slots & 0xffffu);
     const int dlt = static_cast<int>(wwa & kSlotCountMask) - static_cast<int>(wwb & kSlotCountMask);
     if (lane == 0) {
       sh.slot_cnt[sa] = wwb | kSlotMoved; sh.slot_cnt[sb] = wwa | kSlotMoved;   // the two experts trade slots

@@ -112,10 +112,11 @@ def main(argv=None):
     skew_start = (ns_t[:, :, 0].max(axis=1) - start[:, 0]) / 1e3
     ends = ns_t[:, :, 13]
     skew_end = (end - np.where(ends > 0, ends, np.inf).min(axis=1)) / 1e3
-    main_cyc = cyc[sel, :, 2] - cyc[sel, :, 1]
-    main_ns = ns_t[sel, :, 2] - ns_t[sel, :, 1]
-    epi_cyc = cyc[sel, :, 11] - cyc[sel, :, 2]
-    epi_ns = ns_t[sel, :, 11] - ns_t[sel, :, 2]
+    own = (ns_t[sel, :, 2] > 0) & (ns_t[sel, :, 11] > 0)          # blocks that own a tile (helper pairs have no epilogue)
+    main_cyc = (cyc[sel, :, 2] - cyc[sel, :, 1])[own]
+    main_ns = (ns_t[sel, :, 2] - ns_t[sel, :, 1])[own]
+    epi_cyc = (cyc[sel, :, 11] - cyc[sel, :, 2])[own]
+    epi_ns = (ns_t[sel, :, 11] - ns_t[sel, :, 2])[own]
     out.update(span_us=float(span[sel].mean()), gap_us=float(gap.mean()), start_skew_us=float(skew_start[sel].mean()),
                end_skew_us=float(skew_end[sel].mean()), main_loop_ghz=float(main_cyc.mean() / main_ns.mean()),
                epilogue_ghz=float(epi_cyc.mean() / epi_ns.mean()), main_loop_cycles=float(main_cyc.mean()))

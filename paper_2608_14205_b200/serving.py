@@ -15,6 +15,7 @@ prints one JSON report per run (synthetic changing-task steps, see inputs.make_s
 from __future__ import annotations
 
 import argparse
+import copy
 import json
 from typing import Dict, Optional
 
@@ -103,23 +104,29 @@ class ServingLoop:
         self.placement[layer], self._spare = pi_new, pi
         return dict(out=o, pi_old=pi, pi_new=pi_new, **report)
 
+    def realised_loads(self, r: dict, budget: B.FbBudget):
+        """Realised per-expert counts of the last layer step and the rank loads they give under the
+        old, the new and the identity placement - all from the library: per-slot counts of the
+        dispatch index, `rank_load` of the step, and the planner's own rank-load aggregation
+        (fb_plan_swaps with no swap allowed) for the other two placements."""
+        ctx, o, E, R = self.ctx, self.out, self.wl.E, self.wl.R
+        i32 = lambda n: torch.zeros(max(1, n), dtype=torch.int32, device=self.dev)
+        slot_counts, before, vanilla, scratch = i32(E), i32(R), i32(R), i32(R)
+        ctx.fb_dispatch_slot_counts(o["slot_offsets"], slot_counts)
+        realised = slot_counts[r["pi_new"].long()].contiguous()          # per expert: the count of its slot
+        none = copy.copy(budget)
+        none.max_swaps = 0
+        identity = torch.arange(E, dtype=torch.int32, device=self.dev)
+        ctx.fb_plan_swaps(realised, r["pi_old"], none, 0, i32(E), None, i32(1), before, scratch)
+        ctx.fb_plan_swaps(realised, identity, none, 0, i32(E), None, i32(1), vanilla, scratch)
+        torch.cuda.synchronize(self.dev)
+        return (realised.cpu().tolist(), before.cpu().tolist(), o["rank_load"].cpu().tolist(),
+                vanilla.cpu().tolist())
 
-def realized_loads(slot_offsets, pi_old, pi_new, R: int):
-    """Host-side bookkeeping for the report: realised rank loads under two placements."""
-    so = slot_offsets.cpu().tolist()
-    new, old = pi_new.cpu().tolist(), pi_old.cpu().tolist()
-    E = len(new)
-    m = E // R
-    realized = [so[new[e] + 1] - so[new[e]] for e in range(E)]
-    def loads(pi):
-        L = [0] * R
-        for e in range(E):
-            L[pi[e] // m] += realized[e]
-        return L
-    return realized, loads(old), loads(new), loads(list(range(E)))
 
-
-def _max_over_mean(L):
+def max_over_mean(loads) -> float:
+    """Report formatting: the imbalance ratio of a rank-load vector the library returned."""
+    L = [int(v) for v in loads]
     s = sum(L)
     return max(L) * len(L) / s if s else 1.0
 
@@ -147,11 +154,11 @@ def main():
             router = B.make_router(li.W.to(dev), None, sb)
             r = loop.layer_step(l, router, li.h_prev.to(dev), li.H.to(dev), budget, quality=True)
             torch.cuda.synchronize(dev)
-            _, before, after, vanilla = realized_loads(r["out"]["slot_offsets"], r["pi_old"], r["pi_new"], wl.R)
+            _, before, after, vanilla = loop.realised_loads(r, budget)
             recs.append(dict(step=s, layer=l, n_swaps=int(r["out"]["n_swaps"].item()), hit_rate=r["hit_rate"],
                              cos_hidden=r["cos_hidden"], cos_logits=r["cos_logits"],
-                             real_vanilla=_max_over_mean(vanilla), real_before=_max_over_mean(before),
-                             real_after=_max_over_mean(after)))
+                             real_vanilla=max_over_mean(vanilla), real_before=max_over_mean(before),
+                             real_after=max_over_mean(after)))
     moved = [r for r in recs if r["n_swaps"] > 0]
     n = max(1, len(recs))
     print(json.dumps(dict(

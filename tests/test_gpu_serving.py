@@ -43,7 +43,7 @@ def test_serving_loop_matches_the_oracle(name, T, steps, layers, sys_drift, qual
         swaps = [tuple(x) for x in o["swaps"].cpu().numpy().reshape(-1, 4)[:n].tolist()]
         assert o["counts"].cpu().tolist() == rec["counts"].tolist()
         assert swaps == rec["swaps"] and r["pi_new"].cpu().tolist() == rec["pi_new"]
-        realized, before, after, vanilla = S.realized_loads(o["slot_offsets"], r["pi_old"], r["pi_new"], wl.R)
+        realized, before, after, vanilla = loop.realised_loads(r, budget)
         assert realized == rec["realized"].tolist()
         assert O.max_over_mean(before) == rec["real_before"] and O.max_over_mean(after) == rec["real_after"]
         assert O.max_over_mean(vanilla) == rec["real_vanilla"]

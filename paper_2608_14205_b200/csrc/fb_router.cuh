@@ -66,6 +66,7 @@ constexpr int kRouterThreads = 64 + kEpilogueThreads + 32;
 constexpr int kSecondIssuerWarp = kRouterThreads / 32 - 1;
 constexpr int kATileBytes = kTileM * kBlockK * 2;
 constexpr uint32_t kAccumBarrierId = 2;      // named barrier: accumulator finished (MMA warp -> epilogue warps)
+constexpr uint32_t kRowBarrierBase = 3;      // named barriers 3..6: the kEpiSubs warps that share one quarter of the rows
 
 enum RouterMode : int {
   kModePredict = 0,        // histogram -> counts
@@ -723,18 +724,38 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       int32_t* merge_i = reinterpret_cast<int32_t*>(merge_v + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);
       float* part_s = reinterpret_cast<float*>(merge_i + (kEpiSubs - 1) * FB_MAX_TOPK * kTileM);   // [subs][2][128]
 
+      // Between pass 1 and the histogram, data passes only between the kEpiSubs warps that share
+      // this warp's rows: they meet at a barrier of their own and do not wait for the other rows' warps.
+      auto row_sync = [&]() { named_bar_sync(kRowBarrierBase + static_cast<uint32_t>(quarter), kEpiSubs * 32); };
+
       TopK top;
       top.init();
       float sm_max = -INFINITY, sm_sum = 0.0f;               // softmax denominator (weights without renorm)
       constexpr bool has_lb = kLogitBias;
       if (got) {
         // ---------------- pass 1
+        // On the ranking paths E is a multiple of 32 (N == E: every chunk is full) and sub s owns
+        // chunks s, s + kEpiSubs, ...; with the DeepSeek-V3-like gate a chunk is exactly one group.
+        constexpr bool kFullChunks = kSel != kSelectGeneral;
+        constexpr bool kChunkIsGroup = kSel == kSelectSigmoidRank;
         float m1 = -INFINITY, m2 = -INFINITY;
-        for (int c = 0; c < n_chunks; ++c) {
-          if (((owned_chunks >> c) & 1u) == 0) continue;
+#pragma unroll 1
+        for (int c = kFullChunks ? sub : 0; c < n_chunks; c += kFullChunks ? kEpiSubs : 1) {
+          if (!kFullChunks && ((owned_chunks >> c) & 1u) == 0) continue;
           const int c0 = c * 32;
           uint32_t r[32];
           float q[32];
+          if (kFullChunks) {
+            // both accumulators' loads in flight at once, one wait
+            uint32_t r2[32];
+            tmem_ld_32x32b_x32(taddr + c0, r);
+            if (kb_end > 1) tmem_ld_32x32b_x32(taddr + N + c0, r2);
+            tmem_ld_wait();
+            if (kb_end > 1) {
+  #pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+            }
+          } else {
           load_chunk(taddr, c0, N, r);
           if (kb_end > 1) {                                    // add the odd k-blocks' accumulator
             const int halves = (N - c0 >= 32) ? 2 : 1;         // 16 columns at a time keeps registers low
@@ -750,6 +771,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 for (int j = 0; j < 16; ++j) r[16 + j] = __float_as_uint(__uint_as_float(r[16 + j]) + __uint_as_float(r2[j]));
               }
             }
+          }
           }
           if (kSplit) {
             // add the helpers' partial sums of the remaining k-blocks, piece by piece in a fixed order;
@@ -773,7 +795,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
               if (c0 + j < E)
                 p.logits[row * E + c0 + j] = __uint_as_float(r[j]) + (has_lb ? sh.logit_bias[c0 + j] : 0.0f);
           }
-          if (sigmoid_gate && c0 + 32 <= E && !has_lb) {
+          if (sigmoid_gate && (kFullChunks || c0 + 32 <= E) && !has_lb) {
             // whole chunk valid, no logit bias (the common case).  Every key goes through the
             // same two hardware approximations, so equal logits give equal keys in every column
             // (an FMA-pipe reciprocal on alternate columns was no faster and broke exact ties).
@@ -799,9 +821,12 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
               q[j] = (c0 + j < E) ? z : -INFINITY;
             }
           }
+          {
+            float* kcol = key_s + c0 * kTileM + row_in_tile;
   #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c0 + j < N) key_s[(c0 + j) * kTileM + row_in_tile] = q[j];
+            for (int j = 0; j < 32; ++j)
+              if (kFullChunks || c0 + j < N) kcol[j * kTileM] = q[j];
+          }
           if (want_sum) {
             float cmax = q[0];
   #pragma unroll
@@ -826,6 +851,11 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 a2[j] = fmaxf(fminf(a1[j], a1[j + w]), fmaxf(a2[j], a2[j + w]));
                 a1[j] = hi;
               }
+            }
+            if (kChunkIsGroup) {
+              gscore_s[c * kTileM + row_in_tile] = a1[0] + a2[0];
+              glow_s[c * kTileM + row_in_tile] = a2[0];
+              continue;
             }
             m2 = fmaxf(fminf(m1, a1[0]), fmaxf(m2, a2[0]));
             m1 = fmaxf(m1, a1[0]);
@@ -878,7 +908,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       // This warp has read its part of tensor memory: its share of the pair's closing barrier
       // is delivered now, so that nobody waits for it at the end (see the teardown).
       if (kCtas == 2) cluster_arrive();
-      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      row_sync();
       FB_STAMP(4, 64);
       if (got && fast_select) {
         // ---------------- choose: rank the (at most 8) group scores of this row
@@ -931,7 +961,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           }
         }
       }
-      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      row_sync();
       FB_STAMP(7, 64);
       uint32_t* out_hi = reinterpret_cast<uint32_t*>(gscore_s);               // [8][128], group scores are dead now
       uint32_t* out_lo = out_hi + FB_MAX_TOPK * kTileM;
@@ -940,7 +970,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         overflow = rank_candidates(reinterpret_cast<const unsigned long long*>(merge_v), sh.cand_count[row_in_tile], sub,
                                    row_in_tile, out_hi, out_lo);
       }
-      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      row_sync();
       FB_STAMP(8, 64);
       if (got && fast_select && sub == 0) {
         if (!overflow) read_ranked(top, k, out_hi, out_lo, row_in_tile);
@@ -1066,7 +1096,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           part_s[(sub * 2 + 1) * kTileM + row_in_tile] = sm_sum;
         }
       }
-      named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      row_sync();
       const bool writer = got && valid && sub == 0;
       if (got && sub == 0 && !fast_select) {
   #pragma unroll 1

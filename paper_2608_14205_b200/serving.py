@@ -15,7 +15,6 @@ prints one JSON report per run (synthetic changing-task steps, see inputs.make_s
 from __future__ import annotations
 
 import argparse
-import copy
 import json
 from typing import Dict, Optional
 
@@ -114,7 +113,7 @@ class ServingLoop:
         slot_counts, before, vanilla, scratch = i32(E), i32(R), i32(R), i32(R)
         ctx.fb_dispatch_slot_counts(o["slot_offsets"], slot_counts)
         realised = slot_counts[r["pi_new"].long()].contiguous()          # per expert: the count of its slot
-        none = copy.copy(budget)
+        none = type(budget).from_buffer_copy(budget)     # same fields (and the same table pointer, kept alive by `budget`)
         none.max_swaps = 0
         identity = torch.arange(E, dtype=torch.int32, device=self.dev)
         ctx.fb_plan_swaps(realised, r["pi_old"], none, 0, i32(E), None, i32(1), before, scratch)

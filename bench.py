@@ -571,6 +571,23 @@ def main():
         b.record()
         barrier()
         pp_b2b.append(a.elapsed_time(b) / pp_n)
+    # the same launch cut down to its main loop (operands loaded only / loaded and multiplied; nothing after
+    # it): what launch, set-up and the operand stream cost by themselves with this tiling
+    floor_us = {}
+    one_tile_launch = (T + 127) // 128 // 2 <= ctx.fb_max_pairs()       # else the call uses the persistent kernel
+    if pp_n and one_tile_launch:
+        for what, name in ((1, "loads_only_us"), (2, "loads_and_mma_us")):
+            reps = []
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for i in range(pp_n):
+                    L = layers[i % ring]
+                    ctx.fb_router_floor(L["router"], L["h_prev"], T, what)
+                b.record()
+                barrier()
+                reps.append(a.elapsed_time(b) / pp_n * 1e3)
+            floor_us[name] = statistics.median(reps)
     pp_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(pp_n)]
     for i in range(pp_n):
         pp_ev[i][0].record()
@@ -722,6 +739,9 @@ def main():
                                                  note="one event pair per launch: includes launch latency and "
                                                       "event granularity that back-to-back launches hide")
             attach_traffic(roof_pp, wl.name)
+            if floor_us:
+                roof_pp["main_loop_floor"] = dict(floor_us, how="fb_router_floor: the same launch without MMAs / with "
+                                                  "them, and nothing after the main loop; timed like kernel_us")
 
         lb, la = out["load_before"].cpu().tolist(), out["load_after"].cpu().tolist()
         real_b, real_a = real_before.cpu().tolist(), out["rank_load"].cpu().tolist()

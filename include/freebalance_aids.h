@@ -27,6 +27,17 @@ uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
  * alone inside a call that launches several kernels. */
 fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
 
+/* Floor of the one-tile router kernel's main loop.  Launches that kernel for x exactly as
+ * fb_predict_load would (same grid, block pairs, pipeline stages and tensor maps; never the
+ * persistent kernel, never the k-range split), but with what = 1 the operands are only loaded
+ * (no MMA is issued) and with what = 2 they are loaded and multiplied; in both cases nothing
+ * follows the main loop: no gating, no selection, no histogram, no output, no status.  Timed
+ * by the caller it shows what launch, set-up and the operand stream alone cost for this
+ * tiling (1) and what the tensor pipe adds (2).  Errors as fb_predict_load; what outside
+ * {1, 2}: FB_ERR_INVALID_ARG. */
+fb_status fb_router_floor(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T, int32_t what,
+                          fb_stream stream);
+
 /* Stand-in for an attention kernel, for overlap experiments on one GPU (the method hides
  * prediction, planning and weight transfer behind the target layer's attention; "Overlap
  * Analysis").  A compute-bound kernel of `blocks` blocks, one per SM (1024 threads and 120 KB

@@ -55,7 +55,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_pre
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
            "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
-           "fb_time_next_router_launch", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
+           "fb_time_next_router_launch", "fb_router_floor", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
            "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
            "fb_set_stamp_buffer", "fb_clock_probe", "fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns",
            "fb_attention_set_time_ns", "fb_attention_reset", "fb_dispatch_slot_counts", "fb_dispatch_globalize",
@@ -141,6 +141,8 @@ def lib() -> ctypes.CDLL:
     L.fb_calibrate_exchange.argtypes = [vp, u64, u64, i32] + [ctypes.POINTER(u64)] * 4 + [vp]
     L.fb_calibrate_exchange.restype = ctypes.c_int
     L.fb_topk_hits.restype = ctypes.c_int
+    L.fb_router_floor.argtypes = [vp, ctypes.POINTER(FbRouter), vp, i32, i32, vp]
+    L.fb_router_floor.restype = ctypes.c_int
     L.fb_time_next_router_launch.argtypes = [vp, vp, vp]
     L.fb_time_next_router_launch.restype = ctypes.c_int
     L.fb_persistent_launch_count.argtypes = [vp]
@@ -390,6 +392,10 @@ class Context:
     def fb_selftest_wait_timeout(self, limit_ns: int, waited_ns=None, stream=None) -> None:
         _check(lib().fb_selftest_wait_timeout(self._h, limit_ns, _ptr(waited_ns), _stream(stream)),
                "fb_selftest_wait_timeout")
+
+    def fb_router_floor(self, router, x, T: int, what: int, stream=None) -> None:
+        _check(lib().fb_router_floor(self._h, ctypes.byref(router), _ptr(x), T, what, _stream(stream)),
+               "fb_router_floor")
 
     def fb_time_next_router_launch(self, event_before, event_after) -> None:
         """torch.cuda.Event objects (created with enable_timing=True); either may be None."""

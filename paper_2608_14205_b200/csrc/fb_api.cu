@@ -233,7 +233,7 @@ static RouterKernelFn persistent_kernel_fn(bool sigmoid, bool lb) {
 // x2 is the second input of kModeLayer (the normal router input), nullptr otherwise.
 fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T, int mode,
                         uint32_t* counts_out, int32_t* topk_ids, float* topk_w, float* logits,
-                        const fb::PlanParams* plan, cudaStream_t stream, const void* x2 = nullptr) {
+                        const fb::PlanParams* plan, cudaStream_t stream, const void* x2 = nullptr, int probe = 0) {
   const CUtensorMap *mx = nullptr, *mx2 = nullptr, *mw = nullptr;
   fb_status st = make_map(ctx, ctx->x_maps, &ctx->x_next, x, T, fb::kTileM, &mx);
   if (st != FB_OK) return st;
@@ -271,6 +271,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.logits = logits;
   p.tile_counts = ctx->tile_counts;
   p.stamps = ctx->stamps;
+  p.probe = probe;
   if (plan) p.plan = *plan;
   // The fused tail serves the common plans; a plan that needs the general loop (per-expert sizes,
   // more than 16 experts per rank, a planner variant) gets the stand-alone planner kernel behind
@@ -288,7 +289,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   const int sel = fb::select_kind(c.E, ctx->N, c.k, c.gate, p.n_group, p.topk_group,
                                   topk_w != nullptr && !c.renorm && c.gate == FB_GATE_SOFTMAX_TOPK);
   bool persistent = false;
-  if (pair && ctx->persist_stages >= 2 && logits == nullptr) {
+  if (pair && ctx->persist_stages >= 2 && logits == nullptr && probe == 0) {
     const bool want_sum = topk_w != nullptr && !c.renorm && c.gate == FB_GATE_SOFTMAX_TOPK;
     const int pairs_avail = ctx->pair_limit > 0 && ctx->pair_limit < ctx->max_pairs ? ctx->pair_limit : ctx->max_pairs;
     if (fb::persistent_gate_ok(c.E, c.k, c.gate, p.n_group, p.topk_group, want_sum) && blocks / 2 > pairs_avail) {
@@ -309,7 +310,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   // the tail of every tile's k-range (see RouterParams).  The schedule depends on the shape and
   // on the number of pairs only.
   bool split = false;
-  if (pair && !persistent && mode != fb::kModeLayer && ctx->split_partial != nullptr && ctx->split_mode != 0) {
+  if (pair && !persistent && mode != fb::kModeLayer && ctx->split_partial != nullptr && ctx->split_mode != 0 && probe == 0) {
     const int tile_pairs = tiles_pad / 2;
     int pairs_avail = ctx->split_pairs;
     if (ctx->pair_limit > 0 && ctx->pair_limit < pairs_avail) pairs_avail = ctx->pair_limit;
@@ -1023,6 +1024,17 @@ fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* even
   ctx->ev_before = static_cast<cudaEvent_t>(event_before);
   ctx->ev_after = static_cast<cudaEvent_t>(event_after);
   return FB_OK;
+}
+
+fb_status fb_router_floor(fb_ctx* ctx, const fb_router* router, const void* x, int32_t T, int32_t what,
+                          fb_stream stream_) {
+  if (!ctx || !router || !router->W || !x || T <= 0 || (what != 1 && what != 2
+       )) return FB_ERR_INVALID_ARG;
+  if (T > ctx->cfg.T_max) return FB_ERR_UNSUPPORTED_SHAPE;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return FB_ERR_CUDA;
+  return launch_router(ctx, router, x, T, fb::kModePredict, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       static_cast<cudaStream_t>(stream_), nullptr, what);
 }
 
 int32_t fb_max_pairs(const fb_ctx* ctx) { return ctx ? ctx->max_pairs : 0; }

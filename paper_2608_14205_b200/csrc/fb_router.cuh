@@ -99,6 +99,8 @@ struct RouterParams {
   float* logits;                     // [T][E] or nullptr
   uint32_t* tile_counts;             // [tiles][E]    (dispatch mode)
   unsigned long long* stamps;        // [blocks][64] phase time stamps (FB_TIMING builds) or nullptr
+  int32_t probe;                     // measurement aid: 1 = operands are loaded but no MMA is issued and nothing
+                                     // follows the main loop; 2 = with the MMAs, still nothing after them
   // k-range split (kSplit instances): the first 2 * split_helpers blocks are helper pairs, the
   // tiles' owners follow.  An owner accumulates k-blocks [0, split_ko) of its tile; the rest,
   // [split_ko, num_kb), is cut into split_j pieces, each summed by one helper pair (helper
@@ -639,10 +641,12 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
           const uint64_t adesc = umma_smem_desc_sw128(a_addr);
           const uint64_t bdesc = umma_smem_desc_sw128(a_addr + kATileBytes);
+          if (p.probe != 1) {
   #pragma unroll
-          for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
-            // advance 16 elements = 32 bytes inside the swizzled row: +2 in the address field
-            umma_bf16<kCtas>(acc, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb != first_kb || kk != 0) ? 1u : 0u);
+            for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
+              // advance 16 elements = 32 bytes inside the swizzled row: +2 in the address field
+              umma_bf16<kCtas>(acc, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb != first_kb || kk != 0) ? 1u : 0u);
+            }
           }
           // frees the stage (in both blocks of a pair) when these MMAs retire
           if (kCtas == 1) umma_commit_1cta(smem_u32(&sh.empty_bar[s]));
@@ -712,7 +716,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
       if (mode == kModePredictPlan) plan_load_placement(p.plan, sh.plan, et, kEpilogueThreads);
       named_bar_sync(kAccumBarrierId, kEpilogueThreads + 32);
-      const bool got = sh.accum_ok != 0;
+      const bool got = sh.accum_ok != 0 && p.probe == 0;     // a measurement launch ends with its main loop
       tcgen05_fence_after();
       FB_STAMP(2, 64);
 
@@ -1145,7 +1149,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (static_cast<long long>(tile) * kTileM < p.T)       // the padding block of an odd pair owns no tile
           for (int e = et; e < E; e += kEpilogueThreads)
             p.tile_counts[static_cast<size_t>(tile) * E + e] = sh.hist[e];
-      } else {
+      } else if (p.probe == 0) {
         publish_counts(sh, p, et, warp, lane, mode == kModePredictPlan && p.fuse_planner != 0);
       }
       FB_STAMP(12, 64);

@@ -570,6 +570,33 @@ def test_router_launch_events_and_pair_queries():
     tiny.close()
 
 
+def test_main_loop_floor_launches_leave_no_trace():
+    # The measurement launches (operands loaded only / loaded and multiplied, nothing after the main
+    # loop) write no output, take no ticket and leave the context ready for the next normal call.
+    for name, T in (("dsv3", 1500), ("tiny", 300), ("qwen3", 700)):
+        wl = I.WORKLOADS[name]
+        li = I.make_layer(wl, 1, 0, T=T)
+        ctx = P.make_context(wl, T)
+        dev = torch.device("cuda", ctx.device)
+        sb = li.select_bias.to(dev) if li.select_bias is not None else None
+        router = B.make_router(li.W.to(dev), None, sb)
+        x = li.h_prev.to(dev)
+        counts, ref = (torch.full((wl.E,), -7, dtype=torch.int32, device=dev) for _ in range(2))
+        ctx.fb_predict_load(router, x, T, ref)
+        launches = ctx.fb_launch_count()
+        for what in (1, 2, 2, 1):
+            ctx.fb_router_floor(router, x, T, what)
+        torch.cuda.synchronize(dev)
+        assert ctx.fb_device_status() == 0
+        assert ctx.fb_launch_count() == launches + 4
+        ctx.fb_predict_load(router, x, T, counts)
+        torch.cuda.synchronize(dev)
+        assert torch.equal(counts, ref) and int(counts.sum().item()) == T * wl.k
+        with pytest.raises(Exception):
+            ctx.fb_router_floor(router, x, T, 3)
+        ctx.close()
+
+
 def test_two_contexts_on_two_streams_do_not_interfere():
     # each context owns its scratch: calls of different contexts may overlap on the device
     wl = I.WORKLOADS["dsv3"]

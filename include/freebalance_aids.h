@@ -27,6 +27,14 @@ uint64_t fb_persistent_launch_count(const fb_ctx* ctx);
  * alone inside a call that launches several kernels. */
 fb_status fb_time_next_router_launch(fb_ctx* ctx, void* event_before, void* event_after);
 
+/* Diagnostic: later router launches of this context use at most `stages` stages of the
+ * operand pipeline (0 lifts the limit; 1 is not a pipeline: FB_ERR_INVALID_ARG).  Results do
+ * not depend on the depth, only the speed does.  Exists so that tests can run short rings and
+ * rings with an odd number of stages, in which a stage alternates between the two MMA issuers
+ * (they then keep each other informed of their progress; with an even number a stage always
+ * serves the same issuer). */
+fb_status fb_set_stage_limit(fb_ctx* ctx, int32_t stages);
+
 /* Floor of the one-tile router kernel's main loop.  Launches that kernel for x exactly as
  * fb_predict_load would (same grid, block pairs, pipeline stages and tensor maps; never the
  * persistent kernel, never the k-range split), but with what = 1 the operands are only loaded

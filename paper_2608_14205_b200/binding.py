@@ -54,7 +54,7 @@ FB_ERR_INTERNAL = 7
 EXPORTS = ["fb_create", "fb_destroy", "fb_budget_ns", "fb_swap_cost_ns", "fb_predict_load",
            "fb_plan_swaps", "fb_predict_and_plan", "fb_route_dispatch", "fb_layer_step_host",
            "fb_device_status", "fb_launch_count", "fb_status_string", "fb_predict_load_static", "fb_layer_step",
-           "fb_set_pair_limit", "fb_max_pairs", "fb_persistent_launch_count",
+           "fb_set_pair_limit", "fb_set_stage_limit", "fb_max_pairs", "fb_persistent_launch_count",
            "fb_time_next_router_launch", "fb_router_floor", "fb_row_cosine_mean", "fb_topk_hits", "fb_apply_swaps",
            "fb_apply_swaps_staged", "fb_fit_cost_model", "fb_calibrate_exchange", "fb_selftest_wait_timeout",
            "fb_set_stamp_buffer", "fb_clock_probe", "fb_attention_begin", "fb_attention_end", "fb_layer_budget_ns",
@@ -103,6 +103,8 @@ def lib() -> ctypes.CDLL:
                                          vp, vp, vp, vp]
     L.fb_predict_load_static.restype = ctypes.c_int
     L.fb_device_status.argtypes = [vp, ctypes.POINTER(i32), vp]
+    L.fb_set_stage_limit.argtypes = [vp, i32]
+    L.fb_set_stage_limit.restype = ctypes.c_int
     L.fb_set_pair_limit.argtypes = [vp, i32]
     L.fb_set_pair_limit.restype = ctypes.c_int
     L.fb_max_pairs.argtypes = [vp]
@@ -348,6 +350,9 @@ class Context:
 
     def fb_set_pair_limit(self, pairs: int) -> None:
         _check(lib().fb_set_pair_limit(self._h, pairs), "fb_set_pair_limit")
+
+    def fb_set_stage_limit(self, stages: int) -> None:
+        _check(lib().fb_set_stage_limit(self._h, stages), "fb_set_stage_limit")
 
     def fb_set_split(self, mode: int, owner_bias_kblocks: int = -1) -> None:
         _check(lib().fb_set_split(self._h, mode, owner_bias_kblocks), "fb_set_split")

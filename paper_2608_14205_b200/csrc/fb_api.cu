@@ -49,6 +49,7 @@ struct fb_ctx {
   size_t persist_smem = 0;
   int max_pairs = 0;
   int pair_limit = 0;
+  int stage_limit = 0;                 // diagnostic: pipeline stages at most (0 = as many as fit)
   int dispatch_blocks_max = 296;       // resident blocks of the dispatch-index kernel (2 per SM)
   // k-range split of the one-tile pair kernel: block pairs that fit on the GPU at once, the
   // partial tiles and their flags (one slot per helper item), a launch counter for the flags'
@@ -258,6 +259,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
   p.renorm = c.renorm; p.route_scale = c.route_scale;
   p.num_kb = (c.d + fb::kBlockK - 1) / fb::kBlockK;
   p.stages = ctx->stages[pair];
+  if (ctx->stage_limit >= 2 && ctx->stage_limit < p.stages) p.stages = ctx->stage_limit;
   p.tmem_cols = ctx->tmem_cols;
   p.mode = mode;
   p.logit_bias = router->logit_bias;
@@ -304,6 +306,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
       // room for two accumulator sets (4 N columns) when the 512 tensor-memory columns allow it
       if (4 * ctx->N <= 512) p.tmem_cols = next_pow2_at_least_32(4 * ctx->N);
       p.stages = ctx->persist_stages;
+      if (ctx->stage_limit >= 2 && ctx->stage_limit < p.stages) p.stages = ctx->stage_limit;
     }
   }
   // Fewer tile pairs than block pairs fit on the GPU: the spare pairs become helpers that sum
@@ -1010,6 +1013,12 @@ fb_status fb_set_split(fb_ctx* ctx, int32_t mode, int32_t owner_bias_kblocks) {
   if (!ctx || (mode != 0 && mode != 1) || owner_bias_kblocks < -1 || owner_bias_kblocks > 1024) return FB_ERR_INVALID_ARG;
   ctx->split_mode = mode;
   ctx->split_bias = owner_bias_kblocks;
+  return FB_OK;
+}
+
+fb_status fb_set_stage_limit(fb_ctx* ctx, int32_t stages) {
+  if (!ctx || stages < 0 || stages == 1) return FB_ERR_INVALID_ARG;
+  ctx->stage_limit = stages;
   return FB_OK;
 }
 

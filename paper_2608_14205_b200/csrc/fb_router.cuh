@@ -194,6 +194,7 @@ struct RouterShared {
   int32_t abort_flag;
   int32_t is_last;
   int32_t accum_ok;
+  int32_t issuer_progress[2];                // rings with an odd number of stages: see issuer_turn_wait
   float logit_bias[FB_MAX_EXPERTS + 32];     // + 32: a partial last chunk is read in full
   alignas(16) float select_bias[FB_MAX_EXPERTS + 32];
   uint32_t hist[FB_MAX_EXPERTS];
@@ -412,6 +413,28 @@ __device__ __forceinline__ bool flag_wait(const uint32_t* flag, uint32_t epoch, 
   }
 }
 
+// Two MMA issuers share one ring of stages.  With an even number of stages a stage always serves
+// the same issuer, which therefore sees every phase of the stage's "full" barrier.  With an odd
+// number a stage alternates between them, and a parity wait alone cannot tell "the other issuer's
+// use of this stage is still being filled" (a wait for my parity passes on the phase before it)
+// from "my use is complete".  So each issuer publishes the ring position of the last k-block whose
+// operands it has seen arrive, and before it waits for position g on a stage whose previous use
+// (position g - stages) was the other issuer's, it waits until the other one has got that far.
+__device__ __forceinline__ bool issuer_turn_wait(const volatile int32_t* other_progress, int32_t need,
+                                                 volatile int* abort_flag) {
+  uint32_t polls = 0;
+  uint64_t t0 = 0;
+  while (*other_progress < need) {
+    if ((++polls & 0x3Fu) == 0) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+  return true;
+}
+
 // Offset (in floats) of column `col`, row 0 of the partial tile that block `cta` of a pair owns in `slot`.
 __device__ __forceinline__ size_t partial_offset(int slot, uint32_t cta, int N, int col) {
   return ((static_cast<size_t>(slot) * 2 + cta) * static_cast<size_t>(N) + static_cast<size_t>(col)) * kTileM;
@@ -463,6 +486,8 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   if (threadIdx.x == 0) {
     sh.abort_flag = 0;
     sh.is_last = 0;
+    sh.issuer_progress[0] = -1;
+    sh.issuer_progress[1] = -1;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&sh.full_bar[s]), 1);
       mbar_init(smem_u32(&sh.empty_bar[s]), 1);
@@ -537,11 +562,16 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const uint32_t acc = tmem_base + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
         const uint32_t idesc = umma_idesc_bf16_f32(kTileM * 2, static_cast<uint32_t>(p.N));
         bool ok = true;
+        const bool odd_ring = (p.stages & 1) != 0;
+        volatile int32_t* my_progress = &sh.issuer_progress[warp == 1 ? 0 : 1];
+        const volatile int32_t* other_progress = &sh.issuer_progress[warp == 1 ? 1 : 0];
         for (int kb = first_kb; kb < kb1 && ok; kb += 2) {
           const int s = (kb - kb0) % p.stages;
           const uint32_t phase = static_cast<uint32_t>((kb - kb0) / p.stages) & 1u;
-          ok = mbar_wait<true>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
+          if (odd_ring && kb - kb0 >= p.stages) ok = issuer_turn_wait(other_progress, kb - kb0 - p.stages, abort_flag);
+          ok = ok && mbar_wait<true>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
           if (!ok) break;
+          if (odd_ring) *my_progress = kb - kb0;
           tcgen05_fence_after();
           const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
           const uint64_t adesc = umma_smem_desc_sw128(a_addr);
@@ -631,11 +661,17 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const uint32_t acc = tmem_base + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
         const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.N));
         bool ok = true;
+        const bool odd_ring = (p.stages & 1) != 0;
+        volatile int32_t* my_progress = &sh.issuer_progress[warp == 1 ? 0 : 1];
+        const volatile int32_t* other_progress = &sh.issuer_progress[warp == 1 ? 1 : 0];
         for (int kb = first_kb; kb < kb_end && ok; kb += 2) {
           const int s = kb % p.stages;
           const uint32_t phase = static_cast<uint32_t>(kb / p.stages) & 1u;
-          ok = mbar_wait<kCtas == 2>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
+          // an odd ring: the stage's previous use (k-block kb - stages) was the other issuer's
+          if (odd_ring && kb >= p.stages) ok = issuer_turn_wait(other_progress, kb - p.stages, abort_flag);
+          ok = ok && mbar_wait<kCtas == 2>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
           if (!ok) break;
+          if (odd_ring) *my_progress = kb;
           tcgen05_fence_after();
           if (kb == 0) FB_STAMP(16, 32);
           const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;

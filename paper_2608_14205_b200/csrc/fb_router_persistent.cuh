@@ -41,6 +41,7 @@ struct PersistShared {
   int32_t is_last;
   int32_t accum_ok;
   int32_t any_overflow;
+  int32_t issuer_progress[2];                // rings with an odd number of stages: see issuer_turn_wait
   float logit_bias[FB_MAX_EXPERTS];
   alignas(16) float select_bias[FB_MAX_EXPERTS];
   uint32_t hist[FB_MAX_EXPERTS];
@@ -90,6 +91,8 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     sh.abort_flag = 0;
     sh.is_last = 0;
     sh.any_overflow = 0;
+    sh.issuer_progress[0] = -1;
+    sh.issuer_progress[1] = -1;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&sh.full_bar[s]), 1);
       mbar_init(smem_u32(&sh.empty_bar[s]), 1);
@@ -167,6 +170,10 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
       uint32_t phase = 0;
       uint32_t ti = 0;                        // this block pair's tile counter
       bool ok = true;
+      int32_t g = 0;                          // ring position: k-blocks of all of this pair's tiles, in order
+      const bool odd_ring = (p.stages & 1) != 0;
+      volatile int32_t* my_progress = &sh.issuer_progress[warp == 1 ? 0 : 1];
+      const volatile int32_t* other_progress = &sh.issuer_progress[warp == 1 ? 1 : 0];
       for (int pt = pair_first; pt < total_pairs && ok; pt += pair_stride, ++ti) {
         const uint32_t set = ti % acc_sets, use = ti / acc_sets;
         const uint32_t acc = tmem_base + set * 2u * static_cast<uint32_t>(p.N) + (warp == 1 ? 0u : static_cast<uint32_t>(p.N));
@@ -176,10 +183,18 @@ fb_router_persistent_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
           if (!ok) break;
           tcgen05_fence_after();
         }
-        for (int kb = 0; kb < p.num_kb; ++kb) {
+        for (int kb = 0; kb < p.num_kb; ++kb, ++g) {
           if ((kb & 1) == first_kb) {
-            ok = mbar_wait<true>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
+            if (odd_ring && g >= p.stages) {
+              // whose was the stage's previous use (ring position g - stages)?  Its k-block index
+              // inside its own tile decides, as for every k-block.
+              int kbp = kb - p.stages;
+              while (kbp < 0) kbp += p.num_kb;
+              if ((kbp & 1) != first_kb) ok = issuer_turn_wait(other_progress, g - p.stages, abort_flag);
+            }
+            ok = ok && mbar_wait<true>(smem_u32(&sh.full_bar[s]), phase, abort_flag);
             if (!ok) break;
+            if (odd_ring) *my_progress = g;
             tcgen05_fence_after();
             const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
             const uint64_t adesc = umma_smem_desc_sw128(a_addr);

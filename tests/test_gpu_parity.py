@@ -514,6 +514,35 @@ def test_pair_limit_does_not_change_results():
     ctx.close()
 
 
+@pytest.mark.parametrize("name,T,split", [("dsv3", 3000, 0), ("qwen3", 2500, 0), ("dsv3", 1100, 1)])
+def test_pipeline_depth_does_not_change_results(name, T, split):
+    # Short operand rings, and rings with an odd number of stages (a stage then alternates between
+    # the two MMA issuers, which keep each other informed of their progress): same bits as the full
+    # depth, through the one-tile kernel, its k-range split and the persistent kernel.  With three
+    # stages an issuer that took a stale phase of a "full" barrier for its own would read operands
+    # that have not arrived.
+    wl = I.WORKLOADS[name]
+    li = I.make_layer(wl, 3, 0, T=T)
+    ctx = P.make_context(wl, T)
+    ctx.fb_set_split(split)
+    bkw = P.budget_kwargs(wl, T)
+    ref = {lim: P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False, pair_limit=lim) for lim in (0, 3)}
+    for stages in (3, 2, 5):
+        ctx.fb_set_stage_limit(stages)
+        for lim in (0, 3):
+            for _ in range(3):
+                got = P.run_gpu_layer(ctx, wl, li, bkw, want_logits=False, pair_limit=lim)
+                assert got["status"] == 0
+                for key in ("counts", "ids_early", "ids", "w", "perm", "inv_perm", "slot_offsets", "rank_load"):
+                    assert np.array_equal(ref[lim][key], got[key]), (stages, lim, key)
+                assert ref[lim]["swaps"] == got["swaps"] and ref[lim]["layer"]["swaps"] == got["layer"]["swaps"]
+                assert np.array_equal(ref[lim]["layer"]["ids"], got["layer"]["ids"])
+    ctx.fb_set_stage_limit(0)
+    with pytest.raises(Exception):
+        ctx.fb_set_stage_limit(1)
+    ctx.close()
+
+
 @pytest.mark.parametrize("name,T,d", [("qwen3", 8192, None), ("mixtral", 4096, None), ("dsv3", 4096, None),
                                        ("qwen3", 1000, None), ("dsv3", 2049, 2112), ("mixtral", 300, 2048)])
 def test_k_range_split_on_and_off_agree_with_the_oracle(name, T, d):

@@ -731,6 +731,10 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       const bool want_sum = kSel == kSelectGeneral && out_w != nullptr && !p.renorm && !sigmoid_gate;
       // Selection by ranking a short candidate list instead of insertion (see select_kind).
       constexpr bool fast_select = kSel != kSelectGeneral;
+      // Softmax gate over at most 32 experts (one chunk): the thread of sub 0 holds its whole row in
+      // registers after pass 1 and selects there; nothing is parked in shared memory, nothing is
+      // merged, and the warps that share the rows need not meet.
+      const bool small_gate = kSel == kSelectGeneral && !sigmoid_gate && n_chunks == 1;
 
       // Chunk bookkeeping, worked out while the main loop runs (integer divisions by run-time
       // values are slow and would otherwise sit between the chunks of the epilogue):
@@ -766,7 +770,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 
       // Between pass 1 and the histogram, data passes only between the kEpiSubs warps that share
       // this warp's rows: they meet at a barrier of their own and do not wait for the other rows' warps.
-      auto row_sync = [&]() { named_bar_sync(kRowBarrierBase + static_cast<uint32_t>(quarter), kEpiSubs * 32); };
+      auto row_sync = [&]() { if (!small_gate) named_bar_sync(kRowBarrierBase + static_cast<uint32_t>(quarter), kEpiSubs * 32); };
 
       TopK top;
       top.init();
@@ -861,7 +865,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
               q[j] = (c0 + j < E) ? z : -INFINITY;
             }
           }
-          {
+          if (!small_gate) {
             float* kcol = key_s + c0 * kTileM + row_in_tile;
   #pragma unroll
             for (int j = 0; j < 32; ++j)
@@ -877,6 +881,22 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             for (int j = 0; j < 32; ++j) part += __expf(q[j] - nmax);     // exp(-inf) = 0 for padding
             sm_sum = sm_sum * __expf(sm_max - nmax) + part;
             sm_max = nmax;
+          }
+          if (small_gate) {
+            // k rounds of "largest remaining key"; the scan runs in ascending column order with a
+            // strict comparison, so the lower expert id wins a tie.  Padding columns hold -inf.
+  #pragma unroll 1
+            for (int rnd = 0; rnd < k; ++rnd) {
+              float best = q[0];
+              int bi = 0;
+  #pragma unroll
+              for (int j = 1; j < 32; ++j)
+                if (q[j] > best) { best = q[j]; bi = j; }
+              top.insert_any_order(best, bi);
+  #pragma unroll
+              for (int j = 0; j < 32; ++j) q[j] = (j == bi) ? -INFINITY : q[j];
+            }
+            continue;
           }
           if (sigmoid_gate && gs % 32 == 0) {
             // the chunk lies inside one group: branch-free top-2 of its 32 keys by a merge tree
@@ -1055,7 +1075,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           }
         }
       }
-      if (got && !fast_select) {
+      if (got && !fast_select && !small_gate) {
         // ---------------- choose the groups; lower bound for the k-th key
         uint32_t keep = 1u;
         float floor_key = -INFINITY;
@@ -1138,7 +1158,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
       row_sync();
       const bool writer = got && valid && sub == 0;
-      if (got && sub == 0 && !fast_select) {
+      if (got && sub == 0 && !fast_select && !small_gate) {
   #pragma unroll 1
         for (int s2 = 1; s2 < kEpiSubs; ++s2) {
   #pragma unroll 1

@@ -260,23 +260,37 @@ __device__ __forceinline__ uint32_t plan_loop_uniform(const PlanParams& p, PlanS
       // One 64-bit key per candidate: benefit, then the complement of the pair (so that the
       // larger key is the better candidate), then the candidate's index in this lane.  The
       // candidates of a lane are independent of each other; only the maximum chains them.
-      unsigned long long best_key = 0;
+      // Written stage by stage over all candidates (differences, bounds, benefits, keys) and reduced
+      // by a tree, so that nothing but the data flow orders the instructions of different candidates.
+      int dl[kPerLane];
+      uint32_t ben[kPerLane];
+      unsigned long long key[kPerLane];
+#pragma unroll
+      for (int t = 0; t < kPerLane; ++t)
+        dl[t] = static_cast<int>(wa[t] & kSlotCountMask) - static_cast<int>(wb[t] & kSlotCountMask);   // tokens moved a -> b
 #pragma unroll
       for (int t = 0; t < kPerLane; ++t) {
-        const int dlt = static_cast<int>(wa[t] & kSlotCountMask) - static_cast<int>(wb[t] & kSlotCountMask);   // tokens moved a -> b
-        int Mn = La - dlt;                                        // Eq. 6
-        if (Lb + dlt > Mn) Mn = Lb + dlt;                         // Eq. 7
+        int Mn = La - dl[t];                                      // Eq. 6
+        if (Lb + dl[t] > Mn) Mn = Lb + dl[t];                     // Eq. 7
         if (M2 > Mn) Mn = M2;
         // gamma_den * (Phi(L) - Phi(L')), variance term 2 dlt (La - Lb - dlt).  It is positive only
         // for 0 < dlt < D, and inside that range both terms are non-negative.
-        const bool usable = cand_ok[t] && ((wa[t] | wb[t]) >> 31) == 0 && dlt > 0 && dlt < D;   // neither expert moved yet
+        const bool usable = cand_ok[t] && ((wa[t] | wb[t]) >> 31) == 0 && dl[t] > 0 && dl[t] < D;   // neither expert moved yet
         const uint32_t b32 = gden * static_cast<uint32_t>(La - Mn) +
-                             gnum2 * (static_cast<uint32_t>(dlt) * static_cast<uint32_t>(D - dlt));
-        const uint32_t pair = ((wa[t] >> 22) & 0xffu) << 8 | ((wb[t] >> 22) & 0xffu);
-        const unsigned long long key = static_cast<unsigned long long>(usable ? b32 : 0u) << 32 |
-                                       static_cast<unsigned long long>(0xffffu - pair) << 8 | static_cast<unsigned>(t);
-        best_key = key > best_key ? key : best_key;
+                             gnum2 * (static_cast<uint32_t>(dl[t]) * static_cast<uint32_t>(D - dl[t]));
+        ben[t] = usable ? b32 : 0u;
       }
+#pragma unroll
+      for (int t = 0; t < kPerLane; ++t) {
+        const uint32_t pair = ((wa[t] >> 22) & 0xffu) << 8 | ((wb[t] >> 22) & 0xffu);
+        key[t] = static_cast<unsigned long long>(ben[t]) << 32 |
+                 static_cast<unsigned long long>(0xffffu - pair) << 8 | static_cast<unsigned>(t);
+      }
+#pragma unroll
+      for (int w = kPerLane / 2; w >= 1; w >>= 1)
+#pragma unroll
+        for (int t = 0; t < w; ++t) key[t] = key[t] > key[t + w] ? key[t] : key[t + w];
+      const unsigned long long best_key = key[0];
       const uint32_t mine = static_cast<uint32_t>(best_key >> 32);
       const uint32_t top = __reduce_max_sync(full, mine);
       if (stop || top == 0) break;                                // Algorithm 1 lines 6-7

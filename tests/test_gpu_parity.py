@@ -514,14 +514,18 @@ def test_pair_limit_does_not_change_results():
     ctx.close()
 
 
-@pytest.mark.parametrize("name,T,split", [("dsv3", 3000, 0), ("qwen3", 2500, 0), ("dsv3", 1100, 1)])
-def test_pipeline_depth_does_not_change_results(name, T, split):
+@pytest.mark.parametrize("name,T,split,d", [("dsv3", 3000, 0, None), ("qwen3", 2500, 0, None), ("dsv3", 1100, 1, None),
+                                             ("dsv3", 1300, 0, 2112)])
+def test_pipeline_depth_does_not_change_results(name, T, split, d):
     # Short operand rings, and rings with an odd number of stages (a stage then alternates between
     # the two MMA issuers, which keep each other informed of their progress): same bits as the full
     # depth, through the one-tile kernel, its k-range split and the persistent kernel.  With three
     # stages an issuer that took a stale phase of a "full" barrier for its own would read operands
-    # that have not arrived.
+    # that have not arrived.  d = 2112 gives an odd number of k-blocks: in the persistent kernel the
+    # issuer that owns a ring position then changes from tile to tile.
     wl = I.WORKLOADS[name]
+    if d is not None:
+        wl = dataclasses.replace(wl, d=d)
     li = I.make_layer(wl, 3, 0, T=T)
     ctx = P.make_context(wl, T)
     ctx.fb_set_split(split)

@@ -328,7 +328,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
       int ko = (p.num_kb + J) / (J + 1);
       // a helper pays for the copy-out of its partial, the owner for reading it: owners keep a
       // few k-blocks more than an even share
-      ko += ctx->split_bias >= 0 ? ctx->split_bias : 2;
+      ko += ctx->split_bias >= 0 ? ctx->split_bias : 4;
       if (ko > p.num_kb - 2 * J) ko = p.num_kb - 2 * J;     // every piece has at least two k-blocks
       if (ko >= 2) {
         split = true;

@@ -78,6 +78,19 @@ def test_edge_shapes(kw):
     _run(_wl(**kw), 300, with_logit_bias=True)
 
 
+@pytest.mark.parametrize("kw,T", [
+    (dict(E=192, k=6, R=8, d=1600), 700),                                    # pairs: 7 stages
+    (dict(E=192, k=6, R=8, d=1600), 100),                                    # one block: 5 stages
+    (dict(E=224, k=8, R=7, d=1096), 450),                                    # pairs: 7 stages
+    (dict(gate=1, n_group=6, topk_group=3, k=6, E=192, R=6, d=1600), 700),   # ranking selection, 7 stages
+])
+def test_widths_whose_operand_ring_has_an_odd_number_of_stages(kw, T):
+    # At these widths as many stages as fit is an odd number, so a stage alternates between the two
+    # MMA issuers without any diagnostic limit being set.
+    _run(_wl(**kw), T, with_logit_bias=True)
+    _run(_wl(**kw), T, layer=1)
+
+
 def test_select_bias_large_enough_to_change_the_selection():
     wl = _wl(gate=1, n_group=4, topk_group=2, k=2)
     li = I.make_layer(wl, 0, 0, T=200)

@@ -28,6 +28,13 @@
  *   - Calls enqueue work on `stream` and return without synchronising, except
  *     fb_layer_step_host and fb_device_status, which block until the stream drains,
  *     fb_apply_swaps_staged (waits for the plan) and fb_calibrate_exchange (times itself).
+ *   - The method's device calls (fb_predict_load, fb_plan_swaps, fb_predict_and_plan,
+ *     fb_route_dispatch, fb_layer_step, the dispatch-index helpers) allocate nothing,
+ *     query nothing and keep no per-launch state on the host that a kernel depends on,
+ *     so after one ordinary call with the same arguments (which builds the tensor maps
+ *     and loads the kernels) they may be captured into a CUDA graph and the graph
+ *     replayed on new contents of the same buffers.  Budgets and shapes are frozen into
+ *     the graph at capture; fb_device_status is not capturable (it synchronises).
  *   - No call throws or aborts.  Argument and shape problems are reported by the
  *     return value and nothing is launched.  Problems only the device can see (a
  *     placement that is not a bijection, count sums beyond the planner's range, a

@@ -52,12 +52,11 @@ struct fb_ctx {
   int stage_limit = 0;                 // diagnostic: pipeline stages at most (0 = as many as fit)
   int dispatch_blocks_max = 296;       // resident blocks of the dispatch-index kernel (2 per SM)
   // k-range split of the one-tile pair kernel: block pairs that fit on the GPU at once, the
-  // partial tiles and their flags (one slot per helper item), a launch counter for the flags'
-  // epoch, and the caller's switch / tuning value
+  // partial tiles and their flags (one slot per helper item; set by the helper, put back by the
+  // owner), and the caller's switch / tuning value
   int split_pairs = 0;
   float* split_partial = nullptr;
   uint32_t* split_flags = nullptr;
-  uint32_t split_epoch = 0;
   int split_mode = 1;                  // 0 off, 1 on
   int split_bias = -1;                 // extra k-blocks an owner keeps (-1: the built-in choice)
   EncodeTiledFn encode = nullptr;
@@ -335,8 +334,7 @@ fb_status launch_router(fb_ctx* ctx, const fb_router* router, const void* x, int
         p.split_helpers = helpers;
         p.split_ko = ko;
         p.split_j = J;
-        if (++ctx->split_epoch == 0) ctx->split_epoch = 1;
-        p.split_epoch = ctx->split_epoch;
+        p.split_epoch = 1;          // "complete"; the owner that consumed a partial puts the flag back to 0
         p.split_partial = ctx->split_partial;
         p.split_flags = ctx->split_flags;
         blocks += 2 * helpers;
@@ -826,7 +824,13 @@ fb_status fb_device_status(fb_ctx* ctx, int32_t* word, fb_stream stream_) {
   if (!guard.ok) return FB_ERR_CUDA;
   if (cudaStreamSynchronize(stream) != cudaSuccess) return FB_ERR_CUDA;
   if (cudaMemcpy(word, ctx->status, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return FB_ERR_CUDA;
-  if (*word != 0 && cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) return FB_ERR_CUDA;
+  if (*word != 0) {
+    if (cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) return FB_ERR_CUDA;
+    // a launch that gave up may have left partial-tile flags of the k-range split set: re-arm them
+    if (ctx->split_flags != nullptr &&
+        cudaMemset(ctx->split_flags, 0, static_cast<size_t>(ctx->split_pairs) * 2 * sizeof(uint32_t)) != cudaSuccess)
+      return FB_ERR_CUDA;
+  }
   return FB_OK;
 }
 

@@ -109,7 +109,9 @@ struct RouterParams {
   int32_t split_helpers;             // helper pairs in the grid (0: no split)
   int32_t split_ko;                  // k-blocks an owner keeps
   int32_t split_j;                   // pieces per tile = helper pairs per tile pair
-  uint32_t split_epoch;              // value a partial's flag takes when the partial of THIS launch is complete
+  uint32_t split_epoch;              // value a partial's flag takes when it is complete; the owner that has added
+                                     // the partial puts the flag back to 0, so a launch starts from clean flags
+                                     // whatever ran before it (a replayed graph included)
   float* split_partial;              // [slot][2 blocks][N columns][128 rows]
   uint32_t* split_flags;             // [slot][2 blocks]
   PlanParams plan;
@@ -396,7 +398,7 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, int c0, int N, uint32
   tmem_ld_wait();
 }
 
-// Wait until a partial's flag carries this launch's epoch (bounded like every other wait).
+// Wait until a partial's flag holds the "complete" value (bounded like every other wait).
 __device__ __forceinline__ bool flag_wait(const uint32_t* flag, uint32_t epoch, volatile int* abort_flag) {
   uint32_t polls = 0;
   uint64_t t0 = 0;
@@ -1201,6 +1203,11 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
       }
       named_bar_sync(kPlanBarrierId, kEpilogueThreads);
+      if (kSplit && et < p.split_j) {
+        // every thread of this block has added the helpers' partials (pass 1 lies before the
+        // barrier above): their flags go back to "not ready" for whatever launch comes next
+        p.split_flags[(static_cast<size_t>(tile >> 1) * p.split_j + et) * 2 + cta_rank] = 0u;
+      }
       if (mode == kModeDispatch) {
         if (static_cast<long long>(tile) * kTileM < p.T)       // the padding block of an odd pair owns no tile
           for (int e = et; e < E; e += kEpilogueThreads)

@@ -468,10 +468,10 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   // kModeLayer: which pass this block belongs to, its tile there and its input
-  const bool second_pass = p.mode == kModeLayer && static_cast<int>(blockIdx.x) >= p.tiles_first;
-  const int mode = p.mode == kModeLayer ? (second_pass ? kModeDispatch : kModePredictPlan) : p.mode;
   const bool is_helper = kSplit && static_cast<int>(blockIdx.x) < 2 * p.split_helpers;
   const int owner_block = kSplit ? static_cast<int>(blockIdx.x) - 2 * p.split_helpers : static_cast<int>(blockIdx.x);
+  const bool second_pass = p.mode == kModeLayer && !is_helper && owner_block >= p.tiles_first;
+  const int mode = p.mode == kModeLayer ? (second_pass ? kModeDispatch : kModePredictPlan) : p.mode;
   const int tile = second_pass ? owner_block - p.tiles_first : owner_block;
   const int kb_end = kSplit ? p.split_ko : p.num_kb;        // k-blocks this block accumulates for its own tile
   const CUtensorMap* xmap = second_pass ? &tmap_x2 : &tmap_x;
@@ -537,7 +537,11 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int rest = p.num_kb - p.split_ko;
     const int tp = hp / p.split_j, piece = hp % p.split_j;
     const int kb0 = p.split_ko + rest * piece / p.split_j, kb1 = p.split_ko + rest * (piece + 1) / p.split_j;
-    const int my_tile = 2 * tp + static_cast<int>(cta_rank);
+    // (tile pairs are numbered over both passes of a layer launch; a pair never straddles them)
+    const int pair_tile = 2 * tp + static_cast<int>(cta_rank);
+    const bool helps_second = p.mode == kModeLayer && pair_tile >= p.tiles_first;
+    const int my_tile = helps_second ? pair_tile - p.tiles_first : pair_tile;
+    const CUtensorMap* hmap = helps_second ? &tmap_x2 : &tmap_x;
     if (warp == 0) {
       // ---------------------------------------------------------- TMA producer
       if (lane == 0) {
@@ -550,7 +554,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
           const uint32_t full = map_to_cta(smem_u32(&sh.full_bar[s]), 0u);
           if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&sh.full_bar[s]), 2u * stage_bytes);
-          tma_load_2d_pair(a_dst, &tmap_x, full, kb * kBlockK, my_tile * kTileM, pol_x);
+          tma_load_2d_pair(a_dst, hmap, full, kb * kBlockK, my_tile * kTileM, pol_x);
           tma_load_2d_pair(a_dst + kATileBytes, &tmap_w, full, kb * kBlockK,
                            static_cast<int32_t>(cta_rank) * (p.N / 2), pol_w);
         }
@@ -702,7 +706,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         bool ok = mbar_wait<kCtas == 2>(smem_u32(&sh.accum_bar), 0u, abort_flag);
         if (kSplit) {
           // ... and for the helpers' partial sums of this tile's remaining k-blocks
-          const int tp = tile >> 1;
+          const int tp = owner_block >> 1;
           for (int j = 0; j < p.split_j && ok; ++j)
             ok = flag_wait(p.split_flags + (static_cast<size_t>(tp) * p.split_j + j) * 2 + cta_rank, p.split_epoch, abort_flag);
         }
@@ -822,7 +826,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           if (kSplit) {
             // add the helpers' partial sums of the remaining k-blocks, piece by piece in a fixed order;
             // a partial tile is stored column by column, so the warp's 32 rows read 128 contiguous bytes
-            const int tp = tile >> 1;
+            const int tp = owner_block >> 1;
             for (int pj = 0; pj < p.split_j; ++pj) {
               const float* part = p.split_partial + partial_offset(tp * p.split_j + pj, cta_rank, N, c0) + row_in_tile;
   #pragma unroll
@@ -1206,7 +1210,7 @@ fb_router_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       if (kSplit && et < p.split_j) {
         // every thread of this block has added the helpers' partials (pass 1 lies before the
         // barrier above): their flags go back to "not ready" for whatever launch comes next
-        p.split_flags[(static_cast<size_t>(tile >> 1) * p.split_j + et) * 2 + cta_rank] = 0u;
+        p.split_flags[(static_cast<size_t>(owner_block >> 1) * p.split_j + et) * 2 + cta_rank] = 0u;
       }
       if (mode == kModeDispatch) {
         if (static_cast<long long>(tile) * kTileM < p.T)       // the padding block of an odd pair owns no tile

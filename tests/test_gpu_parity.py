@@ -361,7 +361,7 @@ def test_dsv3_full_size_every_output():
         assert rep[f"{name}_flagged_tight"] <= 0.05 * wl.T
 
 
-@pytest.mark.parametrize("name", ["sweep32k", "sweep64k"])
+@pytest.mark.parametrize("name", ["sweep32k", "sweep64k", "qwen3_b16"])     # qwen3_b16: 16 x 8K tokens, 131072 rows
 def test_long_prefill_sweep_sampled(name):
     wl = I.WORKLOADS[name]
     rows = np.random.default_rng(0).choice(wl.T, size=2048, replace=False)
